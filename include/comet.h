@@ -1,0 +1,171 @@
+/*
+ * comet.h -- C ABI of libcomet: mixed sparse x dense tensor contractions on one B200 (sm_100a),
+ * driven by per-dimension storage-level attributes.
+ *
+ * A sparse tensor is `order` storage levels. Level l stores tensor mode mode_order[l] with one of
+ * four attributes and a (pos, crd) pair of int32 arrays, plus one value array (the paper's
+ * "Tensor Storage Format" section and its sparse-tensor struct: per-dimension pos/crd of i32 and
+ * values of f64):
+ *
+ *   D  (dense)                pos = [dim] (1 entry), no crd; position = parent_position*dim + coordinate
+ *   CU (compressed, unique)   crd = the distinct coordinates under each parent position, ascending;
+ *                             pos has parents+1 entries: children of parent p are crd[pos[p] .. pos[p+1])
+ *                             (Table 1: "for i from pos[m] to pos[m+1] { idx = crd[i] }", m = the
+ *                             position produced by the level above, 0 at the first level)
+ *   CN (compressed, nonunique) first level only: crd = every entry's coordinate, pos = [0, nnz]
+ *   S  (singleton)            crd[p] = coordinate of the entry at parent position p, no pos
+ *
+ * COO = [CN,S(,S)], CSR = [D,CU], DCSR = [CU,CU], CSF = [CU,CU,CU]. Every packed format is in
+ * lexicographic order of (mode_order[0], mode_order[1], ...) coordinates. Indices are 0-based.
+ *
+ * Conventions for every entry point
+ *   - Pointers are DEVICE pointers unless the parameter name starts with h_ (host memory).
+ *   - Inputs are borrowed and never modified. Dense outputs are caller-allocated and are
+ *     OVERWRITTEN (C = A.B, not +=); rows / fibers without a stored entry become +0.0.
+ *   - Dense operands are row-major with an explicit leading dimension in elements.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream). Contractions
+ *     are asynchronous on that stream and never synchronise; comet_pack and the *_symbolic calls
+ *     synchronise the stream once to learn data-dependent sizes.
+ *   - A handle caches scratch memory and may be used from one stream at a time.
+ *   - Errors are return codes; nothing aborts, throws or traps. Errors detectable on the host are
+ *     returned before anything is launched.
+ *   - Limits: nnz, every extent and every pos value must be < 2^31 - 1 (int32 indices).
+ *   - Values are fp64 (COMET_F64). COMET_F32 is reserved and reported as unsupported.
+ */
+#ifndef COMET_H
+#define COMET_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { COMET_D = 0, COMET_CU = 1, COMET_CN = 2, COMET_S = 3 } comet_attr_t;
+typedef enum { COMET_F64 = 0, COMET_F32 = 1 } comet_dtype_t;
+
+typedef enum {
+  COMET_OK = 0,
+  COMET_ERR_INVALID_ARG = -1,        /* NULL pointer, negative size, bad enum, bad mode_order */
+  COMET_ERR_UNSUPPORTED_FORMAT = -2, /* attribute combination / dtype this entry point does not handle */
+  COMET_ERR_COORD_OUT_OF_RANGE = -3, /* an input coordinate lies outside [0, dim) */
+  COMET_ERR_DUPLICATE_COORD = -4,    /* two input entries share all coordinates */
+  COMET_ERR_INDEX_OVERFLOW = -5,     /* nnz or an extent does not fit int32 */
+  COMET_ERR_ALLOC = -6,              /* the allocator returned NULL */
+  COMET_ERR_CUDA = -7,               /* a CUDA runtime call failed; see comet_last_cuda_error */
+  COMET_ERR_WORKSPACE = -8,          /* a fixed-size workspace is too small for this problem */
+  COMET_ERR_MISALIGNED = -9,         /* a pointer is not aligned to its element type */
+  COMET_ERR_INVALID_TENSOR = -10     /* comet_validate: pos/crd arrays violate the level invariants */
+} comet_status_t;
+
+#define COMET_MAX_ORDER 4
+
+/* The sparse tensor descriptor (a plain struct the caller may also fill in by hand for arrays it
+ * built itself; run comet_validate on such a tensor before contracting it). */
+typedef struct {
+  int32_t order;
+  int32_t dtype;                        /* comet_dtype_t of val */
+  int64_t dims[COMET_MAX_ORDER];        /* extent of tensor MODE m (not of level m) */
+  int32_t mode_order[COMET_MAX_ORDER];  /* storage level l holds tensor mode mode_order[l] */
+  int32_t attr[COMET_MAX_ORDER];        /* comet_attr_t per level */
+  int32_t *pos[COMET_MAX_ORDER];        /* device; D: 1 entry; CU: parents+1; CN: 2; S: NULL */
+  int64_t pos_len[COMET_MAX_ORDER];
+  int32_t *crd[COMET_MAX_ORDER];        /* device; D: NULL; CU: #nodes; CN, S: #positions */
+  int64_t crd_len[COMET_MAX_ORDER];
+  void *val;                            /* device; nnz values in leaf order */
+  int64_t nnz;
+  void *owner;                          /* non-NULL: arrays were allocated by the library (see comet_sptensor_free) */
+} comet_sptensor_t;
+
+typedef struct comet_context *comet_handle_t;
+
+/* Device-memory allocator used for library-owned outputs (packed tensors, symbolic outputs) and
+ * scratch. alloc returns a device pointer aligned to at least 256 bytes, or NULL. Both callbacks
+ * may be called from any comet_* call and must not call back into the library. */
+typedef struct {
+  void *(*alloc)(void *ctx, size_t bytes, void *stream);
+  void (*free)(void *ctx, void *ptr, void *stream);
+  void *ctx;
+} comet_allocator_t;
+
+/* Create / destroy a handle on the current CUDA device. `allocator` may be NULL: cudaMalloc/cudaFree
+ * are then used. Returns COMET_ERR_INVALID_ARG for a NULL out-pointer, COMET_ERR_CUDA if no device. */
+comet_status_t comet_create(comet_handle_t *handle, const comet_allocator_t *allocator);
+comet_status_t comet_destroy(comet_handle_t handle);
+const char *comet_status_string(comet_status_t status);
+/* The cudaError_t (as int) of the last failing CUDA call seen by this handle, 0 if none. */
+int comet_last_cuda_error(comet_handle_t handle);
+
+/* COO -> packed format (the format conversion the paper's input-reading runtime function performs
+ * after reading a COO file; Tensor Storage Format section for what each level holds).
+ *   h_dims[order]       extents per tensor mode
+ *   h_coo_crd[order]    HOST array of DEVICE pointers, one int32[nnz] coordinate array per mode
+ *   coo_val             DEVICE, nnz values, copied bitwise into leaf order
+ *   h_mode_order[order] a permutation of 0..order-1; h_attr[order] one comet_attr_t per level
+ * Supported attribute tuples: [CN,S,...,S], [CU,...,CU], [D,CU,...,CU] (orders 2..4), provided the
+ * coordinate bit widths sum to <= 64. Input order is arbitrary; duplicates and out-of-range
+ * coordinates are detected on the device and reported (COMET_ERR_DUPLICATE_COORD,
+ * COMET_ERR_COORD_OUT_OF_RANGE); `out` is then left zeroed. On success `out` owns its arrays
+ * (allocated through the handle's allocator) until comet_sptensor_free. Synchronises `stream` once. */
+comet_status_t comet_pack(comet_handle_t handle, int32_t order, const int64_t *h_dims, int64_t nnz,
+                          const int32_t *const *h_coo_crd, const void *coo_val, comet_dtype_t dtype,
+                          const int32_t *h_mode_order, const int32_t *h_attr, void *stream,
+                          comet_sptensor_t *out);
+
+/* Releases the arrays of a library-owned tensor (no-op for caller-built descriptors) and zeroes it. */
+comet_status_t comet_sptensor_free(comet_handle_t handle, comet_sptensor_t *tensor, void *stream);
+
+/* Checks a caller-built descriptor against the level invariants (the paper keeps the caller's layout
+ * and only describes it with attributes): pos monotone from 0 to the level's crd length, CU
+ * coordinates strictly ascending inside each parent, every coordinate inside its extent.
+ * Synchronises `stream`; returns COMET_ERR_INVALID_TENSOR on a violation. */
+comet_status_t comet_validate(comet_handle_t handle, const comet_sptensor_t *tensor, void *stream);
+
+/* SpMV  y_i = sum_j A_ij x_j  (SpMV definition in the Sparse Tensor Operations subsection).
+ * A: 2 levels, [D,CU] (CSR), [CU,CU] (DCSR) or [CN,S] (COO). x: dims[mode_order[1]] values;
+ * y: dims[mode_order[0]] values, every entry written. */
+comet_status_t comet_spmv(comet_handle_t handle, const comet_sptensor_t *A, const void *x, void *y, void *stream);
+
+/* SpMM  C_ir = sum_j A_ij B_jr  (SpMM definition). B: dims[mode_order[1]] x R, leading dimension
+ * ldb >= R; C: dims[mode_order[0]] x R, leading dimension ldc >= R; every row of C is written.
+ * Formats as for comet_spmv. Any R >= 1; R in {2,4,8,16,32,64,128} with 16-byte-aligned rows takes
+ * the vectorised path. */
+comet_status_t comet_spmm(comet_handle_t handle, const comet_sptensor_t *A, const void *B, int64_t R, int64_t ldb,
+                          void *C, int64_t ldc, void *stream);
+
+/* TTV  Y = X x_n v  (SpTTV definition; `mode` = n, 0-based, must be the mode of X's LAST level).
+ * X: 3 levels, [CU,CU,CU] (CSF) or [CN,S,S] (COO). The result is sparse, one order lower:
+ * comet_ttv_symbolic builds its structure over (mode_order[0], mode_order[1]) with level attributes
+ * h_out_attr = {D,CU} (CSR) or {CU,CU} (DCSR); values are then (re)computed by comet_ttv, which
+ * writes only Y->val. The structure depends on X's structure alone, never on values. Y owns its
+ * arrays; X need not outlive it. comet_ttv_symbolic synchronises `stream` once for COO inputs. */
+comet_status_t comet_ttv_symbolic(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode,
+                                  const int32_t *h_out_attr, void *stream, comet_sptensor_t *Y);
+comet_status_t comet_ttv(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode, const void *v,
+                         comet_sptensor_t *Y, void *stream);
+
+/* TTM  Y = X x_n U, U in R^{I_n x R} with rows indexed by the contracted mode (SpTTM definition);
+ * mode n is replaced by r in place. `mode` must be the mode of X's last level. The result is
+ * semi-sparse [CU,CU,D]: its two sparse levels equal X's first two levels and every stored fiber is
+ * a dense row of R values (val is #fibers x R, row-major). comet_ttm_symbolic builds that structure,
+ * comet_ttm writes only Y->val. */
+comet_status_t comet_ttm_symbolic(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode, int64_t R,
+                                  void *stream, comet_sptensor_t *Y);
+comet_status_t comet_ttm(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode, const void *U, int64_t R,
+                         int64_t ldu, comet_sptensor_t *Y, void *stream);
+
+/* MTTKRP  out_{i_n r} = sum x_{i1 i2 i3} P_{p r} Q_{q r} over the two other modes p < q (the paper
+ * names the operation without defining it; this is the textbook matricised-tensor-times-Khatri-Rao
+ * product). `mode` = n must be the mode of X's FIRST level. X: [CN,S,S] (COO) or [CU,CU,CU] (CSF).
+ *   h_factors[3]  HOST array of DEVICE pointers, factor of mode m is dims[m] x R with leading
+ *                 dimension h_ld[m]; the entry at `mode` is ignored
+ *   out           dims[mode] x R, leading dimension ldo, every row written. */
+comet_status_t comet_mttkrp(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode,
+                            const void *const *h_factors, const int64_t *h_ld, int64_t R, void *out, int64_t ldo,
+                            void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COMET_H */

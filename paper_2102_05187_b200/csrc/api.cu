@@ -1,0 +1,296 @@
+// extern "C" entry points for the contractions: descriptor checks, dispatch on the level attributes
+// (the role Table 1 of the paper plays for its loop generator), symbolic output construction.
+#include "common.cuh"
+#include "kernels.cuh"
+
+#include <string.h>
+
+#include <new>
+
+using namespace comet;
+
+namespace {
+
+constexpr int64_t kIndexLimit = 2147483646;   // sizes must be < 2^31 - 1
+
+bool is_fmt(const comet_sptensor_t *t, int order, int a0, int a1, int a2 = -1) {
+  if (t->order != order) return false;
+  if (t->attr[0] != a0 || t->attr[1] != a1) return false;
+  return order < 3 || t->attr[2] == a2;
+}
+
+comet_status_t check_tensor(const comet_sptensor_t *t, int order) {
+  if (!t) return COMET_ERR_INVALID_ARG;
+  if (t->order != order) return COMET_ERR_UNSUPPORTED_FORMAT;
+  if (t->dtype != COMET_F64) return COMET_ERR_UNSUPPORTED_FORMAT;
+  if (t->nnz < 0) return COMET_ERR_INVALID_ARG;
+  if (t->nnz > kIndexLimit) return COMET_ERR_INDEX_OVERFLOW;
+  bool seen[COMET_MAX_ORDER] = {false, false, false, false};
+  for (int l = 0; l < order; ++l) {
+    const int m = t->mode_order[l];
+    if (m < 0 || m >= order || seen[m]) return COMET_ERR_INVALID_ARG;
+    seen[m] = true;
+    if (t->dims[l] < 0) return COMET_ERR_INVALID_ARG;
+    if (t->dims[l] > kIndexLimit) return COMET_ERR_INDEX_OVERFLOW;
+    const int a = t->attr[l];
+    if (a < COMET_D || a > COMET_S) return COMET_ERR_INVALID_ARG;
+    if ((a == COMET_CU || a == COMET_CN) && !t->pos[l]) return COMET_ERR_INVALID_ARG;
+    if (a != COMET_D && t->crd_len[l] > 0 && !t->crd[l]) return COMET_ERR_INVALID_ARG;
+  }
+  if (t->nnz > 0 && !t->val) return COMET_ERR_INVALID_ARG;
+  return COMET_OK;
+}
+
+bool misaligned8(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 7) != 0; }
+
+struct Owner {           // bookkeeping of a library-owned tensor: the blocks to release
+  int count;
+  void *blocks[2 * COMET_MAX_ORDER + 1];
+};
+
+void *owned_alloc(Context *ctx, Owner *o, size_t bytes, cudaStream_t stream) {
+  void *p = ctx_alloc(ctx, bytes, stream);
+  if (p) o->blocks[o->count++] = p;
+  return p;
+}
+
+void release(Context *ctx, Owner *o, cudaStream_t stream) {
+  if (!o) return;
+  for (int b = 0; b < o->count; ++b) ctx_free(ctx, o->blocks[b], stream);
+  delete o;
+}
+
+// pos of a CSR output from a compressed root level: out[i] = pos1[#stored root coordinates < i]
+__global__ void expand_root_pos_kernel(const int32_t *__restrict__ crd0, const int32_t *__restrict__ pos1, int64_t S,
+                                       int64_t rows, int32_t *__restrict__ out) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i > rows) return;
+  int64_t lo = 0, hi = S;
+  while (lo < hi) {
+    const int64_t mid = (lo + hi) >> 1;
+    if ((int64_t)crd0[mid] < i) lo = mid + 1; else hi = mid;
+  }
+  out[i] = pos1[lo];
+}
+
+__global__ void set_word_kernel(int32_t *p, int32_t v) { *p = v; }
+
+}  // namespace
+
+namespace comet {
+void *owner_new() { Owner *o = new (std::nothrow) Owner(); if (o) o->count = 0; return o; }
+void *owner_alloc(Context *ctx, void *owner, size_t bytes, cudaStream_t stream) {
+  return owned_alloc(ctx, static_cast<Owner *>(owner), bytes, stream);
+}
+void owner_release(Context *ctx, void *owner, cudaStream_t stream) { release(ctx, static_cast<Owner *>(owner), stream); }
+}  // namespace comet
+
+extern "C" comet_status_t comet_sptensor_free(comet_handle_t handle, comet_sptensor_t *t, void *stream) {
+  if (!handle || !t) return COMET_ERR_INVALID_ARG;
+  Context *ctx = reinterpret_cast<Context *>(handle);
+  if (t->owner) release(ctx, static_cast<Owner *>(t->owner), (cudaStream_t)stream);
+  memset(t, 0, sizeof(*t));
+  return COMET_OK;
+}
+
+// ------------------------------------------------------------------------------------------ SpMV / SpMM
+extern "C" comet_status_t comet_spmv(comet_handle_t handle, const comet_sptensor_t *A, const void *x, void *y,
+                                     void *stream) {
+  if (!handle || !x || !y) return COMET_ERR_INVALID_ARG;
+  comet_status_t st = check_tensor(A, 2);
+  if (st != COMET_OK) return st;
+  if (misaligned8(x) || misaligned8(y)) return COMET_ERR_MISALIGNED;
+  Context *ctx = reinterpret_cast<Context *>(handle);
+  cudaStream_t s = (cudaStream_t)stream;
+  const int64_t rows = A->dims[A->mode_order[0]];
+  if (is_fmt(A, 2, COMET_D, COMET_CU))
+    return seg_dot(ctx, A->pos[1] + 1, A->crd[1], (const double *)A->val, rows, A->nnz, (const double *)x,
+                   (double *)y, nullptr, rows, s);
+  if (is_fmt(A, 2, COMET_CU, COMET_CU))
+    return seg_dot(ctx, A->pos[1] + 1, A->crd[1], (const double *)A->val, A->crd_len[0], A->nnz, (const double *)x,
+                   (double *)y, A->crd[0], rows, s);
+  return COMET_ERR_UNSUPPORTED_FORMAT;
+}
+
+extern "C" comet_status_t comet_spmm(comet_handle_t handle, const comet_sptensor_t *A, const void *B, int64_t R,
+                                     int64_t ldb, void *C, int64_t ldc, void *stream) {
+  if (!handle || !B || !C || R < 1 || ldb < R || ldc < R) return COMET_ERR_INVALID_ARG;
+  comet_status_t st = check_tensor(A, 2);
+  if (st != COMET_OK) return st;
+  if (misaligned8(B) || misaligned8(C)) return COMET_ERR_MISALIGNED;
+  Context *ctx = reinterpret_cast<Context *>(handle);
+  cudaStream_t s = (cudaStream_t)stream;
+  const int64_t rows = A->dims[A->mode_order[0]];
+  if (is_fmt(A, 2, COMET_D, COMET_CU))
+    return seg_gather(ctx, A->pos[1] + 1, A->crd[1], (const double *)A->val, rows, A->nnz, (const double *)B, ldb, R,
+                      (double *)C, ldc, nullptr, rows, s);
+  if (is_fmt(A, 2, COMET_CU, COMET_CU)) {
+    if (A->crd_len[0] == 0) return zero_rows(ctx, (double *)C, rows, R, ldc, s);
+    return seg_gather(ctx, A->pos[1] + 1, A->crd[1], (const double *)A->val, A->crd_len[0], A->nnz,
+                      (const double *)B, ldb, R, (double *)C, ldc, A->crd[0], rows, s);
+  }
+  return COMET_ERR_UNSUPPORTED_FORMAT;
+}
+
+// ------------------------------------------------------------------------------------------ TTV / TTM
+static comet_status_t check_last_mode(const comet_sptensor_t *X, int32_t mode) {
+  comet_status_t st = check_tensor(X, 3);
+  if (st != COMET_OK) return st;
+  if (mode < 0 || mode > 2) return COMET_ERR_INVALID_ARG;
+  if (!is_fmt(X, 3, COMET_CU, COMET_CU, COMET_CU)) return COMET_ERR_UNSUPPORTED_FORMAT;
+  if (X->mode_order[2] != mode) return COMET_ERR_UNSUPPORTED_FORMAT;   // re-pack with the contracted mode last
+  return COMET_OK;
+}
+
+// Copies X's two upper levels into Y (levels 0 and 1), device to device.
+static comet_status_t copy_upper_levels(Context *ctx, const comet_sptensor_t *X, comet_sptensor_t *Y, Owner *o,
+                                        cudaStream_t s) {
+  for (int l = 0; l < 2; ++l) {
+    Y->pos_len[l] = X->pos_len[l];
+    Y->crd_len[l] = X->crd_len[l];
+    Y->pos[l] = (int32_t *)owned_alloc(ctx, o, (size_t)X->pos_len[l] * 4, s);
+    Y->crd[l] = (int32_t *)owned_alloc(ctx, o, (size_t)X->crd_len[l] * 4, s);
+    if (!Y->pos[l] || !Y->crd[l]) return COMET_ERR_ALLOC;
+    if (X->pos_len[l])
+      COMET_CUDA_TRY(ctx, cudaMemcpyAsync(Y->pos[l], X->pos[l], (size_t)X->pos_len[l] * 4, cudaMemcpyDeviceToDevice, s));
+    if (X->crd_len[l])
+      COMET_CUDA_TRY(ctx, cudaMemcpyAsync(Y->crd[l], X->crd[l], (size_t)X->crd_len[l] * 4, cudaMemcpyDeviceToDevice, s));
+  }
+  return COMET_OK;
+}
+
+extern "C" comet_status_t comet_ttv_symbolic(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode,
+                                             const int32_t *h_out_attr, void *stream, comet_sptensor_t *Y) {
+  if (!handle || !Y || !h_out_attr) return COMET_ERR_INVALID_ARG;
+  comet_status_t st = check_last_mode(X, mode);
+  if (st != COMET_OK) return st;
+  const bool csr = h_out_attr[0] == COMET_D && h_out_attr[1] == COMET_CU;
+  const bool dcsr = h_out_attr[0] == COMET_CU && h_out_attr[1] == COMET_CU;
+  if (!csr && !dcsr) return COMET_ERR_UNSUPPORTED_FORMAT;
+  Context *ctx = reinterpret_cast<Context *>(handle);
+  cudaStream_t s = (cudaStream_t)stream;
+  memset(Y, 0, sizeof(*Y));
+  Owner *o = static_cast<Owner *>(owner_new());
+  if (!o) return COMET_ERR_ALLOC;
+  const int64_t S = X->crd_len[0], F = X->crd_len[1];
+  const int64_t rows = X->dims[X->mode_order[0]];
+  Y->order = 2;
+  Y->dtype = COMET_F64;
+  Y->dims[0] = rows;
+  Y->dims[1] = X->dims[X->mode_order[1]];
+  Y->mode_order[0] = 0;
+  Y->mode_order[1] = 1;
+  Y->attr[0] = h_out_attr[0];
+  Y->attr[1] = h_out_attr[1];
+  Y->nnz = F;
+  st = COMET_OK;
+  if (dcsr) {
+    st = copy_upper_levels(ctx, X, Y, o, s);
+  } else {
+    Y->pos_len[0] = 1; Y->crd_len[0] = 0; Y->pos_len[1] = rows + 1; Y->crd_len[1] = F;
+    Y->pos[0] = (int32_t *)owned_alloc(ctx, o, 4, s);
+    Y->pos[1] = (int32_t *)owned_alloc(ctx, o, (size_t)(rows + 1) * 4, s);
+    Y->crd[1] = (int32_t *)owned_alloc(ctx, o, (size_t)F * 4, s);
+    if (!Y->pos[0] || !Y->pos[1] || !Y->crd[1]) st = COMET_ERR_ALLOC;
+    if (st == COMET_OK) {
+      set_word_kernel<<<1, 1, 0, s>>>(Y->pos[0], (int32_t)rows);
+      expand_root_pos_kernel<<<(unsigned)ceil_div(rows + 1, 256), 256, 0, s>>>(X->crd[0], X->pos[1], S, rows, Y->pos[1]);
+      cudaError_t e = cudaGetLastError();
+      if (e == cudaSuccess && F)
+        e = cudaMemcpyAsync(Y->crd[1], X->crd[1], (size_t)F * 4, cudaMemcpyDeviceToDevice, s);
+      if (e != cudaSuccess) st = cuda_fail(ctx, e);
+    }
+  }
+  if (st == COMET_OK) {
+    Y->val = owned_alloc(ctx, o, (size_t)F * sizeof(double), s);
+    if (!Y->val) st = COMET_ERR_ALLOC;
+  }
+  if (st != COMET_OK) { release(ctx, o, s); memset(Y, 0, sizeof(*Y)); return st; }
+  Y->owner = o;
+  return COMET_OK;
+}
+
+extern "C" comet_status_t comet_ttv(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode, const void *v,
+                                    comet_sptensor_t *Y, void *stream) {
+  if (!handle || !v || !Y) return COMET_ERR_INVALID_ARG;
+  comet_status_t st = check_last_mode(X, mode);
+  if (st != COMET_OK) return st;
+  if (Y->order != 2 || Y->nnz != X->crd_len[1] || (Y->nnz > 0 && !Y->val)) return COMET_ERR_INVALID_ARG;
+  if (misaligned8(v)) return COMET_ERR_MISALIGNED;
+  Context *ctx = reinterpret_cast<Context *>(handle);
+  return seg_dot(ctx, X->pos[2] + 1, X->crd[2], (const double *)X->val, X->crd_len[1], X->nnz, (const double *)v,
+                 (double *)Y->val, nullptr, X->crd_len[1], (cudaStream_t)stream);
+}
+
+extern "C" comet_status_t comet_ttm_symbolic(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode,
+                                             int64_t R, void *stream, comet_sptensor_t *Y) {
+  if (!handle || !Y || R < 1) return COMET_ERR_INVALID_ARG;
+  if (R > kIndexLimit) return COMET_ERR_INDEX_OVERFLOW;
+  comet_status_t st = check_last_mode(X, mode);
+  if (st != COMET_OK) return st;
+  Context *ctx = reinterpret_cast<Context *>(handle);
+  cudaStream_t s = (cudaStream_t)stream;
+  memset(Y, 0, sizeof(*Y));
+  Owner *o = static_cast<Owner *>(owner_new());
+  if (!o) return COMET_ERR_ALLOC;
+  const int64_t F = X->crd_len[1];
+  Y->order = 3;
+  Y->dtype = COMET_F64;
+  for (int m = 0; m < 3; ++m) { Y->dims[m] = X->dims[m]; Y->mode_order[m] = X->mode_order[m]; }
+  Y->dims[mode] = R;                      // mode n is replaced by r in place
+  Y->attr[0] = COMET_CU; Y->attr[1] = COMET_CU; Y->attr[2] = COMET_D;
+  Y->nnz = F * R;
+  st = copy_upper_levels(ctx, X, Y, o, s);
+  if (st == COMET_OK) {
+    Y->pos_len[2] = 1;
+    Y->pos[2] = (int32_t *)owned_alloc(ctx, o, 4, s);
+    Y->val = owned_alloc(ctx, o, (size_t)F * R * sizeof(double), s);
+    if (!Y->pos[2] || !Y->val) st = COMET_ERR_ALLOC;
+    else {
+      set_word_kernel<<<1, 1, 0, s>>>(Y->pos[2], (int32_t)R);
+      cudaError_t e = cudaGetLastError();
+      if (e != cudaSuccess) st = cuda_fail(ctx, e);
+    }
+  }
+  if (st != COMET_OK) { release(ctx, o, s); memset(Y, 0, sizeof(*Y)); return st; }
+  Y->owner = o;
+  return COMET_OK;
+}
+
+extern "C" comet_status_t comet_ttm(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode, const void *U,
+                                    int64_t R, int64_t ldu, comet_sptensor_t *Y, void *stream) {
+  if (!handle || !U || !Y || R < 1 || ldu < R) return COMET_ERR_INVALID_ARG;
+  comet_status_t st = check_last_mode(X, mode);
+  if (st != COMET_OK) return st;
+  const int64_t F = X->crd_len[1];
+  if (Y->order != 3 || Y->nnz != F * R || (Y->nnz > 0 && !Y->val)) return COMET_ERR_INVALID_ARG;
+  if (misaligned8(U)) return COMET_ERR_MISALIGNED;
+  Context *ctx = reinterpret_cast<Context *>(handle);
+  return seg_gather(ctx, X->pos[2] + 1, X->crd[2], (const double *)X->val, F, X->nnz, (const double *)U, ldu, R,
+                    (double *)Y->val, R, nullptr, F, (cudaStream_t)stream);
+}
+
+// ------------------------------------------------------------------------------------------ MTTKRP
+extern "C" comet_status_t comet_mttkrp(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode,
+                                       const void *const *h_factors, const int64_t *h_ld, int64_t R, void *out,
+                                       int64_t ldo, void *stream) {
+  if (!handle || !h_factors || !h_ld || !out || R < 1 || ldo < R) return COMET_ERR_INVALID_ARG;
+  comet_status_t st = check_tensor(X, 3);
+  if (st != COMET_OK) return st;
+  if (mode < 0 || mode > 2) return COMET_ERR_INVALID_ARG;
+  if (X->mode_order[0] != mode) return COMET_ERR_UNSUPPORTED_FORMAT;   // re-pack with the output mode first
+  const int m1 = X->mode_order[1], m2 = X->mode_order[2];
+  if (!h_factors[m1] || !h_factors[m2] || h_ld[m1] < R || h_ld[m2] < R) return COMET_ERR_INVALID_ARG;
+  if (misaligned8(h_factors[m1]) || misaligned8(h_factors[m2]) || misaligned8(out)) return COMET_ERR_MISALIGNED;
+  Context *ctx = reinterpret_cast<Context *>(handle);
+  cudaStream_t s = (cudaStream_t)stream;
+  const int64_t rows = X->dims[mode];
+  const double *P = (const double *)h_factors[m1], *Q = (const double *)h_factors[m2];
+  if (is_fmt(X, 3, COMET_CN, COMET_S, COMET_S))
+    return mttkrp_coo(ctx, X->crd[0], X->crd[1], X->crd[2], (const double *)X->val, X->nnz, rows, P, h_ld[m1], Q,
+                      h_ld[m2], R, (double *)out, ldo, s);
+  if (is_fmt(X, 3, COMET_CU, COMET_CU, COMET_CU))
+    return mttkrp_csf(ctx, X->pos[1], X->crd[0], X->crd[1], X->pos[2], X->crd[2], (const double *)X->val,
+                      X->crd_len[0], X->crd_len[1], X->nnz, rows, P, h_ld[m1], Q, h_ld[m2], R, (double *)out, ldo, s);
+  return COMET_ERR_UNSUPPORTED_FORMAT;
+}

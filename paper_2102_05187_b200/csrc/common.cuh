@@ -1,0 +1,65 @@
+// Shared device/host helpers of libcomet (sm_100a). Internal: not part of the C ABI.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/comet.h"
+
+namespace comet {
+
+constexpr int kSmCount = 148;            // B200: 2 dies x 74 SMs; grids are sized against this
+constexpr int kBlockThreads = 256;
+
+struct Context {
+  comet_allocator_t allocator;            // user allocator or the cudaMalloc fallback
+  bool user_allocator;
+  int device;
+  int last_cuda_error;
+  void *scratch;                          // cached scratch, grown on demand
+  size_t scratch_bytes;
+  int32_t *h_pinned;                      // small pinned buffer for device->host size reads
+  int32_t *d_status;                      // device words written by checking kernels
+};
+
+// Grows the cached scratch buffer to at least `bytes` and returns it (NULL on allocation failure).
+void *scratch_get(Context *ctx, size_t bytes, cudaStream_t stream);
+void *ctx_alloc(Context *ctx, size_t bytes, cudaStream_t stream);
+void ctx_free(Context *ctx, void *p, cudaStream_t stream);
+comet_status_t cuda_fail(Context *ctx, cudaError_t e);
+
+#define COMET_CUDA_TRY(ctx, expr)                         \
+  do {                                                    \
+    cudaError_t e__ = (expr);                             \
+    if (e__ != cudaSuccess) return cuda_fail((ctx), e__); \
+  } while (0)
+
+#define COMET_LAUNCH_CHECK(ctx) COMET_CUDA_TRY((ctx), cudaGetLastError())
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// ------------------------------------------------------------------------------------------------
+// device helpers
+
+// Streaming (read-once) loads: evict-first so that index/value streams do not displace the dense
+// operand rows that are re-used out of L2.
+__device__ __forceinline__ int32_t ld_stream(const int32_t *p) { return __ldcs(p); }
+__device__ __forceinline__ double ld_stream(const double *p) { return __ldcs(p); }
+
+// Merge-path split: the merge list interleaves segment-end markers (segment s ends at leaf position
+// seg_end[s]) with the leaf positions 0..N-1; at state (i, j) the next item is leaf j if
+// j < seg_end[i], else the end marker of segment i. Marker s is therefore item number seg_end[s] + s.
+// Returns how many markers lie among the first `diag` items; the leaf count is diag minus that.
+__device__ __forceinline__ int64_t merge_path_segments(const int32_t *__restrict__ seg_end, int64_t M, int64_t N,
+                                                       int64_t diag) {
+  int64_t lo = diag > N ? diag - N : 0;
+  int64_t hi = diag < M ? diag : M;
+  while (lo < hi) {
+    int64_t mid = (lo + hi) >> 1;
+    if ((int64_t)__ldg(seg_end + mid) + mid < diag) lo = mid + 1; else hi = mid;
+  }
+  return lo;
+}
+
+}  // namespace comet

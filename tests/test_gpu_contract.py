@@ -1,0 +1,244 @@
+"""GPU parity: every contraction of the CUDA library against the CPU oracle, element by element, on
+the same seeded inputs. Structure arrays come from the oracle's packing here (caller-built
+descriptors), so these tests isolate the contraction kernels; test_gpu_pack.py covers the packing."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+from oracle import D, CU, CN, S
+
+pytestmark = pytest.mark.gpu
+
+comet = pytest.importorskip("paper_2102_05187_b200")
+from gpu_util import FP64_TOL, assert_close, assert_equal_arrays, dev, upload_packed  # noqa: E402
+
+
+def _np(coords):
+    return [c.numpy() for c in coords]
+
+
+@pytest.fixture(autouse=True)
+def _need_gpu(cuda_device):
+    yield
+
+
+@pytest.fixture(params=[None, 8, 37])
+def tile_items(request, monkeypatch):
+    """Default tiling, and tiny / odd tiles so that segments straddle many tiles (carry path)."""
+    if request.param is None:
+        monkeypatch.delenv("COMET_TILE_ITEMS", raising=False)
+    else:
+        monkeypatch.setenv("COMET_TILE_ITEMS", str(request.param))
+    return request.param
+
+
+def test_worked_example():
+    mc = ([0, 0, 2, 2, 2, 3], [1, 4, 0, 1, 5, 3])
+    mv = [1.0, 2.0, 3.0, 4.0, 5.0, 6.0]
+    for attr in [(D, CU), (CU, CU)]:
+        A = upload_packed(oracle.pack(mc, mv, (4, 6), (0, 1), attr))
+        y = comet.spmv(A, dev([1.0, 2, 3, 4, 5, 6]))
+        assert y.tolist() == [12.0, 0.0, 41.0, 24.0]
+        Y = comet.spmm(A, dev(np.arange(12.0).reshape(6, 2)))
+        assert Y.tolist() == [[18, 21], [0, 0], [58, 70], [36, 42]]
+    tc = ([0, 0, 0, 2, 2, 2, 2], [0, 0, 2, 1, 1, 2, 2], [1, 3, 0, 1, 2, 0, 3])
+    tv = [1.0, 2.0, 3.0, 4.0, 5.0, 6.0, 7.0]
+    X = upload_packed(oracle.pack(tc, tv, (3, 3, 4), (0, 1, 2), (CU, CU, CU)))
+    Y = comet.ttv(X, 2, dev([1.0, 10, 100, 1000]))
+    assert Y.val.tolist() == [2010.0, 3.0, 540.0, 7006.0]
+    assert Y.pos(1).tolist() == [0, 2, 2, 4] and Y.crd(1).tolist() == [0, 2, 1, 2] and Y.pos(0).tolist() == [3]
+    Z = comet.ttm(X, 2, dev(np.array([[1.0, 0], [0, 1], [1, 1], [2, -1]])))
+    assert Z.val.reshape(4, 2).tolist() == [[4, -1], [3, 0], [5, 9], [20, -7]]
+    assert Z.attr == (CU, CU, D) and Z.dims == (3, 3, 2) and Z.pos(2).tolist() == [2]
+    assert Z.crd(0).tolist() == [0, 2] and Z.pos(1).tolist() == [0, 2, 4] and Z.crd(1).tolist() == [0, 2, 1, 2]
+    F = [None, dev(np.array([[1.0, 2], [3, 4], [5, 6]])), dev(np.array([[1.0, -1], [2, 0], [0, 1], [1, 1]]))]
+    for attr in [(CU, CU, CU), (CN, S, S)]:
+        X = upload_packed(oracle.pack(tc, tv, (3, 3, 4), (0, 1, 2), attr))
+        assert comet.mttkrp(X, 0, F).tolist() == [[19, -14], [0, 0], [89, 26]]
+
+
+MATRIX_CASES = [((64, 48), 700, 1), ((300, 200), 5000, 2), ((1, 500), 300, 3), ((500, 1), 200, 4),
+                ((40, 40), 1600, 5), ((200, 300), 1, 6), ((200, 300), 0, 7), ((3000, 100), 400, 8)]
+
+
+@pytest.mark.parametrize("dims,nnz,seed", MATRIX_CASES)
+@pytest.mark.parametrize("attr", [(D, CU), (CU, CU)])
+def test_spmv(dims, nnz, seed, attr, tile_items):
+    coords, val = synth.random_coo(dims, nnz, seed)
+    c, v = _np(coords), val.numpy()
+    x = synth.random_dense((dims[1],), seed).numpy()
+    want, norm = oracle.spmv(c, v, dims, x)
+    A = upload_packed(oracle.pack(c, v, dims, (0, 1), attr))
+    y = torch.full((dims[0],), float("nan"), dtype=torch.float64, device="cuda")   # every entry must be written
+    comet.spmv(A, dev(x), y)
+    assert_close(y, want, norm, what="spmv")
+
+
+@pytest.mark.parametrize("dims,nnz,seed", MATRIX_CASES)
+@pytest.mark.parametrize("attr", [(D, CU), (CU, CU)])
+@pytest.mark.parametrize("R", [1, 2, 3, 8, 16, 17, 32, 64, 100, 128, 130])
+def test_spmm(dims, nnz, seed, attr, R, tile_items):
+    if tile_items == 37 and R not in (2, 17, 64):
+        pytest.skip("odd tiling is sampled on a few widths")
+    coords, val = synth.random_coo(dims, nnz, seed)
+    c, v = _np(coords), val.numpy()
+    B = synth.random_dense((dims[1], R), seed).numpy()
+    want, norm = oracle.spmm(c, v, dims, B)
+    A = upload_packed(oracle.pack(c, v, dims, (0, 1), attr))
+    C = torch.full((dims[0], R), float("nan"), dtype=torch.float64, device="cuda")
+    comet.spmm(A, dev(B), C)
+    assert_close(C, want, norm, what=f"spmm R={R}")
+
+
+def test_spmm_strided_and_unaligned_operands():
+    dims, R = (120, 90), 16
+    coords, val = synth.random_coo(dims, 1500, 3)
+    c, v = _np(coords), val.numpy()
+    B = synth.random_dense((dims[1], R), 3).numpy()
+    want, norm = oracle.spmm(c, v, dims, B)
+    A = upload_packed(oracle.pack(c, v, dims, (0, 1), (D, CU)))
+    for ldb, ldc, off in [(R + 4, R + 2, 0), (R + 1, R + 3, 0), (R, R, 1)]:
+        Bbuf = torch.zeros(dims[1] * ldb + 8, dtype=torch.float64, device="cuda")
+        Bd = Bbuf[off:off + dims[1] * ldb].view(dims[1], ldb)[:, :R]
+        Bd.copy_(dev(B))
+        Cbuf = torch.full((dims[0] * ldc + 8,), 7.0, dtype=torch.float64, device="cuda")
+        Cd = Cbuf[off:off + dims[0] * ldc].view(dims[0], ldc)[:, :R]
+        comet.spmm(A, Bd, Cd)
+        assert_close(Cd, want, norm, what=f"spmm ld=({ldb},{ldc}) off={off}")
+        if ldc > R:
+            assert bool((Cbuf[off:off + dims[0] * ldc].view(dims[0], ldc)[:, R:] == 7.0).all())   # padding untouched
+
+
+def test_exact_on_small_integers():
+    dims = (90, 70)
+    coords, val = synth.random_coo(dims, 2500, 11, integer_values=True)
+    c, v = _np(coords), val.numpy()
+    B = synth.random_dense((dims[1], 32), 11, integer_values=True).numpy()
+    want, _ = oracle.spmm(c, v, dims, B)
+    A = upload_packed(oracle.pack(c, v, dims, (0, 1), (D, CU)))
+    assert_equal_arrays(comet.spmm(A, dev(B)), want, "integer spmm")
+    assert_equal_arrays(comet.spmv(A, dev(B[:, 0].copy())), want[:, 0], "integer spmv")
+
+
+TENSOR_CASES = [((20, 18, 16), 900, 1), ((50, 40, 30), 6000, 2), ((1, 30, 30), 300, 3), ((30, 1, 30), 300, 4),
+                ((30, 30, 1), 300, 5), ((12, 11, 10), 1320, 6), ((40, 40, 40), 1, 7), ((40, 40, 40), 0, 8),
+                ((2000, 5, 7), 500, 9)]
+
+
+@pytest.mark.parametrize("dims,nnz,seed", TENSOR_CASES)
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_ttv_ttm(dims, nnz, seed, mode, tile_items):
+    coords, val = synth.random_coo(dims, nnz, seed)
+    c, v = _np(coords), val.numpy()
+    kept = [m for m in range(3) if m != mode]
+    mode_order = (kept[0], kept[1], mode)                       # contracted mode stored last
+    pk = oracle.pack(c, v, dims, mode_order, (CU, CU, CU))
+    X = upload_packed(pk)
+    vec = synth.random_dense((dims[mode],), seed).numpy()
+    keys, want, norm = oracle.ttv(c, v, dims, mode, vec)
+    for out_attr in [(D, CU), (CU, CU)]:
+        Y = comet.ttv_symbolic(X, mode, out_attr)
+        Y.val.fill_(float("nan"))
+        comet.ttv(X, mode, dev(vec), Y)
+        assert_close(Y.val, want, norm, what="ttv")
+        # structure: the sparse matrix over the kept modes, packed in the asked format
+        ka, kb = keys // dims[kept[1]], keys % dims[kept[1]]
+        ref = oracle.pack([ka, kb], np.ones(len(keys)), (dims[kept[0]], dims[kept[1]]), (0, 1), out_attr)
+        for l in range(2):
+            assert_equal_arrays(Y.pos(l), ref.pos[l], f"ttv pos{l}")
+            assert_equal_arrays(Y.crd(l), ref.crd[l], f"ttv crd{l}")
+    for R in (1, 4, 16, 5):
+        U = synth.random_dense((dims[mode], R), seed + 1).numpy()
+        _, wantm, normm = oracle.ttm(c, v, dims, mode, U)
+        Z = comet.ttm_symbolic(X, mode, R)
+        Z.val.fill_(float("nan"))
+        comet.ttm(X, mode, dev(U), Z)
+        assert_close(Z.val.reshape(-1, R), wantm, normm, what=f"ttm R={R}")
+        for l in range(2):
+            assert_equal_arrays(Z.pos(l), pk.pos[l], f"ttm pos{l}")
+            assert_equal_arrays(Z.crd(l), pk.crd[l], f"ttm crd{l}")
+
+
+@pytest.mark.parametrize("dims,nnz,seed", TENSOR_CASES)
+@pytest.mark.parametrize("mode", [0, 1, 2])
+@pytest.mark.parametrize("attr", [(CN, S, S), (CU, CU, CU)])
+def test_mttkrp(dims, nnz, seed, mode, attr, tile_items):
+    coords, val = synth.random_coo(dims, nnz, seed)
+    c, v = _np(coords), val.numpy()
+    kept = [m for m in range(3) if m != mode]
+    mode_order = (mode, kept[0], kept[1])                       # output mode stored first
+    X = upload_packed(oracle.pack(c, v, dims, mode_order, attr))
+    for R in (1, 8, 32, 7):
+        F = [synth.random_dense((d, R), seed, 60 + m).numpy() for m, d in enumerate(dims)]
+        want, norm = oracle.mttkrp(c, v, dims, mode, F)
+        out = torch.full((dims[mode], R), float("nan"), dtype=torch.float64, device="cuda")
+        comet.mttkrp(X, mode, [None if m == mode else dev(f) for m, f in enumerate(F)], out)
+        assert_close(out, want, norm, what=f"mttkrp R={R}")
+
+
+def test_mttkrp_exact_on_small_integers():
+    dims = (25, 20, 15)
+    coords, val = synth.random_coo(dims, 2000, 5, integer_values=True)
+    c, v = _np(coords), val.numpy()
+    F = [synth.random_dense((d, 16), 5, 60 + m, integer_values=True).numpy() for m, d in enumerate(dims)]
+    want, _ = oracle.mttkrp(c, v, dims, 0, F)
+    for attr in [(CN, S, S), (CU, CU, CU)]:
+        X = upload_packed(oracle.pack(c, v, dims, (0, 1, 2), attr))
+        assert_equal_arrays(comet.mttkrp(X, 0, [None, dev(F[1]), dev(F[2])]), want, "integer mttkrp")
+
+
+def test_results_are_reproducible_run_to_run():
+    case = synth.make(2, scale=1 / 256)
+    c, v = _np(case.coords), case.val.numpy()
+    A = upload_packed(oracle.pack(c, v, case.dims, (0, 1), (D, CU)))
+    B = case.dense["B"].cuda()
+    first = comet.spmm(A, B).clone()
+    for _ in range(3):
+        assert torch.equal(comet.spmm(A, B), first)
+
+
+@pytest.mark.parametrize("config", [1, 2, 3, 4, 5])
+def test_scaled_workloads(config):
+    """The five benchmark workloads at 1/64 scale (several tiles, ragged tails, skewed segments)."""
+    case = synth.make(config, scale=1 / 64)
+    c, v = _np(case.coords), case.val.numpy()
+    if config == 1:
+        want, norm = oracle.spmv(c, v, case.dims, case.dense["x"].numpy())
+        A = upload_packed(oracle.pack(c, v, case.dims, (0, 1), (D, CU)))
+        assert_close(comet.spmv(A, case.dense["x"].cuda()), want, norm, what="C1")
+    elif config == 2:
+        want, norm = oracle.spmm(c, v, case.dims, case.dense["B"].numpy())
+        A = upload_packed(oracle.pack(c, v, case.dims, (0, 1), (D, CU)))
+        assert_close(comet.spmm(A, case.dense["B"].cuda()), want, norm, what="C2")
+    elif config == 3:
+        _, want, norm = oracle.ttv(c, v, case.dims, 2, case.dense["v"].numpy())
+        X = upload_packed(oracle.pack(c, v, case.dims, (0, 1, 2), (CU, CU, CU)))
+        assert_close(comet.ttv(X, 2, case.dense["v"].cuda()).val, want, norm, what="C3")
+    elif config == 4:
+        _, want, norm = oracle.ttm(c, v, case.dims, 2, case.dense["U"].numpy())
+        X = upload_packed(oracle.pack(c, v, case.dims, (0, 1, 2), (CU, CU, CU)))
+        assert_close(comet.ttm(X, 2, case.dense["U"].cuda()).val.reshape(-1, case.R), want, norm, what="C4")
+    else:
+        F = [None, case.dense["B"].numpy(), case.dense["C"].numpy()]
+        want, norm = oracle.mttkrp(c, v, case.dims, 0, F)
+        Fd = [None, case.dense["B"].cuda(), case.dense["C"].cuda()]
+        for attr in [(CN, S, S), (CU, CU, CU)]:
+            X = upload_packed(oracle.pack(c, v, case.dims, (0, 1, 2), attr))
+            assert_close(comet.mttkrp(X, 0, Fd), want, norm, what=f"C5 {attr}")
+
+
+def test_argument_errors_are_reported_not_raised_by_cuda():
+    A = upload_packed(oracle.pack([[0], [1]], [1.0], (2, 2), (0, 1), (D, CU)))
+    B = torch.ones((2, 4), dtype=torch.float64, device="cuda")
+    with pytest.raises(comet.CometError) as e:
+        comet.spmm(A, B, torch.empty((2, 2), dtype=torch.float64, device="cuda"))     # ldc < R
+    assert e.value.status == -1
+    X = upload_packed(oracle.pack([[0], [1], [1]], [1.0], (2, 2, 2), (0, 1, 2), (CU, CU, CU)))
+    with pytest.raises(comet.CometError) as e:
+        comet.ttv(X, 0, torch.ones(2, dtype=torch.float64, device="cuda"))             # mode 0 is not stored last
+    assert e.value.status == -2
+    with pytest.raises(comet.CometError) as e:
+        comet.mttkrp(X, 2, [B[:, :1], B[:, :1], None])                                 # mode 2 is not stored first
+    assert e.value.status == -2
