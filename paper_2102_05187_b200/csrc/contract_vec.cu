@@ -3,16 +3,15 @@
 // out[s, :] += val[p] * B[crd[p], :]" where a segment is a CSR row (SpMM) or a CSF fiber (TTM).
 //
 // Work split (B200): the merge list of segment-end markers and leaf positions is cut into tiles of a
-// fixed number of items, one tile per WORKER. A worker is a group of LPN lanes of a warp; lane g of
-// the group owns columns {(t*LPN + g)*VEC .. +VEC} for t < CPL, so one gather of a dense row is one
-// fully coalesced LPN*VEC*8-byte request and nothing is ever reduced across lanes. A worker walks
-// its tile sequentially, keeps up to UNROLL independent row gathers in flight, stores every segment
+// fixed number of items, one tile per WORKER (a group of LPN lanes of a warp, see walk.cuh). A worker
+// walks its tile sequentially with a rolling window of row gathers in flight, stores every segment
 // that ENDS inside its tile with plain vector stores (so every output row is written exactly once,
 // without a memset), and hands the partial sum of the segment it stops in to a carry slot. A second
 // small kernel adds the carries of earlier tiles onto the stored rows in tile order, which makes the
 // result deterministic (no atomics anywhere).
 #include "common.cuh"
 #include "kernels.cuh"
+#include "walk.cuh"
 
 namespace comet {
 
@@ -35,138 +34,79 @@ struct SegGatherArgs {
   int32_t carry_ld;
 };
 
-template <int VEC> struct Piece;
-template <> struct Piece<2> {
-  static __device__ __forceinline__ void load(const double *p, double *d) {
-    double2 v = __ldg(reinterpret_cast<const double2 *>(p));
-    d[0] = v.x; d[1] = v.y;
+// What the walker does with one leaf entry: close the segments that end in front of it, accumulate.
+template <int LPN, int CPL, int VEC, bool MAPPED>
+struct SegGatherPolicy {
+  using Entry = Entry16;
+  using L = Lanes<LPN, CPL, VEC>;
+  static constexpr int kRows = 1;
+  struct Window { double r[1][CPL][VEC]; };
+
+  const SegGatherArgs &a;
+  const L &ln;
+  double acc[CPL][VEC];
+  int64_t i;          // open segment
+  int32_t next_end;   // leaf position where it ends (-1: no segment left)
+  int32_t last_flush; // leaf position of the latest flush (entries at or after it are still in acc)
+
+  __device__ __forceinline__ SegGatherPolicy(const SegGatherArgs &args, const L &lanes, int64_t i0, int32_t j0)
+      : a(args), ln(lanes), i(i0), last_flush(j0) {
+    ln.zero(acc);
+    next_end = (i < a.M) ? __ldg(a.seg_end + i) : -1;
   }
-  static __device__ __forceinline__ void store(double *p, const double *d) {
-    __stcs(reinterpret_cast<double2 *>(p), make_double2(d[0], d[1]));
+  __device__ __forceinline__ Entry fetch(int32_t j) const { return Entry{ld_stream(a.val + j), ld_stream(a.crd + j), 0}; }
+  static __device__ __forceinline__ Entry idle() { return Entry{0.0, 0, 0}; }
+  __device__ __forceinline__ const double *row(const Entry &e, int) const { return a.B + (int64_t)e.a * a.ldb; }
+
+  // Stores the open segment (and, for a compressed root level, zero-fills the rows in front of it).
+  __device__ __forceinline__ void flush(int32_t j) {
+    int64_t r = i;
+    if (MAPPED) {
+      r = __ldg(a.out_row + i);
+      const int64_t lo = (i > 0) ? (int64_t)__ldg(a.out_row + i - 1) + 1 : 0;
+      ln.zero_rows(a.C, a.ldc, lo, r);
+      if (i == a.M - 1) ln.zero_rows(a.C, a.ldc, r + 1, a.out_rows);
+    }
+    ln.store_row(a.C + r * a.ldc, acc);
+    ln.zero(acc);
+    ++i;
+    next_end = (i < a.M) ? __ldg(a.seg_end + i) : -1;
+    last_flush = j;
   }
-  static __device__ __forceinline__ void store_plain(double *p, const double *d) {
-    *reinterpret_cast<double2 *>(p) = make_double2(d[0], d[1]);
+  __device__ __forceinline__ void consume(int32_t j, const Entry &e, const double (&rows)[1][CPL][VEC]) {
+    while (j == next_end) flush(j);          // segments (possibly empty ones) that end in front of leaf j
+#pragma unroll
+    for (int t = 0; t < CPL; ++t)
+      if (ln.ok[t])
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) acc[t][k] = fma(e.v, rows[0][t][k], acc[t][k]);
   }
 };
-template <> struct Piece<1> {
-  static __device__ __forceinline__ void load(const double *p, double *d) { d[0] = __ldg(p); }
-  static __device__ __forceinline__ void store(double *p, const double *d) { __stcs(p, d[0]); }
-  static __device__ __forceinline__ void store_plain(double *p, const double *d) { *p = d[0]; }
-};
 
-template <int LPN> __device__ __forceinline__ unsigned group_mask() {
-  if (LPN == 32) return 0xffffffffu;
-  const unsigned lane = threadIdx.x & 31;
-  return ((1u << LPN) - 1u) << (lane & ~(LPN - 1));
-}
-
-template <int LPN, int CPL, int VEC>
+template <int LPN, int CPL, int VEC, bool MAPPED>
 __global__ void __launch_bounds__(kBlockThreads) seg_gather_kernel(const SegGatherArgs a) {
-  constexpr int UNROLL = LPN < 8 ? LPN : 8;
-  constexpr int WORKERS = kBlockThreads / LPN;
-  const int g = threadIdx.x & (LPN - 1);
-  const int64_t tile = (int64_t)blockIdx.x * WORKERS + threadIdx.x / LPN;
+  using L = Lanes<LPN, CPL, VEC>;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int worker = threadIdx.x / LPN;
+  const int64_t tile = (int64_t)blockIdx.x * L::kWorkers + worker;
   if (tile >= a.num_tiles) return;                       // whole groups leave together
-  const unsigned mask = group_mask<LPN>();
+  Entry16 *ring = reinterpret_cast<Entry16 *>(smem_raw) + worker * 2 * L::kChunk;
+  const L ln(a.R);
 
   const int64_t total = a.M + a.N;
   const int64_t d0 = tile * a.tile_items;
   const int64_t d1 = (d0 + a.tile_items < total) ? d0 + a.tile_items : total;
-  int64_t i = merge_path_segments(a.seg_end, a.M, a.N, d0);
-  const int64_t j0 = d0 - i;
+  const int64_t i0 = merge_path_segments(a.seg_end, a.M, a.N, d0);
   const int64_t i1 = merge_path_segments(a.seg_end, a.M, a.N, d1);
-  const int64_t j1 = d1 - i1;
+  const int32_t j0 = (int32_t)(d0 - i0), j1 = (int32_t)(d1 - i1);
 
-  bool col_ok[CPL];
-  int64_t col[CPL];
-#pragma unroll
-  for (int t = 0; t < CPL; ++t) {
-    col[t] = (int64_t)(t * LPN + g) * VEC;
-    col_ok[t] = col[t] < a.R;                            // only the scalar (VEC == 1) path can be ragged
-  }
+  SegGatherPolicy<LPN, CPL, VEC, MAPPED> p(a, ln, i0, j0);
+  walk_tile(ln, p, j0, j1, ring);
+  while (p.i < i1) p.flush(j1);                          // end markers that close the tile
 
-  double acc[CPL][VEC];
-#pragma unroll
-  for (int t = 0; t < CPL; ++t)
-#pragma unroll
-    for (int e = 0; e < VEC; ++e) acc[t][e] = 0.0;
-  bool dirty = false;
-  int64_t next_end = (i < a.M) ? (int64_t)__ldg(a.seg_end + i) : -1;
-
-  auto flush = [&]() {
-    int64_t row = i;
-    if (a.out_row) {
-      row = __ldg(a.out_row + i);
-      int64_t lo = (i > 0) ? (int64_t)__ldg(a.out_row + i - 1) + 1 : 0;
-      const double zero[VEC] = {};
-      for (int64_t z = lo; z < row; ++z)
-#pragma unroll
-        for (int t = 0; t < CPL; ++t)
-          if (col_ok[t]) Piece<VEC>::store(a.C + z * a.ldc + col[t], zero);
-      if (i == a.M - 1)
-        for (int64_t z = row + 1; z < a.out_rows; ++z)
-#pragma unroll
-          for (int t = 0; t < CPL; ++t)
-            if (col_ok[t]) Piece<VEC>::store(a.C + z * a.ldc + col[t], zero);
-    }
-#pragma unroll
-    for (int t = 0; t < CPL; ++t) {
-      if (col_ok[t]) Piece<VEC>::store(a.C + row * a.ldc + col[t], acc[t]);
-#pragma unroll
-      for (int e = 0; e < VEC; ++e) acc[t][e] = 0.0;
-    }
-    dirty = false;
-    ++i;
-    next_end = (i < a.M) ? (int64_t)__ldg(a.seg_end + i) : -1;
-  };
-
-  for (int64_t base = j0; base < j1; base += LPN) {
-    const int64_t mine = base + g;
-    int32_t my_c = 0;
-    double my_v = 0.0;
-    if (mine < j1) {
-      my_c = ld_stream(a.crd + mine);
-      my_v = ld_stream(a.val + mine);
-    }
-    const int n = (j1 - base < LPN) ? (int)(j1 - base) : LPN;
-    for (int u0 = 0; u0 < n; u0 += UNROLL) {
-      double rows[UNROLL][CPL][VEC];
-      double vv[UNROLL];
-#pragma unroll
-      for (int q = 0; q < UNROLL; ++q) {
-        const int src = (u0 + q) & (LPN - 1);
-        const int32_t c = __shfl_sync(mask, my_c, src, LPN);
-        vv[q] = __shfl_sync(mask, my_v, src, LPN);
-        if (u0 + q < n) {
-          const double *brow = a.B + (int64_t)c * a.ldb;
-#pragma unroll
-          for (int t = 0; t < CPL; ++t)
-            if (col_ok[t]) Piece<VEC>::load(brow + col[t], rows[q][t]);
-        }
-      }
-#pragma unroll
-      for (int q = 0; q < UNROLL; ++q) {
-        if (u0 + q < n) {
-          const int64_t jj = base + u0 + q;
-          while (jj == next_end) flush();                // segments (possibly empty ones) that end before leaf jj
-#pragma unroll
-          for (int t = 0; t < CPL; ++t)
-            if (col_ok[t])
-#pragma unroll
-              for (int e = 0; e < VEC; ++e) acc[t][e] = fma(vv[q], rows[q][t][e], acc[t][e]);
-          dirty = true;
-        }
-      }
-    }
-  }
-  while (i < i1) flush();                                // end markers that close the tile
-
-  if (g == 0) a.carry_seg[tile] = (dirty && i < a.M) ? (int32_t)i : -1;
-  if (dirty && i < a.M) {
-#pragma unroll
-    for (int t = 0; t < CPL; ++t)
-      if (col_ok[t]) Piece<VEC>::store_plain(a.carry_val + tile * a.carry_ld + col[t], acc[t]);
-  }
+  const bool carry = p.i < a.M && j1 > p.last_flush;     // leaf entries of a segment that ends in a later tile
+  if (ln.g == 0) a.carry_seg[tile] = carry ? (int32_t)p.i : -1;
+  if (carry) ln.store_carry(a.carry_val + tile * a.carry_ld, p.acc);
 }
 
 // Adds the carries onto the stored rows. Tiles that stopped inside the same segment are consecutive;
@@ -215,6 +155,18 @@ int32_t choose_tile_items(int64_t total_items, int workers_per_block) {
   return (int32_t)t;
 }
 
+template <int LPN, int CPL, int VEC, bool MAPPED>
+static comet_status_t launch_mapped(Context *ctx, const SegGatherArgs &a, int64_t blocks, cudaStream_t stream) {
+  using L = Lanes<LPN, CPL, VEC>;
+  constexpr size_t smem = (size_t)L::kWorkers * 2 * L::kChunk * sizeof(Entry16);
+  auto kernel = seg_gather_kernel<LPN, CPL, VEC, MAPPED>;
+  if (smem > 48 * 1024)
+    COMET_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  kernel<<<(unsigned)blocks, kBlockThreads, smem, stream>>>(a);
+  COMET_LAUNCH_CHECK(ctx);
+  return COMET_OK;
+}
+
 template <int LPN, int CPL, int VEC>
 static comet_status_t launch_one(Context *ctx, SegGatherArgs a, cudaStream_t stream) {
   constexpr int WORKERS = kBlockThreads / LPN;
@@ -229,8 +181,9 @@ static comet_status_t launch_one(Context *ctx, SegGatherArgs a, cudaStream_t str
   a.carry_val = (double *)scratch;
   a.carry_seg = (int32_t *)(scratch + val_bytes);
   const int64_t blocks = ceil_div(a.num_tiles, WORKERS);
-  seg_gather_kernel<LPN, CPL, VEC><<<(unsigned)blocks, kBlockThreads, 0, stream>>>(a);
-  COMET_LAUNCH_CHECK(ctx);
+  comet_status_t st = a.out_row ? launch_mapped<LPN, CPL, VEC, true>(ctx, a, blocks, stream)
+                                : launch_mapped<LPN, CPL, VEC, false>(ctx, a, blocks, stream);
+  if (st != COMET_OK) return st;
   const int64_t fix_threads = a.num_tiles * a.R;
   carry_fixup_kernel<<<(unsigned)ceil_div(fix_threads, 256), 256, 0, stream>>>(
       a.carry_val, a.carry_seg, a.num_tiles, a.R, a.carry_ld, a.C, a.ldc, a.out_row);

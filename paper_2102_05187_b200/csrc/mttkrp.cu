@@ -4,35 +4,15 @@
 //   COO [CN,S,S]  sorted entries, an output row is a run of equal root coordinates;
 //   CSF [CU,CU,CU] per fiber t = sum x * Q[k, :], then out[i, :] += t * P[j, :] (one P row per fiber).
 //
-// Same worker scheme as the SpMM/TTM kernel: a worker is LPN lanes of a warp, each owning VEC columns
-// of every 16*LPN-byte row piece, walking a tile of consecutive leaf entries with UNROLL independent
-// row gathers in flight. A worker stores the output rows that END in its tile (and zero-fills the
+// Same worker scheme as the SpMM/TTM kernel (walk.cuh): a worker is LPN lanes of a warp walking a tile of
+// consecutive leaf entries with a rolling window of row gathers in flight. A worker stores the output rows that END in its tile (and zero-fills the
 // rows between consecutive stored rows, so no memset is needed), and writes the partial sum of the
 // row it stops in to a carry slot that the fix-up kernel adds in tile order (deterministic).
 #include "common.cuh"
 #include "kernels.cuh"
+#include "walk.cuh"
 
 namespace comet {
-
-template <int LPN> __device__ __forceinline__ unsigned lane_group_mask() {
-  if (LPN == 32) return 0xffffffffu;
-  const unsigned lane = threadIdx.x & 31;
-  return ((1u << LPN) - 1u) << (lane & ~(LPN - 1));
-}
-
-__device__ __forceinline__ void load_piece(const double *p, double (&d)[2]) {
-  const double2 v = __ldg(reinterpret_cast<const double2 *>(p));
-  d[0] = v.x; d[1] = v.y;
-}
-__device__ __forceinline__ void load_piece(const double *p, double (&d)[1]) { d[0] = __ldg(p); }
-__device__ __forceinline__ void store_piece(double *p, const double (&d)[2]) {
-  __stcs(reinterpret_cast<double2 *>(p), make_double2(d[0], d[1]));
-}
-__device__ __forceinline__ void store_piece(double *p, const double (&d)[1]) { __stcs(p, d[0]); }
-__device__ __forceinline__ void store_piece_plain(double *p, const double (&d)[2]) {
-  *reinterpret_cast<double2 *>(p) = make_double2(d[0], d[1]);
-}
-__device__ __forceinline__ void store_piece_plain(double *p, const double (&d)[1]) { *p = d[0]; }
 
 struct MttkrpArgs {
   // COO: crd0/crd1/crd2/val over N entries. CSF: pos1 (S+1), crd0 (S), crd1 (F), seg_end2 (= pos2+1, F), crd2, val.
@@ -53,237 +33,174 @@ struct MttkrpArgs {
   int32_t carry_ld;
 };
 
-template <int LPN, int CPL, int VEC> struct RowOut {
-  int64_t col[CPL];
-  bool ok[CPL];
+// ------------------------------------------------------------------------------------------- COO
+template <int LPN, int CPL, int VEC>
+struct CooPolicy {
+  using Entry = Entry32;                 // value, root coordinate, level-1 coordinate, leaf coordinate
+  using L = Lanes<LPN, CPL, VEC>;
+  static constexpr int kRows = 2;
+  struct Window { double r[2][CPL][VEC]; };
+
   const MttkrpArgs &a;
-  __device__ RowOut(const MttkrpArgs &args, int g) : a(args) {
-#pragma unroll
-    for (int t = 0; t < CPL; ++t) {
-      col[t] = (int64_t)(t * LPN + g) * VEC;
-      ok[t] = col[t] < args.R;
-    }
+  const L &ln;
+  double acc[CPL][VEC];
+  int32_t cur;                           // output row being accumulated
+
+  __device__ __forceinline__ CooPolicy(const MttkrpArgs &args, const L &lanes, int32_t first_row)
+      : a(args), ln(lanes), cur(first_row) { ln.zero(acc); }
+  __device__ __forceinline__ Entry fetch(int32_t j) const {
+    return Entry{ld_stream(a.val + j), ld_stream(a.crd0 + j), ld_stream(a.crd1 + j), ld_stream(a.crd2 + j), 0, 0};
   }
-  __device__ __forceinline__ void zero_rows(int64_t lo, int64_t hi) const {   // rows lo .. hi-1
-    const double zero[VEC] = {};
-    for (int64_t z = lo; z < hi; ++z)
-#pragma unroll
-      for (int t = 0; t < CPL; ++t)
-        if (ok[t]) store_piece(a.out + z * a.ldo + col[t], zero);
+  static __device__ __forceinline__ Entry idle() { return Entry{0.0, 0, 0, 0, 0, 0}; }
+  __device__ __forceinline__ const double *row(const Entry &e, int w) const {
+    return w == 0 ? a.P + (int64_t)e.b * a.ldp : a.Q + (int64_t)e.c * a.ldq;
   }
-  __device__ __forceinline__ void store_row(int64_t row, double (&acc)[CPL][VEC]) const {
-#pragma unroll
-    for (int t = 0; t < CPL; ++t) {
-      if (ok[t]) store_piece(a.out + row * a.ldo + col[t], acc[t]);
-#pragma unroll
-      for (int e = 0; e < VEC; ++e) acc[t][e] = 0.0;
-    }
+  // The run of `cur` ends here: store it, zero-fill the rows up to the next stored row.
+  __device__ __forceinline__ void next_row(int32_t row) {
+    ln.store_row(a.out + (int64_t)cur * a.ldo, acc);
+    ln.zero_rows(a.out, a.ldo, (int64_t)cur + 1, row);
+    ln.zero(acc);
+    cur = row;
   }
-  __device__ __forceinline__ void store_carry(int64_t tile, const double (&acc)[CPL][VEC]) const {
+  __device__ __forceinline__ void consume(int32_t, const Entry &e, const double (&rows)[2][CPL][VEC]) {
+    if (e.a != cur) next_row(e.a);
 #pragma unroll
     for (int t = 0; t < CPL; ++t)
-      if (ok[t]) store_piece_plain(a.carry_val + tile * a.carry_ld + col[t], acc[t]);
+      if (ln.ok[t])
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) acc[t][k] = fma(e.v * rows[0][t][k], rows[1][t][k], acc[t][k]);
   }
 };
 
-// ------------------------------------------------------------------------------------------- COO
 template <int LPN, int CPL, int VEC>
 __global__ void __launch_bounds__(kBlockThreads) mttkrp_coo_kernel(const MttkrpArgs a) {
-  constexpr int UNROLL = LPN < 8 ? LPN : 8;
-  constexpr int WORKERS = kBlockThreads / LPN;
-  const int g = threadIdx.x & (LPN - 1);
-  const int64_t tile = (int64_t)blockIdx.x * WORKERS + threadIdx.x / LPN;
+  using L = Lanes<LPN, CPL, VEC>;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int worker = threadIdx.x / LPN;
+  const int64_t tile = (int64_t)blockIdx.x * L::kWorkers + worker;
   if (tile >= a.num_tiles) return;
-  const unsigned mask = lane_group_mask<LPN>();
-  const RowOut<LPN, CPL, VEC> o(a, g);
+  Entry32 *ring = reinterpret_cast<Entry32 *>(smem_raw) + worker * 2 * L::kChunk;
+  const L ln(a.R);
 
   const int64_t j0 = tile * a.tile_items;
   const int64_t j1 = (j0 + a.tile_items < a.N) ? j0 + a.tile_items : a.N;
-  int64_t cur = __ldg(a.crd0 + j0);
+  const int32_t first = __ldg(a.crd0 + j0);
   {
     const int64_t prev = j0 > 0 ? (int64_t)__ldg(a.crd0 + j0 - 1) : -1;
-    if (prev != cur) o.zero_rows(prev + 1, cur);         // the gap in front of a row is filled where the row starts
+    if (prev != first) ln.zero_rows(a.out, a.ldo, prev + 1, first);   // the gap in front of a row is filled where it starts
   }
-  double acc[CPL][VEC];
-#pragma unroll
-  for (int t = 0; t < CPL; ++t)
-#pragma unroll
-    for (int e = 0; e < VEC; ++e) acc[t][e] = 0.0;
+  CooPolicy<LPN, CPL, VEC> p(a, ln, first);
+  walk_tile(ln, p, (int32_t)j0, (int32_t)j1, ring);
 
-  for (int64_t base = j0; base < j1; base += LPN) {
-    const int64_t mine = base + g;
-    int32_t my_i = 0, my_j = 0, my_k = 0;
-    double my_v = 0.0;
-    if (mine < j1) {
-      my_i = ld_stream(a.crd0 + mine);
-      my_j = ld_stream(a.crd1 + mine);
-      my_k = ld_stream(a.crd2 + mine);
-      my_v = ld_stream(a.val + mine);
-    }
-    const int n = (j1 - base < LPN) ? (int)(j1 - base) : LPN;
-    for (int u0 = 0; u0 < n; u0 += UNROLL) {
-      double prow[UNROLL][CPL][VEC], qrow[UNROLL][CPL][VEC];
-      double vv[UNROLL];
-      int32_t ri[UNROLL];
-#pragma unroll
-      for (int q = 0; q < UNROLL; ++q) {
-        const int src = (u0 + q) & (LPN - 1);
-        ri[q] = __shfl_sync(mask, my_i, src, LPN);
-        const int32_t cj = __shfl_sync(mask, my_j, src, LPN);
-        const int32_t ck = __shfl_sync(mask, my_k, src, LPN);
-        vv[q] = __shfl_sync(mask, my_v, src, LPN);
-        if (u0 + q < n) {
-          const double *pr = a.P + (int64_t)cj * a.ldp;
-          const double *qr = a.Q + (int64_t)ck * a.ldq;
-#pragma unroll
-          for (int t = 0; t < CPL; ++t)
-            if (o.ok[t]) {
-              load_piece(pr + o.col[t], prow[q][t]);
-              load_piece(qr + o.col[t], qrow[q][t]);
-            }
-        }
-      }
-#pragma unroll
-      for (int q = 0; q < UNROLL; ++q) {
-        if (u0 + q < n) {
-          if (ri[q] != cur) {
-            o.store_row(cur, acc);
-            o.zero_rows(cur + 1, ri[q]);
-            cur = ri[q];
-          }
-#pragma unroll
-          for (int t = 0; t < CPL; ++t)
-            if (o.ok[t])
-#pragma unroll
-              for (int e = 0; e < VEC; ++e) acc[t][e] = fma(vv[q] * prow[q][t][e], qrow[q][t][e], acc[t][e]);
-        }
-      }
-    }
-  }
   const int64_t nxt = j1 < a.N ? (int64_t)__ldg(a.crd0 + j1) : -1;
-  if (nxt == cur) {
-    if (g == 0) a.carry_seg[tile] = (int32_t)cur;
-    o.store_carry(tile, acc);
+  if (nxt == p.cur) {                                    // the row continues in the next tile
+    if (ln.g == 0) a.carry_seg[tile] = p.cur;
+    ln.store_carry(a.carry_val + tile * a.carry_ld, p.acc);
   } else {
-    if (g == 0) a.carry_seg[tile] = -1;
-    o.store_row(cur, acc);
-    if (j1 == a.N) o.zero_rows(cur + 1, a.rows);
+    if (ln.g == 0) a.carry_seg[tile] = -1;
+    ln.store_row(a.out + (int64_t)p.cur * a.ldo, p.acc);
+    if (j1 == a.N) ln.zero_rows(a.out, a.ldo, (int64_t)p.cur + 1, a.rows);
   }
 }
 
 // ------------------------------------------------------------------------------------------- CSF
 template <int LPN, int CPL, int VEC>
+struct CsfPolicy {
+  using Entry = Entry16;                 // value, leaf coordinate
+  using L = Lanes<LPN, CPL, VEC>;
+  static constexpr int kRows = 1;
+  struct Window { double r[1][CPL][VEC]; };
+
+  const MttkrpArgs &a;
+  const L &ln;
+  double tac[CPL][VEC], aac[CPL][VEC];   // open fiber sum, open slice sum
+  int64_t f, s;                          // open fiber, open slice
+  int32_t next_end;                      // leaf position where the open fiber ends
+  int64_t slice_end;                     // fiber index where the open slice ends
+  int32_t last_fold;                     // leaf position of the latest fold (entries at or after it are in tac)
+  bool a_dirty;
+
+  __device__ __forceinline__ CsfPolicy(const MttkrpArgs &args, const L &lanes, int64_t f0, int64_t s0, int32_t j0)
+      : a(args), ln(lanes), f(f0), s(s0), last_fold(j0), a_dirty(false) {
+    ln.zero(tac);
+    ln.zero(aac);
+    next_end = f < a.F ? __ldg(a.seg_end2 + f) : -1;
+    slice_end = s < a.S ? (int64_t)__ldg(a.pos1 + s + 1) : -1;
+  }
+  __device__ __forceinline__ Entry fetch(int32_t j) const { return Entry{ld_stream(a.val + j), ld_stream(a.crd2 + j), 0}; }
+  static __device__ __forceinline__ Entry idle() { return Entry{0.0, 0, 0}; }
+  __device__ __forceinline__ const double *row(const Entry &e, int) const { return a.Q + (int64_t)e.a * a.ldq; }
+
+  __device__ __forceinline__ void fold(int32_t j) {      // aac += tac * P[crd1[f], :]
+    const double *pr = a.P + (int64_t)__ldg(a.crd1 + f) * a.ldp;
+    double prow[CPL][VEC];
+    ln.gather(pr, prow);
+#pragma unroll
+    for (int t = 0; t < CPL; ++t)
+      if (ln.ok[t])
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) { aac[t][k] = fma(tac[t][k], prow[t][k], aac[t][k]); tac[t][k] = 0.0; }
+    a_dirty = true;
+    last_fold = j;
+  }
+  __device__ __forceinline__ void end_fiber(int32_t j) {
+    fold(j);
+    ++f;
+    next_end = f < a.F ? __ldg(a.seg_end2 + f) : -1;
+    if (f == slice_end) {                                // the slice is complete: this worker owns its row
+      const int64_t row = __ldg(a.crd0 + s);
+      const int64_t lo = s > 0 ? (int64_t)__ldg(a.crd0 + s - 1) + 1 : 0;
+      ln.zero_rows(a.out, a.ldo, lo, row);
+      ln.store_row(a.out + row * a.ldo, aac);
+      if (s == a.S - 1) ln.zero_rows(a.out, a.ldo, row + 1, a.rows);
+      ln.zero(aac);
+      a_dirty = false;
+      ++s;
+      slice_end = s < a.S ? (int64_t)__ldg(a.pos1 + s + 1) : -1;
+    }
+  }
+  __device__ __forceinline__ void consume(int32_t j, const Entry &e, const double (&rows)[1][CPL][VEC]) {
+    while (j == next_end) end_fiber(j);
+#pragma unroll
+    for (int t = 0; t < CPL; ++t)
+      if (ln.ok[t])
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) tac[t][k] = fma(e.v, rows[0][t][k], tac[t][k]);
+  }
+};
+
+template <int LPN, int CPL, int VEC>
 __global__ void __launch_bounds__(kBlockThreads) mttkrp_csf_kernel(const MttkrpArgs a) {
-  constexpr int UNROLL = LPN < 8 ? LPN : 8;
-  constexpr int WORKERS = kBlockThreads / LPN;
-  const int g = threadIdx.x & (LPN - 1);
-  const int64_t tile = (int64_t)blockIdx.x * WORKERS + threadIdx.x / LPN;
+  using L = Lanes<LPN, CPL, VEC>;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int worker = threadIdx.x / LPN;
+  const int64_t tile = (int64_t)blockIdx.x * L::kWorkers + worker;
   if (tile >= a.num_tiles) return;
-  const unsigned mask = lane_group_mask<LPN>();
-  const RowOut<LPN, CPL, VEC> o(a, g);
+  Entry16 *ring = reinterpret_cast<Entry16 *>(smem_raw) + worker * 2 * L::kChunk;
+  const L ln(a.R);
 
   // tile = a span of the merge list of fiber-end markers and leaf positions
   const int64_t total = a.F + a.N;
   const int64_t d0 = tile * a.tile_items;
   const int64_t d1 = (d0 + a.tile_items < total) ? d0 + a.tile_items : total;
-  int64_t f = merge_path_segments(a.seg_end2, a.F, a.N, d0);
-  const int64_t j0 = d0 - f;
+  const int64_t f0 = merge_path_segments(a.seg_end2, a.F, a.N, d0);
   const int64_t f1 = merge_path_segments(a.seg_end2, a.F, a.N, d1);
-  const int64_t j1 = d1 - f1;
+  const int32_t j0 = (int32_t)(d0 - f0), j1 = (int32_t)(d1 - f1);
 
-  // slice that holds fiber f: the largest s with pos1[s] <= f (every slice is non-empty)
-  int64_t s;
-  {
-    int64_t lo = 0, hi = a.S;                            // answer in [0, S]; S only when f == F
-    while (lo < hi) {
-      const int64_t mid = (lo + hi) >> 1;
-      if ((int64_t)__ldg(a.pos1 + mid + 1) <= f) lo = mid + 1; else hi = mid;
-    }
-    s = lo;
+  // slice that holds fiber f0: the number of slices that end at or before it (every slice is non-empty)
+  int64_t lo = 0, hi = a.S;
+  while (lo < hi) {
+    const int64_t mid = (lo + hi) >> 1;
+    if ((int64_t)__ldg(a.pos1 + mid + 1) <= f0) lo = mid + 1; else hi = mid;
   }
-  int64_t slice_end = s < a.S ? (int64_t)__ldg(a.pos1 + s + 1) : -1;
-  int64_t next_end = f < a.F ? (int64_t)__ldg(a.seg_end2 + f) : -1;
 
-  double tac[CPL][VEC], aac[CPL][VEC];                   // open fiber sum, open slice sum
-#pragma unroll
-  for (int t = 0; t < CPL; ++t)
-#pragma unroll
-    for (int e = 0; e < VEC; ++e) { tac[t][e] = 0.0; aac[t][e] = 0.0; }
-  bool t_dirty = false, a_dirty = false;
-
-  auto fold_fiber = [&]() {                              // aac += tac * P[crd1[f]]
-    const double *pr = a.P + (int64_t)__ldg(a.crd1 + f) * a.ldp;
-#pragma unroll
-    for (int t = 0; t < CPL; ++t)
-      if (o.ok[t]) {
-        double p[VEC];
-        load_piece(pr + o.col[t], p);
-#pragma unroll
-        for (int e = 0; e < VEC; ++e) { aac[t][e] = fma(tac[t][e], p[e], aac[t][e]); tac[t][e] = 0.0; }
-      }
-    t_dirty = false;
-    a_dirty = true;
-  };
-  auto end_fiber = [&]() {
-    fold_fiber();
-    ++f;
-    next_end = f < a.F ? (int64_t)__ldg(a.seg_end2 + f) : -1;
-    if (f == slice_end) {                                // the slice is complete: this worker owns its row
-      const int64_t row = __ldg(a.crd0 + s);
-      const int64_t lo = s > 0 ? (int64_t)__ldg(a.crd0 + s - 1) + 1 : 0;
-      o.zero_rows(lo, row);
-      o.store_row(row, aac);
-      if (s == a.S - 1) o.zero_rows(row + 1, a.rows);
-      a_dirty = false;
-      ++s;
-      slice_end = s < a.S ? (int64_t)__ldg(a.pos1 + s + 1) : -1;
-    }
-  };
-
-  for (int64_t base = j0; base < j1; base += LPN) {
-    const int64_t mine = base + g;
-    int32_t my_k = 0;
-    double my_v = 0.0;
-    if (mine < j1) {
-      my_k = ld_stream(a.crd2 + mine);
-      my_v = ld_stream(a.val + mine);
-    }
-    const int n = (j1 - base < LPN) ? (int)(j1 - base) : LPN;
-    for (int u0 = 0; u0 < n; u0 += UNROLL) {
-      double qrow[UNROLL][CPL][VEC];
-      double vv[UNROLL];
-#pragma unroll
-      for (int q = 0; q < UNROLL; ++q) {
-        const int src = (u0 + q) & (LPN - 1);
-        const int32_t ck = __shfl_sync(mask, my_k, src, LPN);
-        vv[q] = __shfl_sync(mask, my_v, src, LPN);
-        if (u0 + q < n) {
-          const double *qr = a.Q + (int64_t)ck * a.ldq;
-#pragma unroll
-          for (int t = 0; t < CPL; ++t)
-            if (o.ok[t]) load_piece(qr + o.col[t], qrow[q][t]);
-        }
-      }
-#pragma unroll
-      for (int q = 0; q < UNROLL; ++q) {
-        if (u0 + q < n) {
-          const int64_t jj = base + u0 + q;
-          while (jj == next_end) end_fiber();
-#pragma unroll
-          for (int t = 0; t < CPL; ++t)
-            if (o.ok[t])
-#pragma unroll
-              for (int e = 0; e < VEC; ++e) tac[t][e] = fma(vv[q], qrow[q][t][e], tac[t][e]);
-          t_dirty = true;
-        }
-      }
-    }
-  }
-  while (f < f1) end_fiber();
-  if (t_dirty) fold_fiber();                             // an unfinished fiber contributes through distributivity
-  const bool carry = a_dirty && s < a.S;
-  if (g == 0) a.carry_seg[tile] = carry ? (int32_t)s : -1;
-  if (carry) o.store_carry(tile, aac);
+  CsfPolicy<LPN, CPL, VEC> p(a, ln, f0, lo, j0);
+  walk_tile(ln, p, j0, j1, ring);
+  while (p.f < f1) p.end_fiber(j1);
+  if (j1 > p.last_fold) p.fold(j1);                      // an unfinished fiber contributes through distributivity
+  const bool carry = p.a_dirty && p.s < a.S;
+  if (ln.g == 0) a.carry_seg[tile] = carry ? (int32_t)p.s : -1;
+  if (carry) ln.store_carry(a.carry_val + tile * a.carry_ld, p.aac);
 }
 
 // ------------------------------------------------------------------------------------------- host
@@ -303,8 +220,12 @@ static comet_status_t launch_mttkrp(Context *ctx, MttkrpArgs a, cudaStream_t str
   a.carry_val = (double *)scratch;
   a.carry_seg = (int32_t *)(scratch + val_bytes);
   const unsigned blocks = (unsigned)ceil_div(a.num_tiles, WORKERS);
-  if (CSF) mttkrp_csf_kernel<LPN, CPL, VEC><<<blocks, kBlockThreads, 0, stream>>>(a);
-  else mttkrp_coo_kernel<LPN, CPL, VEC><<<blocks, kBlockThreads, 0, stream>>>(a);
+  using L = Lanes<LPN, CPL, VEC>;
+  constexpr size_t smem = (size_t)L::kWorkers * 2 * L::kChunk * (CSF ? sizeof(Entry16) : sizeof(Entry32));
+  auto kernel = CSF ? mttkrp_csf_kernel<LPN, CPL, VEC> : mttkrp_coo_kernel<LPN, CPL, VEC>;
+  if (smem > 48 * 1024)
+    COMET_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  kernel<<<blocks, kBlockThreads, smem, stream>>>(a);
   COMET_LAUNCH_CHECK(ctx);
   carry_fixup_kernel<<<(unsigned)ceil_div(a.num_tiles * a.R, 256), 256, 0, stream>>>(
       a.carry_val, a.carry_seg, a.num_tiles, a.R, a.carry_ld, a.out, a.ldo, CSF ? a.crd0 : nullptr);
