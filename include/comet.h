@@ -104,7 +104,7 @@ int comet_last_cuda_error(comet_handle_t handle);
  *   coo_val             DEVICE, nnz values, copied bitwise into leaf order
  *   h_mode_order[order] a permutation of 0..order-1; h_attr[order] one comet_attr_t per level
  * Supported attribute tuples: [CN,S,...,S], [CU,...,CU], [D,CU,...,CU] (orders 2..4), provided the
- * coordinate bit widths sum to <= 64. Input order is arbitrary; duplicates and out-of-range
+ * coordinate bit widths (ceil(log2(extent)) per mode) sum to <= 63. Input order is arbitrary; duplicates and out-of-range
  * coordinates are detected on the device and reported (COMET_ERR_DUPLICATE_COORD,
  * COMET_ERR_COORD_OUT_OF_RANGE); `out` is then left zeroed. On success `out` owns its arrays
  * (allocated through the handle's allocator) until comet_sptensor_free. Synchronises `stream` once. */

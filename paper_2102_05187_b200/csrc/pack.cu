@@ -1,8 +1,635 @@
-// Placeholder translation unit: replaced by the GPU packing path.
+// comet_pack: COO -> per-level pos/crd arrays on the GPU (the conversion the paper's input-reading
+// runtime function performs; Tensor Storage Format section for what each attribute stores), and
+// comet_validate for caller-built descriptors.
+//
+//   1. keys      one 64-bit key per entry: the coordinates in storage-level order, level 0 in the most
+//                significant bits (so key order = lexicographic order); coordinates are range-checked.
+//   2. sort      stable LSD radix sort of (key, entry index), 8 bits per pass, only over the bits in use.
+//                Per pass: per-tile digit histogram -> exclusive scan of the (digit, tile) table ->
+//                stable scatter (warp-level match ranks, per-warp digit counters in shared memory).
+//   3. levels    head flags from key prefixes: entry p opens a new node at level l when the key prefix
+//                down to level l differs from its predecessor's. Counting pass -> scan -> ONE host
+//                synchronisation to learn the node counts -> exact allocation -> emit pass that writes
+//                crd (compaction), pos (rank of the first child at every parent head), and the values
+//                permuted into leaf order. Equal adjacent keys are duplicates and are reported.
+//
+// No inter-CTA waiting anywhere: every scan is reduce / scan-of-sums / apply in separate launches.
 #include "common.cuh"
-extern "C" comet_status_t comet_pack(comet_handle_t, int32_t, const int64_t *, int64_t, const int32_t *const *,
-                                     const void *, comet_dtype_t, const int32_t *, const int32_t *, void *,
-                                     comet_sptensor_t *) { return COMET_ERR_UNSUPPORTED_FORMAT; }
-extern "C" comet_status_t comet_validate(comet_handle_t, const comet_sptensor_t *, void *) {
-  return COMET_ERR_UNSUPPORTED_FORMAT;
+#include "kernels.cuh"
+
+#include <string.h>
+
+namespace comet {
+
+constexpr int kSortThreads = 256;
+constexpr int kSortItems = 16;
+constexpr int kSortTile = kSortThreads * kSortItems;   // keys per CTA per pass
+constexpr int kSortWarps = kSortThreads / 32;
+
+constexpr int kScanThreads = 256;
+constexpr int kScanItems = 8;
+constexpr int kScanTile = kScanThreads * kScanItems;
+
+enum { kStatusRange = 0, kStatusDuplicate = 1, kStatusInvalid = 2 };   // words of Context::d_status
+
+struct KeyLayout {
+  int order;
+  int shift[COMET_MAX_ORDER];      // bit position of level l's coordinate inside the key
+  int bits[COMET_MAX_ORDER];
+  int total_bits;
+  int64_t dim[COMET_MAX_ORDER];    // extent of the mode stored at level l
+};
+
+struct CoordPtrs { const int32_t *p[COMET_MAX_ORDER]; };   // level order
+
+// ------------------------------------------------------------------------------------------------ keys
+__global__ void make_keys_kernel(CoordPtrs c, KeyLayout k, int64_t n, uint64_t *__restrict__ keys,
+                                 uint32_t *__restrict__ idx, int32_t *__restrict__ status) {
+  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= n) return;
+  uint64_t key = 0;
+  bool bad = false;
+  for (int l = 0; l < k.order; ++l) {
+    const int64_t v = c.p[l][p];
+    bad |= (v < 0) | (v >= k.dim[l]);
+    key |= (uint64_t)(v & ((1ll << k.bits[l]) - 1)) << k.shift[l];
+  }
+  if (bad) atomicOr(status + kStatusRange, 1);
+  keys[p] = key;
+  idx[p] = (uint32_t)p;
+}
+
+// ------------------------------------------------------------------------------------------------ scan
+// Exclusive scan of uint32 in three launches: tile sums, scan of the sums by one CTA, apply.
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t *s_warp, uint32_t *total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
+  uint32_t inc = v;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint32_t t = __shfl_up_sync(0xffffffffu, inc, off);
+    if (lane >= off) inc += t;
+  }
+  if (lane == 31) s_warp[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t w = lane < warps ? s_warp[lane] : 0;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const uint32_t t = __shfl_up_sync(0xffffffffu, w, off);
+      if (lane >= off) w += t;
+    }
+    if (lane < warps) s_warp[lane] = w;        // inclusive over warps
+  }
+  __syncthreads();
+  const uint32_t before = warp > 0 ? s_warp[warp - 1] : 0;
+  if (total) *total = s_warp[warps - 1];
+  __syncthreads();
+  return before + inc - v;
+}
+
+__global__ void scan_tile_sums_kernel(const uint32_t *__restrict__ in, int64_t n, uint32_t *__restrict__ sums) {
+  __shared__ uint32_t s_warp[32];
+  const int64_t base = (int64_t)blockIdx.x * kScanTile;
+  uint32_t v = 0;
+#pragma unroll
+  for (int t = 0; t < kScanItems; ++t) {
+    const int64_t i = base + (int64_t)t * kScanThreads + threadIdx.x;
+    if (i < n) v += in[i];
+  }
+  uint32_t total;
+  block_exclusive_scan(v, s_warp, &total);
+  if (threadIdx.x == 0) sums[blockIdx.x] = total;
+}
+
+// One CTA: exclusive scan of `sums` in place (any length, chunk by chunk with a running carry);
+// the grand total goes to *total_out when given.
+__global__ void scan_sums_kernel(uint32_t *__restrict__ sums, int64_t m, uint32_t *__restrict__ total_out) {
+  __shared__ uint32_t s_warp[32];
+  uint32_t carry = 0;
+  for (int64_t base = 0; base < m; base += blockDim.x) {
+    const int64_t i = base + threadIdx.x;
+    const uint32_t v = i < m ? sums[i] : 0;
+    uint32_t total;
+    const uint32_t ex = block_exclusive_scan(v, s_warp, &total);
+    if (i < m) sums[i] = carry + ex;
+    carry += total;
+  }
+  if (total_out && threadIdx.x == 0) *total_out = carry;
+}
+
+__global__ void scan_apply_kernel(const uint32_t *__restrict__ in, int64_t n, const uint32_t *__restrict__ sums,
+                                  uint32_t *__restrict__ out) {
+  __shared__ uint32_t s_warp[32];
+  const int64_t base = (int64_t)blockIdx.x * kScanTile + (int64_t)threadIdx.x * kScanItems;
+  uint32_t v[kScanItems];
+  uint32_t mine = 0;
+#pragma unroll
+  for (int t = 0; t < kScanItems; ++t) {
+    v[t] = (base + t < n) ? in[base + t] : 0;
+    mine += v[t];
+  }
+  uint32_t run = sums[blockIdx.x] + block_exclusive_scan(mine, s_warp, nullptr);
+#pragma unroll
+  for (int t = 0; t < kScanItems; ++t) {
+    if (base + t < n) out[base + t] = run;
+    run += v[t];
+  }
+}
+
+// out = exclusive scan of in (may alias); tmp holds ceil(n / kScanTile) words; total (device) optional.
+static comet_status_t exclusive_scan(Context *ctx, const uint32_t *in, uint32_t *out, int64_t n, uint32_t *tmp,
+                                     uint32_t *total, cudaStream_t s) {
+  if (n <= 0) {
+    if (total) COMET_CUDA_TRY(ctx, cudaMemsetAsync(total, 0, sizeof(uint32_t), s));
+    return COMET_OK;
+  }
+  const int64_t tiles = ceil_div(n, kScanTile);
+  scan_tile_sums_kernel<<<(unsigned)tiles, kScanThreads, 0, s>>>(in, n, tmp);
+  scan_sums_kernel<<<1, 1024, 0, s>>>(tmp, tiles, total);
+  scan_apply_kernel<<<(unsigned)tiles, kScanThreads, 0, s>>>(in, n, tmp, out);
+  COMET_LAUNCH_CHECK(ctx);
+  return COMET_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ radix sort
+__global__ void __launch_bounds__(kSortThreads) radix_histogram_kernel(const uint64_t *__restrict__ keys, int64_t n,
+                                                                       int shift, int64_t tiles,
+                                                                       uint32_t *__restrict__ table) {
+  __shared__ uint32_t s_cnt[256];
+  s_cnt[threadIdx.x] = 0;
+  __syncthreads();
+  const int64_t base = (int64_t)blockIdx.x * kSortTile;
+#pragma unroll
+  for (int t = 0; t < kSortItems; ++t) {
+    const int64_t i = base + (int64_t)t * kSortThreads + threadIdx.x;
+    if (i < n) atomicAdd(&s_cnt[(keys[i] >> shift) & 255], 1u);
+  }
+  __syncthreads();
+  table[(int64_t)threadIdx.x * tiles + blockIdx.x] = s_cnt[threadIdx.x];     // digit-major
+}
+
+__global__ void __launch_bounds__(kSortThreads) radix_scatter_kernel(
+    const uint64_t *__restrict__ kin, const uint32_t *__restrict__ pin, uint64_t *__restrict__ kout,
+    uint32_t *__restrict__ pout, const uint32_t *__restrict__ table, int64_t n, int shift, int64_t tiles) {
+  __shared__ uint32_t s_cnt[kSortWarps][256];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int w = 0; w < kSortWarps; ++w) s_cnt[w][tid] = 0;
+  __syncthreads();
+
+  // Item r of lane l of warp w sits at tile_base + w*(32*ITEMS) + r*32 + l: memory order is (w, r, l).
+  const int64_t warp_base = (int64_t)blockIdx.x * kSortTile + (int64_t)warp * (32 * kSortItems);
+  uint64_t key[kSortItems];
+  uint32_t pay[kSortItems];
+  uint32_t rank[kSortItems];
+  const unsigned lt = (1u << lane) - 1u;
+#pragma unroll
+  for (int r = 0; r < kSortItems; ++r) {
+    const int64_t i = warp_base + r * 32 + lane;
+    const bool valid = i < n;
+    key[r] = valid ? kin[i] : ~0ull;          // slots past the end rank after every real key of the tile
+    pay[r] = valid ? pin[i] : 0u;
+    const uint32_t d = (uint32_t)(key[r] >> shift) & 255u;
+    const unsigned peers = __match_any_sync(0xffffffffu, d);
+    const int leader = __ffs(peers) - 1;
+    uint32_t old = 0;
+    if (lane == leader) {
+      old = s_cnt[warp][d];
+      s_cnt[warp][d] = old + __popc(peers);
+    }
+    old = __shfl_sync(0xffffffffu, old, leader);
+    rank[r] = old + __popc(peers & lt);
+    __syncwarp();
+  }
+  __syncthreads();
+  {
+    // digit `tid`: where each warp's run of this digit starts in the output
+    uint32_t run = table[(int64_t)tid * tiles + blockIdx.x];
+#pragma unroll
+    for (int w = 0; w < kSortWarps; ++w) {
+      const uint32_t c = s_cnt[w][tid];
+      s_cnt[w][tid] = run;
+      run += c;
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int r = 0; r < kSortItems; ++r) {
+    const int64_t i = warp_base + r * 32 + lane;
+    if (i < n) {
+      const uint32_t d = (uint32_t)(key[r] >> shift) & 255u;
+      const uint32_t dst = s_cnt[warp][d] + rank[r];
+      kout[dst] = key[r];
+      pout[dst] = pay[r];
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ levels
+struct LevelPlan {
+  int order;
+  int attr[COMET_MAX_ORDER];
+  int shift[COMET_MAX_ORDER];
+  int bits[COMET_MAX_ORDER];
+  int counted[COMET_MAX_ORDER];     // index of the level's node counter (-1: positions are entry ranks or dense)
+  int ncounted;
+};
+
+__device__ __forceinline__ bool is_head(uint64_t k, uint64_t kprev, bool first, int shift) {
+  return first || (k >> shift) != (kprev >> shift);
+}
+
+constexpr int kLevelThreads = 256;
+constexpr int kLevelItems = 8;
+constexpr int kLevelTile = kLevelThreads * kLevelItems;
+
+// Per tile: how many nodes each counted level opens; duplicates (equal adjacent keys) are flagged.
+__global__ void __launch_bounds__(kLevelThreads) level_count_kernel(const uint64_t *__restrict__ keys, int64_t n,
+                                                                    LevelPlan plan, int64_t tiles,
+                                                                    uint32_t *__restrict__ counts,
+                                                                    int32_t *__restrict__ status) {
+  __shared__ uint32_t s_cnt[COMET_MAX_ORDER];
+  if (threadIdx.x < COMET_MAX_ORDER) s_cnt[threadIdx.x] = 0;
+  __syncthreads();
+  const int64_t base = (int64_t)blockIdx.x * kLevelTile;
+  uint32_t mine[COMET_MAX_ORDER] = {0, 0, 0, 0};
+  bool dup = false;
+#pragma unroll
+  for (int t = 0; t < kLevelItems; ++t) {
+    const int64_t p = base + (int64_t)t * kLevelThreads + threadIdx.x;
+    if (p < n) {
+      const uint64_t k = keys[p];
+      const uint64_t kp = p > 0 ? keys[p - 1] : 0;
+      dup |= (p > 0) & (k == kp);
+      for (int l = 0; l < plan.order; ++l)
+        if (plan.counted[l] >= 0 && is_head(k, kp, p == 0, plan.shift[l])) mine[plan.counted[l]] += 1;
+    }
+  }
+  for (int c = 0; c < plan.ncounted; ++c) {
+    uint32_t v = mine[c];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_down_sync(0xffffffffu, v, off);
+    if ((threadIdx.x & 31) == 0 && v) atomicAdd(&s_cnt[c], v);
+  }
+  if (dup) atomicOr(status + kStatusDuplicate, 1);
+  __syncthreads();
+  if (threadIdx.x < plan.ncounted) counts[(int64_t)threadIdx.x * tiles + blockIdx.x] = s_cnt[threadIdx.x];
+}
+
+struct LevelOut {
+  int32_t *pos[COMET_MAX_ORDER];
+  int32_t *crd[COMET_MAX_ORDER];
+  double *val;
+  int64_t dim0;                // extent of level 0 (for a dense root)
+  uint32_t nodes[COMET_MAX_ORDER];   // node count of every counted level
+};
+
+// Per tile: ranks of the heads (tile-local scan + the tile's scanned offset), then crd / pos / val.
+__global__ void __launch_bounds__(kLevelThreads) level_emit_kernel(const uint64_t *__restrict__ keys,
+                                                                   const uint32_t *__restrict__ perm,
+                                                                   const double *__restrict__ val_in, int64_t n,
+                                                                   LevelPlan plan, int64_t tiles,
+                                                                   const uint32_t *__restrict__ offsets,
+                                                                   LevelOut out) {
+  __shared__ uint32_t s_warp[32];
+  const int64_t base = (int64_t)blockIdx.x * kLevelTile + (int64_t)threadIdx.x * kLevelItems;   // blocked: 8 consecutive
+  uint64_t k[kLevelItems + 1];
+  k[0] = (base > 0 && base - 1 < n) ? keys[base - 1] : 0;
+#pragma unroll
+  for (int t = 0; t < kLevelItems; ++t) k[t + 1] = (base + t < n) ? keys[base + t] : 0;
+
+  // rank[l] = nodes of level l opened before this thread's first entry
+  uint32_t rank[COMET_MAX_ORDER];
+  for (int l = 0; l < plan.order; ++l) {
+    rank[l] = 0;
+    if (plan.counted[l] < 0) continue;
+    uint32_t mine = 0;
+#pragma unroll
+    for (int t = 0; t < kLevelItems; ++t)
+      if (base + t < n && is_head(k[t + 1], k[t], base + t == 0, plan.shift[l])) mine += 1;
+    rank[l] = offsets[(int64_t)plan.counted[l] * tiles + blockIdx.x] + block_exclusive_scan(mine, s_warp, nullptr);
+  }
+
+#pragma unroll
+  for (int t = 0; t < kLevelItems; ++t) {
+    const int64_t p = base + t;
+    if (p >= n) break;
+    const uint64_t key = k[t + 1], kp = k[t];
+    const bool first = p == 0;
+    // position of this entry's node at each level (entry rank where the level is not counted)
+    uint32_t parent_pos = 0;
+    bool parent_head = first;      // does this entry open a new node at the parent level?
+    for (int l = 0; l < plan.order; ++l) {
+      const int32_t coord = (int32_t)((key >> plan.shift[l]) & ((1ull << plan.bits[l]) - 1));
+      const int a = plan.attr[l];
+      if (a == COMET_D) {
+        parent_pos = (uint32_t)coord;
+        parent_head = is_head(key, kp, first, plan.shift[l]);
+      } else if (a == COMET_CU) {
+        const bool head = is_head(key, kp, first, plan.shift[l]);
+        const bool leaf = plan.counted[l] < 0;               // leaf level: one node per entry
+        const uint32_t node = leaf ? (uint32_t)p : (head ? rank[l] : rank[l] - 1);
+        if (head) {
+          out.crd[l][node] = coord;
+          if (l == 0) {
+            // root: pos = [0, nodes], written by the host-side finisher
+          } else if (plan.attr[l - 1] == COMET_D) {
+            // dense parent: every parent coordinate after the previous node's and up to this one starts here
+            if (parent_head) {
+              const int64_t prev = first ? -1 : (int64_t)((kp >> plan.shift[l - 1]) & ((1ull << plan.bits[l - 1]) - 1));
+              for (int64_t r = prev + 1; r <= (int64_t)parent_pos; ++r) out.pos[l][r] = (int32_t)node;
+            }
+          } else if (parent_head) {
+            out.pos[l][parent_pos] = (int32_t)node;           // first child of parent node parent_pos
+          }
+        }
+        parent_pos = node;
+        parent_head = head;
+        if (!leaf && head) rank[l] += 1;
+      } else {                                                // CN, S: one position per entry
+        out.crd[l][p] = coord;
+        parent_pos = (uint32_t)p;
+        parent_head = true;
+      }
+    }
+    out.val[p] = val_in[perm[p]];
+  }
+}
+
+// Closes the pos arrays: the terminal entry of every compressed level (and the empty tail of a CSR pos).
+__global__ void level_finish_kernel(const uint64_t *__restrict__ keys, int64_t n, LevelPlan plan, LevelOut out) {
+  const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  uint32_t parents = 1;
+  for (int l = 0; l < plan.order; ++l) {
+    const int a = plan.attr[l];
+    const uint32_t nodes = plan.counted[l] >= 0 ? out.nodes[plan.counted[l]] : (uint32_t)n;
+    if (a == COMET_D) {
+      if (tid == 0) out.pos[l][0] = (int32_t)out.dim0;
+      parents = (uint32_t)out.dim0;
+    } else if (a == COMET_CU) {
+      if (l == 0) {
+        if (tid == 0) { out.pos[0][0] = 0; out.pos[0][1] = (int32_t)nodes; }
+      } else if (plan.attr[l - 1] == COMET_D) {
+        // rows after the last stored one (all rows when the tensor is empty) start at `nodes`
+        const int64_t last = n > 0 ? (int64_t)((keys[n - 1] >> plan.shift[l - 1]) & ((1ull << plan.bits[l - 1]) - 1)) : -1;
+        for (int64_t r = last + 1 + tid; r <= (int64_t)out.dim0; r += (int64_t)gridDim.x * blockDim.x)
+          out.pos[l][r] = (int32_t)nodes;
+      } else if (tid == 0) {
+        out.pos[l][parents] = (int32_t)nodes;
+      }
+      parents = nodes;
+    } else if (a == COMET_CN) {
+      if (tid == 0) { out.pos[l][0] = 0; out.pos[l][1] = (int32_t)n; }
+      parents = (uint32_t)n;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ validate
+__global__ void validate_level_kernel(const int32_t *__restrict__ pos, int64_t parents, const int32_t *__restrict__ crd,
+                                      int64_t crd_len, int64_t dim, int attr, int32_t *__restrict__ status) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  bool bad = false;
+  if (attr == COMET_CU) {
+    if (i == 0) bad |= pos[0] != 0 || (int64_t)pos[parents] != crd_len;
+    if (i < parents) {
+      const int64_t lo = pos[i], hi = pos[i + 1];
+      bad |= lo > hi || lo < 0 || hi > crd_len;
+      if (!bad)
+        for (int64_t q = lo; q < hi; ++q) {
+          const int32_t c = crd[q];
+          bad |= c < 0 || c >= dim || (q > lo && crd[q - 1] >= c);
+        }
+    }
+  } else if (i < crd_len) {
+    const int32_t c = crd[i];
+    bad |= c < 0 || c >= dim;
+    if (attr == COMET_CN && i > 0) bad |= crd[i - 1] > c;
+  }
+  if (bad) atomicOr(status + kStatusInvalid, 1);
+}
+
+}  // namespace comet
+
+using namespace comet;
+
+namespace {
+
+int bits_for(int64_t dim) {          // bits needed for coordinates 0 .. dim-1
+  int b = 0;
+  while (b < 62 && (1ll << b) < dim) ++b;
+  return b;
+}
+
+bool supported_attrs(int order, const int32_t *attr) {
+  bool coo = attr[0] == COMET_CN, csf = attr[0] == COMET_CU, dcs = attr[0] == COMET_D;
+  for (int l = 1; l < order; ++l) {
+    coo = coo && attr[l] == COMET_S;
+    csf = csf && attr[l] == COMET_CU;
+    dcs = dcs && attr[l] == COMET_CU;
+  }
+  return order >= 2 && (coo || csf || dcs);
+}
+
+struct TempBlocks {
+  Context *ctx;
+  cudaStream_t s;
+  void *p[8];
+  int n = 0;
+  TempBlocks(Context *c, cudaStream_t st) : ctx(c), s(st) {}
+  void *get(size_t bytes) {
+    void *q = ctx_alloc(ctx, bytes, s);
+    if (q) p[n++] = q;
+    return q;
+  }
+  ~TempBlocks() { for (int i = 0; i < n; ++i) ctx_free(ctx, p[i], s); }
+};
+
+}  // namespace
+
+extern "C" comet_status_t comet_pack(comet_handle_t handle, int32_t order, const int64_t *h_dims, int64_t nnz,
+                                     const int32_t *const *h_coo_crd, const void *coo_val, comet_dtype_t dtype,
+                                     const int32_t *h_mode_order, const int32_t *h_attr, void *stream,
+                                     comet_sptensor_t *out) {
+  if (!handle || !out || !h_dims || !h_coo_crd || !h_mode_order || !h_attr) return COMET_ERR_INVALID_ARG;
+  memset(out, 0, sizeof(*out));
+  if (order < 1 || order > COMET_MAX_ORDER || nnz < 0) return COMET_ERR_INVALID_ARG;
+  if (dtype != COMET_F64) return COMET_ERR_UNSUPPORTED_FORMAT;
+  if (nnz > 2147483647ll - 1024) return COMET_ERR_INDEX_OVERFLOW;
+  bool seen[COMET_MAX_ORDER] = {false, false, false, false};
+  for (int l = 0; l < order; ++l) {
+    const int m = h_mode_order[l];
+    if (m < 0 || m >= order || seen[m]) return COMET_ERR_INVALID_ARG;
+    seen[m] = true;
+    if (h_attr[l] < COMET_D || h_attr[l] > COMET_S) return COMET_ERR_INVALID_ARG;
+    if (h_dims[l] < 0) return COMET_ERR_INVALID_ARG;
+    if (h_dims[l] > 2147483646ll) return COMET_ERR_INDEX_OVERFLOW;
+    if (nnz > 0 && !h_coo_crd[l]) return COMET_ERR_INVALID_ARG;
+  }
+  if (nnz > 0 && !coo_val) return COMET_ERR_INVALID_ARG;
+  if (!supported_attrs(order, h_attr)) return COMET_ERR_UNSUPPORTED_FORMAT;
+
+  Context *ctx = reinterpret_cast<Context *>(handle);
+  cudaStream_t s = (cudaStream_t)stream;
+
+  KeyLayout key{};
+  LevelPlan plan{};
+  CoordPtrs coords{};
+  key.order = plan.order = order;
+  int total_bits = 0;
+  for (int l = order - 1; l >= 0; --l) {
+    const int m = h_mode_order[l];
+    key.dim[l] = h_dims[m];
+    key.bits[l] = plan.bits[l] = bits_for(h_dims[m]);
+    key.shift[l] = plan.shift[l] = total_bits;
+    total_bits += key.bits[l];
+    plan.attr[l] = h_attr[l];
+    coords.p[l] = h_coo_crd[m];
+  }
+  if (total_bits > 63) return COMET_ERR_UNSUPPORTED_FORMAT;   // the coordinate bits must fit one 64-bit key
+  key.total_bits = total_bits;
+  plan.ncounted = 0;
+  for (int l = 0; l < order; ++l) {
+    // a compressed-unique level above the leaf has fewer nodes than entries and needs a node counter
+    plan.counted[l] = (plan.attr[l] == COMET_CU && l < order - 1) ? plan.ncounted++ : -1;
+  }
+  if (h_attr[0] == COMET_D && h_dims[h_mode_order[0]] == 0 && nnz > 0) return COMET_ERR_COORD_OUT_OF_RANGE;
+
+  const int64_t n = nnz;
+  const int64_t sort_tiles = ceil_div(n > 0 ? n : 1, kSortTile);
+  const int64_t level_tiles = ceil_div(n > 0 ? n : 1, kLevelTile);
+  const int64_t table_len = 256 * sort_tiles;
+  const int64_t counts_len = (int64_t)COMET_MAX_ORDER * level_tiles;
+
+  TempBlocks tmp(ctx, s);
+  uint64_t *keys_a = (uint64_t *)tmp.get((size_t)(n + 1) * 8);
+  uint64_t *keys_b = (uint64_t *)tmp.get((size_t)(n + 1) * 8);
+  uint32_t *perm_a = (uint32_t *)tmp.get((size_t)(n + 1) * 4);
+  uint32_t *perm_b = (uint32_t *)tmp.get((size_t)(n + 1) * 4);
+  const int64_t table_words = table_len > counts_len ? table_len : counts_len;
+  uint32_t *table = (uint32_t *)tmp.get((size_t)table_words * 4);
+  uint32_t *scan_tmp = (uint32_t *)tmp.get((size_t)(ceil_div(table_words, kScanTile) + 1) * 4);
+  if (!keys_a || !keys_b || !perm_a || !perm_b || !table || !scan_tmp) return COMET_ERR_ALLOC;
+
+  COMET_CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_status, 0, 16 * sizeof(int32_t), s));
+  uint32_t *d_nodes = reinterpret_cast<uint32_t *>(ctx->d_status) + 8;   // node counts live beside the status words
+
+  if (n > 0) {
+    make_keys_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(coords, key, n, keys_a, perm_a, ctx->d_status);
+    COMET_LAUNCH_CHECK(ctx);
+    for (int shift = 0; shift < total_bits; shift += 8) {
+      radix_histogram_kernel<<<(unsigned)sort_tiles, kSortThreads, 0, s>>>(keys_a, n, shift, sort_tiles, table);
+      COMET_LAUNCH_CHECK(ctx);
+      comet_status_t st = exclusive_scan(ctx, table, table, table_len, scan_tmp, nullptr, s);
+      if (st != COMET_OK) return st;
+      radix_scatter_kernel<<<(unsigned)sort_tiles, kSortThreads, 0, s>>>(keys_a, perm_a, keys_b, perm_b, table, n,
+                                                                         shift, sort_tiles);
+      COMET_LAUNCH_CHECK(ctx);
+      uint64_t *tk = keys_a; keys_a = keys_b; keys_b = tk;
+      uint32_t *tp = perm_a; perm_a = perm_b; perm_b = tp;
+    }
+    // node counts of the counted levels: per-tile counts -> scanned offsets (kept in `table`) + totals
+    level_count_kernel<<<(unsigned)level_tiles, kLevelThreads, 0, s>>>(keys_a, n, plan, level_tiles, table,
+                                                                       ctx->d_status);
+    COMET_LAUNCH_CHECK(ctx);
+    for (int c = 0; c < plan.ncounted; ++c) {
+      comet_status_t st = exclusive_scan(ctx, table + (int64_t)c * level_tiles, table + (int64_t)c * level_tiles,
+                                         level_tiles, scan_tmp, d_nodes + c, s);
+      if (st != COMET_OK) return st;
+    }
+  }
+  // the one synchronisation: status words and node counts
+  COMET_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->h_pinned, ctx->d_status, 16 * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  COMET_CUDA_TRY(ctx, cudaStreamSynchronize(s));
+  if (ctx->h_pinned[kStatusRange]) return COMET_ERR_COORD_OUT_OF_RANGE;
+  if (ctx->h_pinned[kStatusDuplicate]) return COMET_ERR_DUPLICATE_COORD;
+
+  // exact allocation
+  void *owner = owner_new();
+  if (!owner) return COMET_ERR_ALLOC;
+  LevelOut lo{};
+  bool alloc_ok = true;
+  out->order = order;
+  out->dtype = COMET_F64;
+  out->nnz = n;
+  int64_t parents = 1;
+  for (int l = 0; l < order; ++l) {
+    out->dims[l] = h_dims[l];
+    out->mode_order[l] = h_mode_order[l];
+    out->attr[l] = h_attr[l];
+    const int64_t nodes = plan.counted[l] >= 0 ? (int64_t)reinterpret_cast<uint32_t *>(ctx->h_pinned)[8 + plan.counted[l]] : n;
+    if (plan.counted[l] >= 0) lo.nodes[plan.counted[l]] = (uint32_t)nodes;
+    int64_t pos_len = 0, crd_len = 0;
+    if (h_attr[l] == COMET_D) { pos_len = 1; parents = key.dim[l]; }
+    else if (h_attr[l] == COMET_CU) { pos_len = parents + 1; crd_len = nodes; parents = nodes; }
+    else if (h_attr[l] == COMET_CN) { pos_len = 2; crd_len = n; parents = n; }
+    else { crd_len = n; }
+    out->pos_len[l] = pos_len;
+    out->crd_len[l] = crd_len;
+    if (pos_len) { out->pos[l] = (int32_t *)owner_alloc(ctx, owner, (size_t)pos_len * 4, s); alloc_ok &= out->pos[l] != nullptr; }
+    if (crd_len) { out->crd[l] = (int32_t *)owner_alloc(ctx, owner, (size_t)crd_len * 4, s); alloc_ok &= out->crd[l] != nullptr; }
+    lo.pos[l] = out->pos[l];
+    lo.crd[l] = out->crd[l];
+  }
+  if (n > 0) { out->val = owner_alloc(ctx, owner, (size_t)n * 8, s); alloc_ok &= out->val != nullptr; }
+  lo.val = (double *)out->val;
+  lo.dim0 = key.dim[0];
+  if (!alloc_ok) { owner_release(ctx, owner, s); memset(out, 0, sizeof(*out)); return COMET_ERR_ALLOC; }
+
+  if (n > 0)
+    level_emit_kernel<<<(unsigned)level_tiles, kLevelThreads, 0, s>>>(keys_a, perm_a, (const double *)coo_val, n, plan,
+                                                                      level_tiles, table, lo);
+  level_finish_kernel<<<kSmCount, 256, 0, s>>>(keys_a, n, plan, lo);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { owner_release(ctx, owner, s); memset(out, 0, sizeof(*out)); return cuda_fail(ctx, e); }
+  out->owner = owner;
+  return COMET_OK;
+}
+
+extern "C" comet_status_t comet_validate(comet_handle_t handle, const comet_sptensor_t *t, void *stream) {
+  if (!handle || !t) return COMET_ERR_INVALID_ARG;
+  if (t->order < 1 || t->order > COMET_MAX_ORDER || t->nnz < 0) return COMET_ERR_INVALID_ARG;
+  Context *ctx = reinterpret_cast<Context *>(handle);
+  cudaStream_t s = (cudaStream_t)stream;
+  // host-visible shape checks first
+  int64_t parents = 1;
+  for (int l = 0; l < t->order; ++l) {
+    const int a = t->attr[l];
+    const int64_t dim = t->dims[t->mode_order[l]];
+    if (a == COMET_D) {
+      if (t->pos_len[l] != 1 || !t->pos[l]) return COMET_ERR_INVALID_TENSOR;
+      for (int u = 0; u < l; ++u) if (t->attr[u] != COMET_D) return COMET_ERR_UNSUPPORTED_FORMAT;
+      parents *= dim;
+    } else if (a == COMET_CU) {
+      if (t->pos_len[l] != parents + 1 || !t->pos[l] || (t->crd_len[l] > 0 && !t->crd[l])) return COMET_ERR_INVALID_TENSOR;
+      parents = t->crd_len[l];
+    } else if (a == COMET_CN) {
+      if (l != 0) return COMET_ERR_UNSUPPORTED_FORMAT;
+      if (t->pos_len[l] != 2 || !t->pos[l] || t->crd_len[l] != t->nnz) return COMET_ERR_INVALID_TENSOR;
+      parents = t->nnz;
+    } else if (a == COMET_S) {
+      if (l == 0 || (t->attr[l - 1] != COMET_CN && t->attr[l - 1] != COMET_S)) return COMET_ERR_UNSUPPORTED_FORMAT;
+      if (t->crd_len[l] != parents) return COMET_ERR_INVALID_TENSOR;
+    } else {
+      return COMET_ERR_INVALID_ARG;
+    }
+  }
+  if (t->attr[t->order - 1] != COMET_D && parents != t->nnz) return COMET_ERR_INVALID_TENSOR;
+
+  COMET_CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_status, 0, 16 * sizeof(int32_t), s));
+  parents = 1;
+  for (int l = 0; l < t->order; ++l) {
+    const int a = t->attr[l];
+    const int64_t dim = t->dims[t->mode_order[l]];
+    if (a == COMET_D) { parents *= dim; continue; }
+    const int64_t work = a == COMET_CU ? (parents > 0 ? parents : 1) : t->crd_len[l];
+    if (work > 0) {
+      validate_level_kernel<<<(unsigned)ceil_div(work, 256), 256, 0, s>>>(t->pos[l], parents, t->crd[l], t->crd_len[l],
+                                                                          dim, a, ctx->d_status);
+      COMET_LAUNCH_CHECK(ctx);
+    }
+    parents = a == COMET_S ? parents : t->crd_len[l];
+  }
+  COMET_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->h_pinned, ctx->d_status, 16 * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  COMET_CUDA_TRY(ctx, cudaStreamSynchronize(s));
+  return ctx->h_pinned[kStatusInvalid] ? COMET_ERR_INVALID_TENSOR : COMET_OK;
 }

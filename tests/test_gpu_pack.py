@@ -1,0 +1,147 @@
+"""GPU parity of comet_pack: every level array must equal the oracle's bit for bit (int32 arrays as
+integers, values as 64-bit patterns), for every supported attribute tuple, storage order and order."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+from oracle import D, CU, CN, S
+
+pytestmark = pytest.mark.gpu
+
+comet = pytest.importorskip("paper_2102_05187_b200")
+from gpu_util import assert_close, assert_equal_arrays, dev  # noqa: E402
+
+
+@pytest.fixture(autouse=True)
+def _need_gpu(cuda_device):
+    yield
+
+
+def _np(coords):
+    return [c.numpy() for c in coords]
+
+
+def check_pack(coords, val, dims, mode_order, attr):
+    want = oracle.pack(_np(coords), val.numpy(), dims, mode_order, attr)
+    got = comet.pack([c.cuda() for c in coords], val.cuda(), dims, mode_order, attr)
+    assert got.order == len(dims) and got.nnz == len(val) and got.attr == tuple(attr)
+    assert got.mode_order == tuple(mode_order) and got.dims == tuple(dims)
+    for l in range(len(dims)):
+        assert_equal_arrays(got.pos(l), want.pos[l], f"pos[{l}] {attr} {mode_order}")
+        assert_equal_arrays(got.crd(l), want.crd[l], f"crd[{l}] {attr} {mode_order}")
+    assert_equal_arrays(got.val, want.val, "val")
+    comet.validate(got)
+    return got
+
+
+FORMATS_2D = [(CN, S), (D, CU), (CU, CU)]
+FORMATS_3D = [(CN, S, S), (CU, CU, CU), (D, CU, CU)]
+
+
+@pytest.mark.parametrize("attr", FORMATS_2D)
+@pytest.mark.parametrize("mode_order", [(0, 1), (1, 0)])
+@pytest.mark.parametrize("dims,nnz,seed", [((7, 5), 12, 1), ((1, 9), 4, 2), ((9, 1), 4, 3), ((6, 6), 36, 4),
+                                           ((8, 8), 1, 5), ((8, 8), 0, 6), ((300, 200), 5000, 7),
+                                           ((5000, 3), 9000, 8), ((3, 70000), 20000, 9), ((1, 1), 1, 10)])
+def test_pack_matrices(attr, mode_order, dims, nnz, seed):
+    coords, val = synth.random_coo(dims, nnz, seed)
+    check_pack(coords, val, dims, mode_order, attr)
+
+
+@pytest.mark.parametrize("attr", FORMATS_3D)
+@pytest.mark.parametrize("mode_order", [(0, 1, 2), (1, 0, 2), (2, 1, 0), (1, 2, 0)])
+@pytest.mark.parametrize("dims,nnz,seed", [((4, 5, 6), 30, 1), ((3, 1, 7), 9, 2), ((5, 5, 5), 125, 3),
+                                           ((6, 4, 3), 0, 4), ((9, 8, 7), 1, 5), ((60, 50, 40), 20000, 6),
+                                           ((2000, 3, 1000), 30000, 7)])
+def test_pack_tensors(attr, mode_order, dims, nnz, seed):
+    coords, val = synth.random_coo(dims, nnz, seed)
+    check_pack(coords, val, dims, mode_order, attr)
+
+
+def test_pack_order4():
+    dims = (9, 8, 7, 6)
+    coords, val = synth.random_coo(dims, 1500, 11)
+    for attr in [(CU, CU, CU, CU), (CN, S, S, S), (D, CU, CU, CU)]:
+        check_pack(coords, val, dims, (0, 1, 2, 3), attr)
+        check_pack(coords, val, dims, (3, 1, 0, 2), attr)
+
+
+def test_pack_large_extents_use_many_radix_passes():
+    dims = (1_000_000, 500_000, 200_000)            # 57 key bits: 8 passes
+    coords, val = synth.random_coo(dims, 60_000, 12)
+    check_pack(coords, val, dims, (0, 1, 2), (CU, CU, CU))
+    check_pack(coords, val, dims, (0, 1, 2), (CN, S, S))
+
+
+@pytest.mark.parametrize("config,attr", [(1, (D, CU)), (2, (D, CU)), (3, (CU, CU, CU)), (4, (CU, CU, CU)),
+                                         (5, (CN, S, S)), (5, (CU, CU, CU))])
+def test_pack_scaled_workloads(config, attr):
+    case = synth.make(config, scale=1 / 64)
+    order = tuple(range(len(case.dims)))
+    check_pack(case.coords, case.val, case.dims, order, attr)
+
+
+def test_shuffled_input_gives_identical_arrays():
+    dims = (50, 40, 30)
+    coords, val = synth.random_coo(dims, 8000, 21)
+    a = comet.pack([c.cuda() for c in coords], val.cuda(), dims, (0, 1, 2), (CU, CU, CU))
+    p = torch.randperm(len(val), generator=torch.Generator().manual_seed(3))
+    b = comet.pack([c[p].cuda() for c in coords], val[p].cuda(), dims, (0, 1, 2), (CU, CU, CU))
+    for l in range(3):
+        assert torch.equal(a.pos(l), b.pos(l)) and torch.equal(a.crd(l), b.crd(l))
+    assert torch.equal(a.val, b.val)
+
+
+def test_rejected_inputs():
+    i = torch.tensor([0, 0], dtype=torch.int32).cuda()
+    j = torch.tensor([1, 1], dtype=torch.int32).cuda()
+    v = torch.ones(2, dtype=torch.float64).cuda()
+    for attr in [(D, CU), (CN, S), (CU, CU)]:
+        with pytest.raises(comet.CometError) as e:
+            comet.pack([i, j], v, (2, 2), (0, 1), attr)
+        assert e.value.status == -4                      # duplicate coordinate
+    with pytest.raises(comet.CometError) as e:
+        comet.pack([i, torch.tensor([1, 2], dtype=torch.int32).cuda()], v, (2, 2), (0, 1), (D, CU))
+    assert e.value.status == -3                          # out of range
+    with pytest.raises(comet.CometError) as e:
+        comet.pack([i, torch.tensor([-1, 0], dtype=torch.int32).cuda()], v, (2, 2), (0, 1), (D, CU))
+    assert e.value.status == -3
+    for bad in [(CU, D), (CU, CN), (CU, S), (S, S), (D, D)]:
+        with pytest.raises(comet.CometError) as e:
+            comet.pack([i, j], v, (2, 2), (0, 1), bad)
+        assert e.value.status == -2
+    with pytest.raises(comet.CometError) as e:
+        comet.pack([i, j], v, (2, 2), (0, 0), (D, CU))
+    assert e.value.status == -1
+    # the handle is still usable afterwards
+    ok = comet.pack([torch.tensor([0, 1], dtype=torch.int32).cuda(), j], v, (2, 2), (0, 1), (D, CU))
+    assert ok.pos(1).tolist() == [0, 1, 2]
+
+
+def test_validate_catches_broken_descriptors():
+    dims = (30, 20)
+    coords, val = synth.random_coo(dims, 200, 5)
+    pk = oracle.pack(_np(coords), val.numpy(), dims, (0, 1), (D, CU))
+    def build(pos1, crd1):
+        return comet.SpTensor.from_arrays(dims, (0, 1), (D, CU), [dev(pk.pos[0], torch.int32), dev(pos1, torch.int32)],
+                                          [None, dev(crd1, torch.int32)], dev(pk.val))
+    comet.validate(build(pk.pos[1], pk.crd[1]))
+    bad_pos = pk.pos[1].copy(); bad_pos[5] = bad_pos[6] + 1
+    bad_crd = pk.crd[1].copy(); bad_crd[3] = dims[1]
+    unsorted = pk.crd[1].copy()
+    row = int(np.argmax(np.diff(pk.pos[1]) >= 2))
+    a = pk.pos[1][row]; unsorted[a], unsorted[a + 1] = unsorted[a + 1], unsorted[a]
+    for pos1, crd1 in [(bad_pos, pk.crd[1]), (pk.pos[1], bad_crd), (pk.pos[1], unsorted)]:
+        with pytest.raises(comet.CometError) as e:
+            comet.validate(build(pos1, crd1))
+        assert e.value.status == -10
+
+
+def test_pack_then_contract_end_to_end():
+    case = synth.make(4, scale=1 / 64)
+    X = comet.pack([c.cuda() for c in case.coords], case.val.cuda(), case.dims, (0, 1, 2), (CU, CU, CU))
+    Y = comet.ttm(X, 2, case.dense["U"].cuda())
+    _, want, norm = oracle.ttm(_np(case.coords), case.val.numpy(), case.dims, 2, case.dense["U"].numpy())
+    assert_close(Y.val.reshape(-1, case.R), want, norm, what="pack+ttm")
