@@ -96,6 +96,8 @@ comet_status_t comet_destroy(comet_handle_t handle);
 const char *comet_status_string(comet_status_t status);
 /* The cudaError_t (as int) of the last failing CUDA call seen by this handle, 0 if none. */
 int comet_last_cuda_error(comet_handle_t handle);
+/* Number of CUDA kernels this handle has launched since comet_create (accounting for benchmarks). */
+int64_t comet_kernel_launches(comet_handle_t handle);
 
 /* COO -> packed format (the format conversion the paper's input-reading runtime function performs
  * after reading a COO file; Tensor Storage Format section for what each level holds).

@@ -28,7 +28,8 @@ STATUS_NAMES = {
 }
 
 EXPORTS = [
-    "comet_create", "comet_destroy", "comet_status_string", "comet_last_cuda_error", "comet_pack",
+    "comet_create", "comet_destroy", "comet_status_string", "comet_last_cuda_error", "comet_kernel_launches",
+    "comet_pack",
     "comet_sptensor_free", "comet_validate", "comet_spmv", "comet_spmm", "comet_ttv_symbolic", "comet_ttv",
     "comet_ttm_symbolic", "comet_ttm", "comet_mttkrp",
 ]
@@ -79,8 +80,10 @@ def load_library():
             raise ImportError(f"libcomet.so does not export {name}")
     lib.comet_status_string.restype = C.c_char_p
     lib.comet_status_string.argtypes = [C.c_int]
+    lib.comet_kernel_launches.restype = C.c_int64
+    lib.comet_kernel_launches.argtypes = [C.c_void_p]
     for name in EXPORTS:
-        if name not in ("comet_status_string",):
+        if name not in ("comet_status_string", "comet_kernel_launches"):
             getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -138,6 +141,10 @@ class Handle:
             self.close()
         except Exception:
             pass
+
+    def kernel_launches(self) -> int:
+        """Kernels launched through this handle so far."""
+        return int(self.lib.comet_kernel_launches(self._h))
 
     def check(self, st: int, what: str):
         if st:
@@ -359,3 +366,19 @@ def mttkrp(X: SpTensor, mode: int, factors, out: torch.Tensor | None = None) -> 
                                    C.c_int64(out.stride(0)), _stream_ptr())
     X.handle.check(st, "comet_mttkrp")
     return out
+
+
+def spmm_from_host(h_coords, h_val, dims, h_B, h_out, handle: Handle | None = None):
+    """The whole SpMM path from HOST buffers: copies the COO entries and B to the device (pinned host
+    tensors make the copies asynchronous), packs to CSR, multiplies, and copies C back into `h_out`.
+    Returns after the result has landed in `h_out`."""
+    handle = handle or default_handle()
+    coords = [c.to("cuda", non_blocking=True) for c in h_coords]
+    val = h_val.to("cuda", non_blocking=True)
+    B = h_B.to("cuda", non_blocking=True)
+    A = pack(coords, val, dims, (0, 1), (D, CU), handle)
+    C_dev = spmm(A, B)
+    h_out.copy_(C_dev, non_blocking=True)
+    torch.cuda.current_stream().synchronize()
+    A.free()
+    return h_out

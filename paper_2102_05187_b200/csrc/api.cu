@@ -195,6 +195,7 @@ extern "C" comet_status_t comet_ttv_symbolic(comet_handle_t handle, const comet_
     if (st == COMET_OK) {
       set_word_kernel<<<1, 1, 0, s>>>(Y->pos[0], (int32_t)rows);
       expand_root_pos_kernel<<<(unsigned)ceil_div(rows + 1, 256), 256, 0, s>>>(X->crd[0], X->pos[1], S, rows, Y->pos[1]);
+      ctx->launches += 2;
       cudaError_t e = cudaGetLastError();
       if (e == cudaSuccess && F)
         e = cudaMemcpyAsync(Y->crd[1], X->crd[1], (size_t)F * 4, cudaMemcpyDeviceToDevice, s);
@@ -248,6 +249,7 @@ extern "C" comet_status_t comet_ttm_symbolic(comet_handle_t handle, const comet_
     if (!Y->pos[2] || !Y->val) st = COMET_ERR_ALLOC;
     else {
       set_word_kernel<<<1, 1, 0, s>>>(Y->pos[2], (int32_t)R);
+      ctx->launches += 1;
       cudaError_t e = cudaGetLastError();
       if (e != cudaSuccess) st = cuda_fail(ctx, e);
     }

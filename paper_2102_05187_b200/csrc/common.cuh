@@ -20,6 +20,7 @@ struct Context {
   size_t scratch_bytes;
   int32_t *h_pinned;                      // small pinned buffer for device->host size reads
   int32_t *d_status;                      // device words written by checking kernels
+  int64_t launches;                       // kernels launched through this handle (for accounting)
 };
 
 // Grows the cached scratch buffer to at least `bytes` and returns it (NULL on allocation failure).
@@ -34,7 +35,13 @@ comet_status_t cuda_fail(Context *ctx, cudaError_t e);
     if (e__ != cudaSuccess) return cuda_fail((ctx), e__); \
   } while (0)
 
-#define COMET_LAUNCH_CHECK(ctx) COMET_CUDA_TRY((ctx), cudaGetLastError())
+// After a kernel launch (or `n` back-to-back launches): count them and surface a launch error.
+#define COMET_LAUNCHED(ctx, n)                       \
+  do {                                               \
+    (ctx)->launches += (n);                          \
+    COMET_CUDA_TRY((ctx), cudaGetLastError());       \
+  } while (0)
+#define COMET_LAUNCH_CHECK(ctx) COMET_LAUNCHED(ctx, 1)
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }

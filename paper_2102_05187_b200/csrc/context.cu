@@ -58,6 +58,7 @@ extern "C" comet_status_t comet_create(comet_handle_t *handle, const comet_alloc
   else ctx->allocator = comet_allocator_t{comet::default_alloc, comet::default_free, nullptr};
   ctx->device = dev;
   ctx->last_cuda_error = 0;
+  ctx->launches = 0;
   ctx->scratch = nullptr;
   ctx->scratch_bytes = 0;
   ctx->h_pinned = nullptr;
@@ -86,6 +87,10 @@ extern "C" comet_status_t comet_destroy(comet_handle_t handle) {
 
 extern "C" int comet_last_cuda_error(comet_handle_t handle) {
   return handle ? reinterpret_cast<Context *>(handle)->last_cuda_error : 0;
+}
+
+extern "C" int64_t comet_kernel_launches(comet_handle_t handle) {
+  return handle ? reinterpret_cast<Context *>(handle)->launches : 0;
 }
 
 extern "C" const char *comet_status_string(comet_status_t s) {

@@ -147,7 +147,7 @@ static comet_status_t exclusive_scan(Context *ctx, const uint32_t *in, uint32_t 
   scan_tile_sums_kernel<<<(unsigned)tiles, kScanThreads, 0, s>>>(in, n, tmp);
   scan_sums_kernel<<<1, 1024, 0, s>>>(tmp, tiles, total);
   scan_apply_kernel<<<(unsigned)tiles, kScanThreads, 0, s>>>(in, n, tmp, out);
-  COMET_LAUNCH_CHECK(ctx);
+  COMET_LAUNCHED(ctx, 3);
   return COMET_OK;
 }
 
@@ -579,6 +579,7 @@ extern "C" comet_status_t comet_pack(comet_handle_t handle, int32_t order, const
     level_emit_kernel<<<(unsigned)level_tiles, kLevelThreads, 0, s>>>(keys_a, perm_a, (const double *)coo_val, n, plan,
                                                                       level_tiles, table, lo);
   level_finish_kernel<<<kSmCount, 256, 0, s>>>(keys_a, n, plan, lo);
+  ctx->launches += n > 0 ? 2 : 1;
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { owner_release(ctx, owner, s); memset(out, 0, sizeof(*out)); return cuda_fail(ctx, e); }
   out->owner = owner;
