@@ -167,6 +167,29 @@ comet_status_t comet_mttkrp(comet_handle_t handle, const comet_sptensor_t *X, in
                             const void *const *h_factors, const int64_t *h_ld, int64_t R, void *out, int64_t ldo,
                             void *stream);
 
+/* CSR SpMV without any allocation (the paper has no counterpart; this exists for deployment only).
+ *
+ * Who needs it: callers that cannot obtain device memory at call time. Examples are a service whose
+ * whole GPU has been handed to another component's memory pool, so that a driver allocation would
+ * fail or stall, and a latency-critical loop in which a driver allocation (it can take a lock and
+ * synchronise the device) is not acceptable. comet_spmv needs a handle, and a handle gets its
+ * scratch from an allocator; this entry point needs neither. It calls no cudaMalloc, cudaFree or
+ * any other allocating routine, directly or through a library.
+ *
+ * Same result as comet_spmv for A = [D,CU] (other formats: COMET_ERR_UNSUPPORTED_FORMAT). The caller
+ * still passes the inputs and the output (device pointers, y has dims[mode_order[0]] entries and is
+ * fully overwritten). The per-tile carry slots live in a fixed 768 KiB device array that is part of
+ * the library image: every GPU that loads the library holds it until the process exits.
+ *   - Limit: rows + nnz <= 134,217,728 (65,536 tiles of 2,048 merge items); larger problems return
+ *     COMET_ERR_WORKSPACE and must use comet_spmv.
+ *   - The first call on each device looks up the array's device address (with that device current)
+ *     and remembers it; make that first call outside any stream capture.
+ *   - All calls share the one array, which keeps whatever the previous call left in it (each call
+ *     overwrites every slot it reads, so nothing has to be cleared). Two calls that overlap on the
+ *     GPU -- different streams, or different threads -- race on it: serialise them.
+ *   - Asynchronous on `stream`; errors are return codes as everywhere else. */
+comet_status_t comet_spmv_static(const comet_sptensor_t *A, const void *x, void *y, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -31,7 +31,7 @@ EXPORTS = [
     "comet_create", "comet_destroy", "comet_status_string", "comet_last_cuda_error", "comet_kernel_launches",
     "comet_pack",
     "comet_sptensor_free", "comet_validate", "comet_spmv", "comet_spmm", "comet_ttv_symbolic", "comet_ttv",
-    "comet_ttm_symbolic", "comet_ttm", "comet_mttkrp",
+    "comet_ttm_symbolic", "comet_ttm", "comet_mttkrp", "comet_spmv_static",
 ]
 
 

@@ -16,6 +16,8 @@
 #include "common.cuh"
 #include "kernels.cuh"
 
+#include <mutex>
+
 namespace comet {
 
 struct SegDotArgs {
@@ -176,3 +178,77 @@ comet_status_t seg_dot(Context *ctx, const int32_t *seg_end, const int32_t *crd,
 }
 
 }  // namespace comet
+
+// ------------------------------------------------------------------------------------------------
+// comet_spmv_static: CSR SpMV for callers that must not allocate device memory.
+//
+// The regular entry point takes its carry slots (one double and one int32 per tile) from the handle's
+// scratch, which the handle obtains from an allocator. This variant keeps those slots in a fixed
+// array that is part of the library image, so the call reaches no allocator at all and needs no
+// handle. The price: a hard upper limit on the problem size and one array shared by every call.
+namespace {
+
+constexpr int kStaticThreads = 256;
+constexpr int kStaticIpt = 8;
+constexpr int64_t kStaticMaxTiles = 65536;                                   // tiles of 2048 merge items
+constexpr int64_t kStaticMaxItems = kStaticMaxTiles * kStaticThreads * kStaticIpt;   // rows + nnz <= 134,217,728
+constexpr size_t kStaticValBytes = (size_t)kStaticMaxTiles * sizeof(double);
+constexpr size_t kStaticBytes = kStaticValBytes + (size_t)kStaticMaxTiles * sizeof(int32_t);   // 768 KiB
+
+// Lives in every GPU that loads the library, from load until the process exits. In HOST code this
+// name is only a stand-in for the symbol: the device address comes from cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_spmv_static_scratch[kStaticBytes];
+
+constexpr int kStaticMaxDevices = 64;
+void *g_static_scratch_addr[kStaticMaxDevices];   // per device, filled by the first call on that device
+std::mutex g_static_mutex;
+
+// Device address of the static scratch on the CURRENT device (looked up once per device).
+comet_status_t static_scratch_address(void **out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) { cudaGetLastError(); return COMET_ERR_CUDA; }
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_scratch_addr[dev]) {
+    void *p = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(&p, g_spmv_static_scratch);
+    if (e != cudaSuccess || !p) { cudaGetLastError(); return COMET_ERR_CUDA; }
+    g_static_scratch_addr[dev] = p;
+  }
+  *out = g_static_scratch_addr[dev];
+  return COMET_OK;
+}
+
+}  // namespace
+
+extern "C" comet_status_t comet_spmv_static(const comet_sptensor_t *A, const void *x, void *y, void *stream) {
+  using namespace comet;
+  if (!A || !x || !y) return COMET_ERR_INVALID_ARG;
+  if (A->order != 2 || A->dtype != COMET_F64) return COMET_ERR_UNSUPPORTED_FORMAT;
+  if (A->attr[0] != COMET_D || A->attr[1] != COMET_CU) return COMET_ERR_UNSUPPORTED_FORMAT;
+  const int m0 = A->mode_order[0], m1 = A->mode_order[1];
+  if (!((m0 == 0 && m1 == 1) || (m0 == 1 && m1 == 0))) return COMET_ERR_INVALID_ARG;
+  const int64_t M = A->dims[m0], N = A->nnz;
+  if (M < 0 || N < 0 || !A->pos[1] || A->pos_len[1] != M + 1 || (N > 0 && (!A->crd[1] || !A->val)))
+    return COMET_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(x) & 7) || (reinterpret_cast<uintptr_t>(y) & 7)) return COMET_ERR_MISALIGNED;
+  if (M + N > kStaticMaxItems) return COMET_ERR_WORKSPACE;      // beyond the fixed scratch: use comet_spmv
+  if (M == 0) return COMET_OK;
+
+  void *scratch = nullptr;
+  const comet_status_t st = static_scratch_address(&scratch);
+  if (st != COMET_OK) return st;
+
+  SegDotArgs a{};
+  a.seg_end = A->pos[1] + 1; a.crd = A->crd[1]; a.val = (const double *)A->val;
+  a.M = M; a.N = N; a.x = (const double *)x; a.y = (double *)y; a.out_row = nullptr;
+  a.num_tiles = ceil_div(M + N, (int64_t)kStaticThreads * kStaticIpt);
+  a.carry_val = (double *)scratch;                               // every tile writes its slot before the
+  a.carry_seg = (int32_t *)((char *)scratch + kStaticValBytes);  // fix-up reads it: nothing to clear
+  cudaStream_t s = (cudaStream_t)stream;
+  seg_dot_kernel<kStaticThreads, kStaticIpt><<<(unsigned)a.num_tiles, kStaticThreads, 0, s>>>(a);
+  if (a.num_tiles > 1)
+    carry_fixup_kernel<<<(unsigned)ceil_div(a.num_tiles, 256), 256, 0, s>>>(a.carry_val, a.carry_seg, a.num_tiles, 1, 1,
+                                                                            a.y, 1, nullptr);
+  if (cudaGetLastError() != cudaSuccess) return COMET_ERR_CUDA;
+  return COMET_OK;
+}
