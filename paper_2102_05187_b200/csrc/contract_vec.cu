@@ -13,6 +13,13 @@
 #include "kernels.cuh"
 #include "walk.cuh"
 
+#ifndef COMET_PF_GATHER
+#define COMET_PF_GATHER 4      // row gathers in flight per worker (SpMM, TTM); measured best with 4 CTAs/SM
+#endif
+#ifndef COMET_MINB_GATHER
+#define COMET_MINB_GATHER 4    // CTAs per SM the register budget is held to (64 registers)
+#endif
+
 namespace comet {
 
 struct SegGatherArgs {
@@ -37,60 +44,81 @@ struct SegGatherArgs {
 // What the walker does with one leaf entry: close the segments that end in front of it, accumulate.
 template <int LPN, int CPL, int VEC, bool MAPPED>
 struct SegGatherPolicy {
-  using Entry = Entry16;
   using L = Lanes<LPN, CPL, VEC>;
-  static constexpr int kRows = 1;
-  struct Window { double r[1][CPL][VEC]; };
+  static constexpr int kPF = COMET_PF_GATHER;
+  static constexpr bool kAux = false;
+  static constexpr bool kFullUnroll = true;
+  struct Slot { double r[CPL][VEC]; };
 
   const SegGatherArgs &a;
   const L &ln;
+  const char *bcol;         // this lane's piece 0 of row 0 of B
+  int32_t ldb_bytes;
   double acc[CPL][VEC];
-  int64_t i;          // open segment
-  int32_t next_end;   // leaf position where it ends (-1: no segment left)
-  int32_t last_flush; // leaf position of the latest flush (entries at or after it are still in acc)
+  double *out;              // this lane's piece 0 of the open segment's output row (identity mapping)
+  const int32_t *endp;      // seg_end + open segment
+  int32_t segs_left;        // segments from the open one to the last
+  int32_t next_end;         // leaf position where the open segment ends (-1: no segment left)
+  int32_t base, rel_end;    // chunk base and next_end relative to it
+  int32_t last_flush;       // leaf position of the latest flush (entries at or after it are still in acc)
 
   __device__ __forceinline__ SegGatherPolicy(const SegGatherArgs &args, const L &lanes, int64_t i0, int32_t j0)
-      : a(args), ln(lanes), i(i0), last_flush(j0) {
+      : a(args), ln(lanes), base(j0), last_flush(j0) {
     ln.zero(acc);
-    next_end = (i < a.M) ? __ldg(a.seg_end + i) : -1;
+    bcol = reinterpret_cast<const char *>(a.B + ln.col0);
+    ldb_bytes = (int32_t)(a.ldb * 8);
+    out = a.C + i0 * a.ldc + ln.col0;
+    endp = a.seg_end + i0;
+    segs_left = (int32_t)(a.M - i0);
+    next_end = segs_left > 0 ? __ldg(endp) : -1;
+    rel_end = next_end - base;
   }
-  __device__ __forceinline__ Entry fetch(int32_t j) const { return Entry{ld_stream(a.val + j), ld_stream(a.crd + j), 0}; }
-  static __device__ __forceinline__ Entry idle() { return Entry{0.0, 0, 0}; }
-  __device__ __forceinline__ const double *row(const Entry &e, int) const { return a.B + (int64_t)e.a * a.ldb; }
+  __device__ __forceinline__ int64_t segment() const { return a.M - segs_left; }
+  __device__ __forceinline__ void fetch(int32_t j, Entry16 &e, int32_t &) const {
+    e.v = ld_stream(a.val + j);
+    e.a = ld_stream(a.crd + j);
+  }
+  __device__ __forceinline__ void prefetch(int32_t c, int32_t, Slot &s) const {
+    ln.gather(reinterpret_cast<const double *>(bcol + (int64_t)c * ldb_bytes), s.r);
+  }
+  __device__ __forceinline__ void begin_chunk(int32_t b) { base = b; rel_end = next_end - b; }
 
   // Stores the open segment (and, for a compressed root level, zero-fills the rows in front of it).
   __device__ __forceinline__ void flush(int32_t j) {
-    int64_t r = i;
     if (MAPPED) {
-      r = __ldg(a.out_row + i);
+      const int64_t i = segment();
+      const int64_t r = __ldg(a.out_row + i);
       const int64_t lo = (i > 0) ? (int64_t)__ldg(a.out_row + i - 1) + 1 : 0;
-      ln.zero_rows(a.C, a.ldc, lo, r);
-      if (i == a.M - 1) ln.zero_rows(a.C, a.ldc, r + 1, a.out_rows);
+      double *c0 = a.C + ln.col0;
+      ln.zero_rows(c0, a.ldc, lo, r);
+      if (i == a.M - 1) ln.zero_rows(c0, a.ldc, r + 1, a.out_rows);
+      ln.store_row(c0 + r * a.ldc, acc);
+    } else {
+      ln.store_row(out, acc);
+      out += a.ldc;
     }
-    ln.store_row(a.C + r * a.ldc, acc);
     ln.zero(acc);
-    ++i;
-    next_end = (i < a.M) ? __ldg(a.seg_end + i) : -1;
+    ++endp;
+    --segs_left;
+    next_end = segs_left > 0 ? __ldg(endp) : -1;
+    rel_end = next_end - base;
     last_flush = j;
   }
-  __device__ __forceinline__ void consume(int32_t j, const Entry &e, const double (&rows)[1][CPL][VEC]) {
-    while (j == next_end) flush(j);          // segments (possibly empty ones) that end in front of leaf j
-#pragma unroll
-    for (int t = 0; t < CPL; ++t)
-      if (ln.ok[t])
-#pragma unroll
-        for (int k = 0; k < VEC; ++k) acc[t][k] = fma(e.v, rows[0][t][k], acc[t][k]);
+  __device__ __forceinline__ void consume(int q, double v, int32_t, Slot &s) {
+    while (rel_end == q) flush(base + q);      // segments (possibly empty ones) that end in front of this leaf
+    ln.fma_rows(v, s.r, acc);
   }
 };
 
 template <int LPN, int CPL, int VEC, bool MAPPED>
-__global__ void __launch_bounds__(kBlockThreads) seg_gather_kernel(const SegGatherArgs a) {
+__global__ void __launch_bounds__(kBlockThreads, (CPL * VEC <= 2 ? COMET_MINB_GATHER : 2))
+seg_gather_kernel(const SegGatherArgs a) {
   using L = Lanes<LPN, CPL, VEC>;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int worker = threadIdx.x / LPN;
   const int64_t tile = (int64_t)blockIdx.x * L::kWorkers + worker;
   if (tile >= a.num_tiles) return;                       // whole groups leave together
-  Entry16 *ring = reinterpret_cast<Entry16 *>(smem_raw) + worker * 2 * L::kChunk;
+  const uint32_t smem = smem_u32(smem_raw) + worker * RingLayout<L, false>::kWorkerBytes;
   const L ln(a.R);
 
   const int64_t total = a.M + a.N;
@@ -101,12 +129,13 @@ __global__ void __launch_bounds__(kBlockThreads) seg_gather_kernel(const SegGath
   const int32_t j0 = (int32_t)(d0 - i0), j1 = (int32_t)(d1 - i1);
 
   SegGatherPolicy<LPN, CPL, VEC, MAPPED> p(a, ln, i0, j0);
-  walk_tile(ln, p, j0, j1, ring);
-  while (p.i < i1) p.flush(j1);                          // end markers that close the tile
+  walk_tile(ln, p, j0, j1, smem);
+  while (p.segment() < i1) p.flush(j1);                  // end markers that close the tile
 
-  const bool carry = p.i < a.M && j1 > p.last_flush;     // leaf entries of a segment that ends in a later tile
-  if (ln.g == 0) a.carry_seg[tile] = carry ? (int32_t)p.i : -1;
-  if (carry) ln.store_carry(a.carry_val + tile * a.carry_ld, p.acc);
+  const int64_t seg = p.segment();
+  const bool carry = seg < a.M && j1 > p.last_flush;     // leaf entries of a segment that ends in a later tile
+  if (ln.g == 0) a.carry_seg[tile] = carry ? (int32_t)seg : -1;
+  if (carry) ln.store_carry(a.carry_val + tile * a.carry_ld + ln.col0, p.acc);
 }
 
 // Adds the carries onto the stored rows. Tiles that stopped inside the same segment are consecutive;
@@ -158,7 +187,7 @@ int32_t choose_tile_items(int64_t total_items, int workers_per_block) {
 template <int LPN, int CPL, int VEC, bool MAPPED>
 static comet_status_t launch_mapped(Context *ctx, const SegGatherArgs &a, int64_t blocks, cudaStream_t stream) {
   using L = Lanes<LPN, CPL, VEC>;
-  constexpr size_t smem = (size_t)L::kWorkers * 2 * L::kChunk * sizeof(Entry16);
+  constexpr size_t smem = RingLayout<L, false>::kBlockBytes;
   auto kernel = seg_gather_kernel<LPN, CPL, VEC, MAPPED>;
   if (smem > 48 * 1024)
     COMET_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

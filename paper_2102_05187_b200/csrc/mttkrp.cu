@@ -12,6 +12,19 @@
 #include "kernels.cuh"
 #include "walk.cuh"
 
+#ifndef COMET_PF_COO
+#define COMET_PF_COO 2        // entries in flight per worker, two row gathers each
+#endif
+#ifndef COMET_PF_CSF
+#define COMET_PF_CSF 4
+#endif
+#ifndef COMET_MINB_COO
+#define COMET_MINB_COO 4
+#endif
+#ifndef COMET_MINB_CSF
+#define COMET_MINB_CSF 4
+#endif
+
 namespace comet {
 
 struct MttkrpArgs {
@@ -36,105 +49,140 @@ struct MttkrpArgs {
 // ------------------------------------------------------------------------------------------- COO
 template <int LPN, int CPL, int VEC>
 struct CooPolicy {
-  using Entry = Entry32;                 // value, root coordinate, level-1 coordinate, leaf coordinate
   using L = Lanes<LPN, CPL, VEC>;
-  static constexpr int kRows = 2;
-  struct Window { double r[2][CPL][VEC]; };
+  static constexpr int kPF = COMET_PF_COO;   // two rows per entry
+  static constexpr bool kAux = true;         // the root coordinate rides in the side ring
+  static constexpr bool kFullUnroll = true;
+  struct Slot { double r[2][CPL][VEC]; };
 
   const MttkrpArgs &a;
   const L &ln;
+  const char *pcol, *qcol;               // this lane's piece 0 of row 0 of P and of Q
+  int32_t ldp_bytes, ldq_bytes;
+  double *ocol;                          // this lane's piece 0 of row 0 of the output
   double acc[CPL][VEC];
   int32_t cur;                           // output row being accumulated
 
   __device__ __forceinline__ CooPolicy(const MttkrpArgs &args, const L &lanes, int32_t first_row)
-      : a(args), ln(lanes), cur(first_row) { ln.zero(acc); }
-  __device__ __forceinline__ Entry fetch(int32_t j) const {
-    return Entry{ld_stream(a.val + j), ld_stream(a.crd0 + j), ld_stream(a.crd1 + j), ld_stream(a.crd2 + j), 0, 0};
+      : a(args), ln(lanes), cur(first_row) {
+    ln.zero(acc);
+    pcol = reinterpret_cast<const char *>(a.P + ln.col0);
+    qcol = reinterpret_cast<const char *>(a.Q + ln.col0);
+    ldp_bytes = (int32_t)(a.ldp * 8);
+    ldq_bytes = (int32_t)(a.ldq * 8);
+    ocol = a.out + ln.col0;
   }
-  static __device__ __forceinline__ Entry idle() { return Entry{0.0, 0, 0, 0, 0, 0}; }
-  __device__ __forceinline__ const double *row(const Entry &e, int w) const {
-    return w == 0 ? a.P + (int64_t)e.b * a.ldp : a.Q + (int64_t)e.c * a.ldq;
+  __device__ __forceinline__ void fetch(int32_t j, Entry16 &e, int32_t &aux) const {
+    e.v = ld_stream(a.val + j);
+    e.a = ld_stream(a.crd1 + j);
+    e.b = ld_stream(a.crd2 + j);
+    aux = ld_stream(a.crd0 + j);
   }
+  __device__ __forceinline__ void prefetch(int32_t cj, int32_t ck, Slot &s) const {
+    ln.gather(reinterpret_cast<const double *>(pcol + (int64_t)cj * ldp_bytes), s.r[0]);
+    ln.gather(reinterpret_cast<const double *>(qcol + (int64_t)ck * ldq_bytes), s.r[1]);
+  }
+  __device__ __forceinline__ void begin_chunk(int32_t) {}
   // The run of `cur` ends here: store it, zero-fill the rows up to the next stored row.
   __device__ __forceinline__ void next_row(int32_t row) {
-    ln.store_row(a.out + (int64_t)cur * a.ldo, acc);
-    ln.zero_rows(a.out, a.ldo, (int64_t)cur + 1, row);
+    ln.store_row(ocol + (int64_t)cur * a.ldo, acc);
+    ln.zero_rows(ocol, a.ldo, (int64_t)cur + 1, row);
     ln.zero(acc);
     cur = row;
   }
-  __device__ __forceinline__ void consume(int32_t, const Entry &e, const double (&rows)[2][CPL][VEC]) {
-    if (e.a != cur) next_row(e.a);
+  __device__ __forceinline__ void consume(int, double v, int32_t row, Slot &s) {
+    if (row != cur) next_row(row);
 #pragma unroll
     for (int t = 0; t < CPL; ++t)
       if (ln.ok[t])
 #pragma unroll
-        for (int k = 0; k < VEC; ++k) acc[t][k] = fma(e.v * rows[0][t][k], rows[1][t][k], acc[t][k]);
+        for (int k = 0; k < VEC; ++k) acc[t][k] = fma(v * s.r[0][t][k], s.r[1][t][k], acc[t][k]);
   }
 };
 
 template <int LPN, int CPL, int VEC>
-__global__ void __launch_bounds__(kBlockThreads) mttkrp_coo_kernel(const MttkrpArgs a) {
+__global__ void __launch_bounds__(kBlockThreads, (CPL * VEC <= 2 ? COMET_MINB_COO : 1)) mttkrp_coo_kernel(const MttkrpArgs a) {
   using L = Lanes<LPN, CPL, VEC>;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int worker = threadIdx.x / LPN;
   const int64_t tile = (int64_t)blockIdx.x * L::kWorkers + worker;
   if (tile >= a.num_tiles) return;
-  Entry32 *ring = reinterpret_cast<Entry32 *>(smem_raw) + worker * 2 * L::kChunk;
+  using P = CooPolicy<LPN, CPL, VEC>;
+  const uint32_t smem = smem_u32(smem_raw) + worker * RingLayout<L, true>::kWorkerBytes;
   const L ln(a.R);
 
   const int64_t j0 = tile * a.tile_items;
   const int64_t j1 = (j0 + a.tile_items < a.N) ? j0 + a.tile_items : a.N;
   const int32_t first = __ldg(a.crd0 + j0);
+  P p(a, ln, first);
   {
     const int64_t prev = j0 > 0 ? (int64_t)__ldg(a.crd0 + j0 - 1) : -1;
-    if (prev != first) ln.zero_rows(a.out, a.ldo, prev + 1, first);   // the gap in front of a row is filled where it starts
+    if (prev != first) ln.zero_rows(p.ocol, a.ldo, prev + 1, first);   // the gap in front of a row is filled where it starts
   }
-  CooPolicy<LPN, CPL, VEC> p(a, ln, first);
-  walk_tile(ln, p, (int32_t)j0, (int32_t)j1, ring);
+  walk_tile(ln, p, (int32_t)j0, (int32_t)j1, smem);
 
   const int64_t nxt = j1 < a.N ? (int64_t)__ldg(a.crd0 + j1) : -1;
   if (nxt == p.cur) {                                    // the row continues in the next tile
     if (ln.g == 0) a.carry_seg[tile] = p.cur;
-    ln.store_carry(a.carry_val + tile * a.carry_ld, p.acc);
+    ln.store_carry(a.carry_val + tile * a.carry_ld + ln.col0, p.acc);
   } else {
     if (ln.g == 0) a.carry_seg[tile] = -1;
-    ln.store_row(a.out + (int64_t)p.cur * a.ldo, p.acc);
-    if (j1 == a.N) ln.zero_rows(a.out, a.ldo, (int64_t)p.cur + 1, a.rows);
+    ln.store_row(p.ocol + (int64_t)p.cur * a.ldo, p.acc);
+    if (j1 == a.N) ln.zero_rows(p.ocol, a.ldo, (int64_t)p.cur + 1, a.rows);
   }
 }
 
 // ------------------------------------------------------------------------------------------- CSF
 template <int LPN, int CPL, int VEC>
 struct CsfPolicy {
-  using Entry = Entry16;                 // value, leaf coordinate
   using L = Lanes<LPN, CPL, VEC>;
-  static constexpr int kRows = 1;
-  struct Window { double r[1][CPL][VEC]; };
+  static constexpr int kPF = COMET_PF_CSF;
+  static constexpr bool kAux = false;
+  static constexpr bool kFullUnroll = false;   // the fiber/slice epilogue is long: keep the body small
+  struct Slot { double r[CPL][VEC]; };
 
   const MttkrpArgs &a;
   const L &ln;
+  const char *pcol, *qcol;
+  int32_t ldp_bytes, ldq_bytes;
+  double *ocol;
   double tac[CPL][VEC], aac[CPL][VEC];   // open fiber sum, open slice sum
+  double prow[CPL][VEC];                 // P row of the open fiber, fetched when the fiber opened
   int64_t f, s;                          // open fiber, open slice
   int32_t next_end;                      // leaf position where the open fiber ends
+  int32_t base, rel_end;
   int64_t slice_end;                     // fiber index where the open slice ends
   int32_t last_fold;                     // leaf position of the latest fold (entries at or after it are in tac)
   bool a_dirty;
 
   __device__ __forceinline__ CsfPolicy(const MttkrpArgs &args, const L &lanes, int64_t f0, int64_t s0, int32_t j0)
-      : a(args), ln(lanes), f(f0), s(s0), last_fold(j0), a_dirty(false) {
+      : a(args), ln(lanes), f(f0), s(s0), base(j0), last_fold(j0), a_dirty(false) {
     ln.zero(tac);
     ln.zero(aac);
+    ln.zero(prow);
+    pcol = reinterpret_cast<const char *>(a.P + ln.col0);
+    qcol = reinterpret_cast<const char *>(a.Q + ln.col0);
+    ldp_bytes = (int32_t)(a.ldp * 8);
+    ldq_bytes = (int32_t)(a.ldq * 8);
+    ocol = a.out + ln.col0;
     next_end = f < a.F ? __ldg(a.seg_end2 + f) : -1;
+    rel_end = next_end - base;
     slice_end = s < a.S ? (int64_t)__ldg(a.pos1 + s + 1) : -1;
+    open_fiber();
   }
-  __device__ __forceinline__ Entry fetch(int32_t j) const { return Entry{ld_stream(a.val + j), ld_stream(a.crd2 + j), 0}; }
-  static __device__ __forceinline__ Entry idle() { return Entry{0.0, 0, 0}; }
-  __device__ __forceinline__ const double *row(const Entry &e, int) const { return a.Q + (int64_t)e.a * a.ldq; }
+  __device__ __forceinline__ void open_fiber() {         // start fetching the P row the fiber will be folded with
+    if (f < a.F) ln.gather(reinterpret_cast<const double *>(pcol + (int64_t)__ldg(a.crd1 + f) * ldp_bytes), prow);
+  }
+  __device__ __forceinline__ void fetch(int32_t j, Entry16 &e, int32_t &) const {
+    e.v = ld_stream(a.val + j);
+    e.a = ld_stream(a.crd2 + j);
+  }
+  __device__ __forceinline__ void prefetch(int32_t ck, int32_t, Slot &sl) const {
+    ln.gather(reinterpret_cast<const double *>(qcol + (int64_t)ck * ldq_bytes), sl.r);
+  }
+  __device__ __forceinline__ void begin_chunk(int32_t b) { base = b; rel_end = next_end - b; }
 
   __device__ __forceinline__ void fold(int32_t j) {      // aac += tac * P[crd1[f], :]
-    const double *pr = a.P + (int64_t)__ldg(a.crd1 + f) * a.ldp;
-    double prow[CPL][VEC];
-    ln.gather(pr, prow);
 #pragma unroll
     for (int t = 0; t < CPL; ++t)
       if (ln.ok[t])
@@ -147,36 +195,35 @@ struct CsfPolicy {
     fold(j);
     ++f;
     next_end = f < a.F ? __ldg(a.seg_end2 + f) : -1;
+    rel_end = next_end - base;
+    open_fiber();
     if (f == slice_end) {                                // the slice is complete: this worker owns its row
       const int64_t row = __ldg(a.crd0 + s);
       const int64_t lo = s > 0 ? (int64_t)__ldg(a.crd0 + s - 1) + 1 : 0;
-      ln.zero_rows(a.out, a.ldo, lo, row);
-      ln.store_row(a.out + row * a.ldo, aac);
-      if (s == a.S - 1) ln.zero_rows(a.out, a.ldo, row + 1, a.rows);
+      ln.zero_rows(ocol, a.ldo, lo, row);
+      ln.store_row(ocol + row * a.ldo, aac);
+      if (s == a.S - 1) ln.zero_rows(ocol, a.ldo, row + 1, a.rows);
       ln.zero(aac);
       a_dirty = false;
       ++s;
       slice_end = s < a.S ? (int64_t)__ldg(a.pos1 + s + 1) : -1;
     }
   }
-  __device__ __forceinline__ void consume(int32_t j, const Entry &e, const double (&rows)[1][CPL][VEC]) {
-    while (j == next_end) end_fiber(j);
-#pragma unroll
-    for (int t = 0; t < CPL; ++t)
-      if (ln.ok[t])
-#pragma unroll
-        for (int k = 0; k < VEC; ++k) tac[t][k] = fma(e.v, rows[0][t][k], tac[t][k]);
+  __device__ __forceinline__ void consume(int q, double v, int32_t, Slot &sl) {
+    while (rel_end == q) end_fiber(base + q);
+    ln.fma_rows(v, sl.r, tac);
   }
 };
 
 template <int LPN, int CPL, int VEC>
-__global__ void __launch_bounds__(kBlockThreads) mttkrp_csf_kernel(const MttkrpArgs a) {
+__global__ void __launch_bounds__(kBlockThreads, (CPL * VEC <= 2 ? COMET_MINB_CSF : 2)) mttkrp_csf_kernel(const MttkrpArgs a) {
   using L = Lanes<LPN, CPL, VEC>;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int worker = threadIdx.x / LPN;
   const int64_t tile = (int64_t)blockIdx.x * L::kWorkers + worker;
   if (tile >= a.num_tiles) return;
-  Entry16 *ring = reinterpret_cast<Entry16 *>(smem_raw) + worker * 2 * L::kChunk;
+  using P = CsfPolicy<LPN, CPL, VEC>;
+  const uint32_t smem = smem_u32(smem_raw) + worker * RingLayout<L, false>::kWorkerBytes;
   const L ln(a.R);
 
   // tile = a span of the merge list of fiber-end markers and leaf positions
@@ -194,13 +241,13 @@ __global__ void __launch_bounds__(kBlockThreads) mttkrp_csf_kernel(const MttkrpA
     if ((int64_t)__ldg(a.pos1 + mid + 1) <= f0) lo = mid + 1; else hi = mid;
   }
 
-  CsfPolicy<LPN, CPL, VEC> p(a, ln, f0, lo, j0);
-  walk_tile(ln, p, j0, j1, ring);
+  P p(a, ln, f0, lo, j0);
+  walk_tile(ln, p, j0, j1, smem);
   while (p.f < f1) p.end_fiber(j1);
   if (j1 > p.last_fold) p.fold(j1);                      // an unfinished fiber contributes through distributivity
   const bool carry = p.a_dirty && p.s < a.S;
   if (ln.g == 0) a.carry_seg[tile] = carry ? (int32_t)p.s : -1;
-  if (carry) ln.store_carry(a.carry_val + tile * a.carry_ld, p.aac);
+  if (carry) ln.store_carry(a.carry_val + tile * a.carry_ld + ln.col0, p.aac);
 }
 
 // ------------------------------------------------------------------------------------------- host
@@ -221,7 +268,7 @@ static comet_status_t launch_mttkrp(Context *ctx, MttkrpArgs a, cudaStream_t str
   a.carry_seg = (int32_t *)(scratch + val_bytes);
   const unsigned blocks = (unsigned)ceil_div(a.num_tiles, WORKERS);
   using L = Lanes<LPN, CPL, VEC>;
-  constexpr size_t smem = (size_t)L::kWorkers * 2 * L::kChunk * (CSF ? sizeof(Entry16) : sizeof(Entry32));
+  constexpr size_t smem = CSF ? RingLayout<L, false>::kBlockBytes : RingLayout<L, true>::kBlockBytes;
   auto kernel = CSF ? mttkrp_csf_kernel<LPN, CPL, VEC> : mttkrp_coo_kernel<LPN, CPL, VEC>;
   if (smem > 48 * 1024)
     COMET_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

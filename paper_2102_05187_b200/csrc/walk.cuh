@@ -5,22 +5,28 @@
 // row by the group is one contiguous LPN*VEC*8-byte request and no value ever crosses lanes.
 //
 // A worker walks a tile of consecutive leaf entries [j0, j1):
-//   * the leaf arrays (coordinates, value) are read with coalesced group loads, kChunk entries at a
-//     time, one refill ahead of use, and parked in a per-worker shared-memory ring (2 x kChunk
-//     entries) from which every lane re-reads them with one broadcast LDS per entry;
-//   * the dense-operand rows of the next kPF entries are always in flight (a rolling register
-//     window), so the gather latency is hidden inside one worker, not only across warps;
+//   * the leaf arrays (value, coordinates) are read with coalesced group loads, kChunk entries at a
+//     time and one refill ahead of use, and parked in a per-worker shared-memory ring (2 x kChunk
+//     16-byte entries, plus an optional int32 side ring) from which every lane re-reads an entry with
+//     one broadcast 128-bit LDS;
+//   * the dense-operand rows of the next kPF entries are always in flight in a rolling REGISTER window
+//     (slot q % kPF). Gathered rows never touch shared memory: staging them there was measured and
+//     saturates the L1/shared-memory pipe (90 % on TTM) long before L2 does;
+//   * the chunk body is fully unrolled, so window slots, ring offsets and the position inside the
+//     chunk are compile-time constants;
 //   * what is done with an entry and its gathered rows (segment ends, accumulation, stores) is the
-//     policy's business: consume().
+//     policy's business.
 //
-// Policy interface (all members called by every lane of the group, group-uniform control flow):
-//   typename Entry                       16- or 32-byte POD staged per leaf entry
-//   static constexpr int kRows           dense rows gathered per entry (1 or 2)
-//   Entry fetch(int j) const             read leaf entry j from global memory
-//   static Entry idle()                  a harmless entry (row 0, value 0) for slots past the tile
-//   const double *row(const Entry &, int which) const   base pointer of the row to gather
-//   struct Window { double r[kRows][CPL][VEC]; }   the gathered rows of one entry
-//   void consume(int j, const Entry &, const double (&rows)[kRows][CPL][VEC])
+// Policy interface (called by every lane of the group; control flow is group-uniform):
+//   static constexpr int kPF            entries whose rows are in flight
+//   static constexpr bool kAux          whether a second int32 per entry is staged
+//   static constexpr bool kFullUnroll   unroll the whole chunk (cheap consume) or only kPF-wide steps
+//   struct Slot                         the gathered rows of one in-flight entry (nothing else: the value
+//                                       and the aux word are re-read from the ring when the entry is consumed)
+//   void fetch(int32_t j, Entry16 &e, int32_t &aux) const   read leaf entry j from global memory
+//   void prefetch(int32_t a, int32_t b, Slot &s) const      issue the row gathers of an entry (its two coordinates)
+//   void begin_chunk(int32_t base)      positions inside the chunk are relative to `base`
+//   void consume(int q, double v, int32_t aux, Slot &s)     entry at position base + q
 #pragma once
 
 #include "common.cuh"
@@ -28,14 +34,46 @@
 namespace comet {
 
 struct Entry16 { double v; int32_t a; int32_t b; };
-struct Entry32 { double v; int32_t a; int32_t b; int32_t c; int32_t pad0; int64_t pad1; };
-static_assert(sizeof(Entry16) == 16 && sizeof(Entry32) == 32, "staged entries are whole 16-byte words");
+
+// 32-bit shared-memory addressing through PTX: one LDS/STS each, no generic-pointer conversions.
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ Entry16 lds_entry(uint32_t addr) {
+  int x, y, z, w;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(x), "=r"(y), "=r"(z), "=r"(w) : "r"(addr));
+  Entry16 e;
+  e.v = __hiloint2double(y, x);
+  e.a = z;
+  e.b = w;
+  return e;
+}
+__device__ __forceinline__ double lds_f64(uint32_t addr) {
+  double v;
+  asm volatile("ld.shared.f64 %0, [%1];" : "=d"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void lds_coords(uint32_t entry_addr, int32_t &a, int32_t &b) {   // words 2, 3 of an entry
+  asm volatile("ld.shared.v2.b32 {%0, %1}, [%2+8];" : "=r"(a), "=r"(b) : "r"(entry_addr));
+}
+__device__ __forceinline__ void sts_entry(uint32_t addr, const Entry16 &e) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(__double2loint(e.v)),
+               "r"(__double2hiint(e.v)), "r"(e.a), "r"(e.b)
+               : "memory");
+}
+__device__ __forceinline__ int32_t lds_s32(uint32_t addr) {
+  int32_t v;
+  asm volatile("ld.shared.s32 %0, [%1];" : "=r"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void sts_s32(uint32_t addr, int32_t v) {
+  asm volatile("st.shared.s32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
 
 template <int VEC> struct Piece;
 template <> struct Piece<2> {
+  // volatile: the gathers keep their program order relative to the ring reads, so exactly the rolling
+  // window is in flight (the scheduler otherwise hoists loads of far-ahead entries and spills)
   static __device__ __forceinline__ void load(const double *p, double (&d)[2]) {
-    const double2 v = __ldg(reinterpret_cast<const double2 *>(p));
-    d[0] = v.x; d[1] = v.y;
+    asm volatile("ld.global.nc.v2.f64 {%0, %1}, [%2];" : "=d"(d[0]), "=d"(d[1]) : "l"(p));
   }
   static __device__ __forceinline__ void store_stream(double *p, const double (&d)[2]) {
     __stcs(reinterpret_cast<double2 *>(p), make_double2(d[0], d[1]));
@@ -45,32 +83,32 @@ template <> struct Piece<2> {
   }
 };
 template <> struct Piece<1> {
-  static __device__ __forceinline__ void load(const double *p, double (&d)[1]) { d[0] = __ldg(p); }
+  static __device__ __forceinline__ void load(const double *p, double (&d)[1]) {
+    asm volatile("ld.global.nc.f64 %0, [%1];" : "=d"(d[0]) : "l"(p));
+  }
   static __device__ __forceinline__ void store_stream(double *p, const double (&d)[1]) { __stcs(p, d[0]); }
   static __device__ __forceinline__ void store(double *p, const double (&d)[1]) { *p = d[0]; }
 };
 
-template <int LPN, int CPL, int VEC> struct Lanes {
-  static constexpr int kChunk = LPN >= 4 ? 32 : 8 * LPN;   // leaf entries per refill of the ring
+template <int LPN_, int CPL_, int VEC_> struct Lanes {
+  static constexpr int LPN = LPN_, CPL = CPL_, VEC = VEC_;
+  static constexpr int kChunk = LPN >= 16 ? 32 : (LPN >= 2 ? 16 : 8);   // leaf entries per refill of the ring
   static constexpr int kPer = kChunk / LPN;                // entries each lane loads per refill
-  static constexpr int kPF = 8;                            // gathers in flight per worker
   static constexpr int kWorkers = kBlockThreads / LPN;     // workers per CTA
-  static_assert(kChunk % kPF == 0, "the rolling window must divide the chunk");
+  static constexpr int kStride = LPN * VEC;                // columns between a lane's consecutive pieces
 
   int g;            // lane within the group
   unsigned mask;    // the group's lanes
-  int32_t col[CPL]; // first column of each owned piece
+  int32_t col0;     // first column of piece 0; piece t starts at col0 + t * kStride
   bool ok[CPL];     // piece inside the R columns of this launch (only the scalar path is ever ragged)
 
   __device__ __forceinline__ Lanes(int R) {
     g = threadIdx.x & (LPN - 1);
     const unsigned lane = threadIdx.x & 31;
     mask = LPN == 32 ? 0xffffffffu : (((1u << LPN) - 1u) << (lane & ~(LPN - 1)));
+    col0 = g * VEC;
 #pragma unroll
-    for (int t = 0; t < CPL; ++t) {
-      col[t] = (t * LPN + g) * VEC;
-      ok[t] = VEC == 2 ? true : col[t] < R;
-    }
+    for (int t = 0; t < CPL; ++t) ok[t] = VEC == 2 ? true : (col0 + t * kStride) < R;
   }
   __device__ __forceinline__ void sync() const { __syncwarp(mask); }
 
@@ -80,49 +118,112 @@ template <int LPN, int CPL, int VEC> struct Lanes {
 #pragma unroll
       for (int e = 0; e < VEC; ++e) acc[t][e] = 0.0;
   }
+  // `row` already points at this lane's piece 0 (row base + col0)
   __device__ __forceinline__ void gather(const double *row, double (&dst)[CPL][VEC]) const {
 #pragma unroll
     for (int t = 0; t < CPL; ++t)
-      if (ok[t]) Piece<VEC>::load(row + col[t], dst[t]);
+      if (ok[t]) Piece<VEC>::load(row + t * kStride, dst[t]);
   }
-  // out_row[0..R) = acc, streaming stores (written once, never re-read by this kernel)
   __device__ __forceinline__ void store_row(double *row, const double (&acc)[CPL][VEC]) const {
 #pragma unroll
     for (int t = 0; t < CPL; ++t)
-      if (ok[t]) Piece<VEC>::store_stream(row + col[t], acc[t]);
+      if (ok[t]) Piece<VEC>::store_stream(row + t * kStride, acc[t]);
   }
   __device__ __forceinline__ void store_carry(double *row, const double (&acc)[CPL][VEC]) const {
 #pragma unroll
     for (int t = 0; t < CPL; ++t)
-      if (ok[t]) Piece<VEC>::store(row + col[t], acc[t]);
+      if (ok[t]) Piece<VEC>::store(row + t * kStride, acc[t]);
   }
+  // rows lo .. hi-1 of a matrix whose lane-piece-0 pointer of row 0 is `base`
   __device__ __forceinline__ void zero_rows(double *base, int64_t ld, int64_t lo, int64_t hi) const {
     double z[CPL][VEC];
     zero(z);
     for (int64_t r = lo; r < hi; ++r) store_row(base + r * ld, z);
   }
+  __device__ __forceinline__ void fma_rows(double v, const double (&row)[CPL][VEC], double (&acc)[CPL][VEC]) const {
+#pragma unroll
+    for (int t = 0; t < CPL; ++t)
+      if (ok[t])
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) acc[t][e] = fma(v, row[t][e], acc[t][e]);
+  }
 };
 
-// Walks leaf entries [j0, j1) of one tile. `ring` is this worker's 2*kChunk-entry shared-memory ring.
-template <class L, class Policy>
-__device__ __forceinline__ void walk_tile(const L &ln, Policy &p, int32_t j0, int32_t j1,
-                                          typename Policy::Entry *ring) {
-  using Entry = typename Policy::Entry;
-  constexpr int kChunk = L::kChunk, kPer = L::kPer, kPF = L::kPF, kRows = Policy::kRows;
-  constexpr int LPN = kChunk / kPer;
-  if (j0 >= j1) return;
+// Shared memory of one worker: the entry ring, then (when the policy stages an aux word) the side ring.
+template <class L, bool AUX> struct RingLayout {
+  static constexpr int kEntryBytes = 2 * L::kChunk * 16;
+  static constexpr int kWorkerBytes = kEntryBytes + (AUX ? 2 * L::kChunk * 4 : 0);
+  static constexpr size_t kBlockBytes = (size_t)L::kWorkers * kWorkerBytes;
+};
 
-  Entry regs[kPer];
-  auto load_regs = [&](int32_t base) {
+// One chunk: positions 0..n-1 of the ring half at shared address `cur`; `nxt` is the other half.
+// kFullUnroll policies get the whole chunk unrolled (ring offsets and positions are immediates); the
+// others (heavy per-segment work, where code size matters more) get a loop of kPF-wide unrolled steps.
+template <class L, class Policy, bool TAIL>
+__device__ __forceinline__ void walk_chunk(Policy &p, typename Policy::Slot (&win)[Policy::kPF], uint32_t cur,
+                                           uint32_t nxt, uint32_t cur_aux, uint32_t nxt_aux, int n) {
+  constexpr int kChunk = L::kChunk, kPF = Policy::kPF;
+  if (Policy::kFullUnroll) {
+#pragma unroll
+    for (int q = 0; q < kChunk; ++q) {
+      if (TAIL && q >= n) break;
+      p.consume(q, lds_f64(cur + q * 16), Policy::kAux ? lds_s32(cur_aux + q * 4) : 0, win[q % kPF]);
+      // refill the slot with the entry kPF ahead (it may sit in the next chunk's half of the ring);
+      // the last, partial chunk only looks ahead inside itself
+      if (TAIL && q + kPF >= n) continue;
+      const bool in_cur = q + kPF < kChunk;
+      const int at = in_cur ? q + kPF : q + kPF - kChunk;
+      int32_t ca, cb;
+      lds_coords((in_cur ? cur : nxt) + at * 16, ca, cb);
+      p.prefetch(ca, cb, win[q % kPF]);
+    }
+  } else {
+    // the two halves are adjacent in shared memory: position q + kPF of `cur` wraps into `nxt`
+    const uint32_t lo = cur < nxt ? cur : nxt, lo_aux = cur_aux < nxt_aux ? cur_aux : nxt_aux;
+    const int off = cur < nxt ? 0 : kChunk;
+#pragma unroll 1
+    for (int q0 = 0; q0 < (TAIL ? n : kChunk); q0 += kPF) {
+#pragma unroll
+      for (int u = 0; u < kPF; ++u) {
+        const int q = q0 + u;
+        if (TAIL && q >= n) break;
+        const int r = off + q;
+        p.consume(q, lds_f64(lo + r * 16), Policy::kAux ? lds_s32(lo_aux + r * 4) : 0, win[u]);
+        if (TAIL && q + kPF >= n) continue;
+        int32_t ca, cb;
+        lds_coords(lo + ((r + kPF) & (2 * kChunk - 1)) * 16, ca, cb);
+        p.prefetch(ca, cb, win[u]);
+      }
+    }
+  }
+}
+
+// Walks leaf entries [j0, j1) of one tile. `smem` is the shared address of this worker's ring memory.
+template <class L, class Policy>
+__device__ __forceinline__ void walk_tile(const L &ln, Policy &p, int32_t j0, int32_t j1, uint32_t smem) {
+  constexpr int kChunk = L::kChunk, kPer = L::kPer, kPF = Policy::kPF, LPN = L::LPN;
+  static_assert(kChunk % kPF == 0 && kPF <= kChunk, "the rolling window must divide the chunk");
+  if (j0 >= j1) return;
+  const uint32_t s_aux = smem + RingLayout<L, Policy::kAux>::kEntryBytes;
+
+  Entry16 regs[kPer];
+  int32_t regs_aux[kPer];
+  auto load_regs = [&](int32_t base) {                   // base may run past the tile: idle entries
 #pragma unroll
     for (int t = 0; t < kPer; ++t) {
       const int32_t j = base + t * LPN + ln.g;
-      regs[t] = (j < j1) ? p.fetch(j) : Policy::idle();   // base may run past the tile: idle entries
+      regs[t] = Entry16{0.0, 0, 0};
+      regs_aux[t] = 0;
+      if (j < j1) p.fetch(j, regs[t], regs_aux[t]);
     }
   };
   auto store_regs = [&](int half) {
 #pragma unroll
-    for (int t = 0; t < kPer; ++t) ring[half * kChunk + t * LPN + ln.g] = regs[t];
+    for (int t = 0; t < kPer; ++t) {
+      const int at = half * kChunk + t * LPN + ln.g;
+      sts_entry(smem + at * 16, regs[t]);
+      if (Policy::kAux) sts_s32(s_aux + at * 4, regs_aux[t]);
+    }
   };
 
   load_regs(j0);
@@ -130,13 +231,12 @@ __device__ __forceinline__ void walk_tile(const L &ln, Policy &p, int32_t j0, in
   load_regs(j0 + kChunk);
   ln.sync();
 
-  Entry e[kPF];
-  typename Policy::Window win[kPF];
+  typename Policy::Slot win[kPF];
 #pragma unroll
   for (int u = 0; u < kPF; ++u) {
-    e[u] = ring[u];
-#pragma unroll
-    for (int w = 0; w < kRows; ++w) ln.gather(p.row(e[u], w), win[u].r[w]);
+    int32_t ca, cb;
+    lds_coords(smem + u * 16, ca, cb);
+    p.prefetch(ca, cb, win[u]);
   }
 
   int half = 0;
@@ -145,28 +245,12 @@ __device__ __forceinline__ void walk_tile(const L &ln, Policy &p, int32_t j0, in
     store_regs(half ^ 1);            // entries of the next chunk (idle entries past the tile)
     ln.sync();
     load_regs(base + 2 * kChunk);    // and the chunk after it goes into registers
-    const int n = (j1 - base < kChunk) ? (j1 - base) : kChunk;
-    if (n == kChunk) {
-      for (int q0 = 0; q0 < kChunk; q0 += kPF) {
-#pragma unroll
-        for (int u = 0; u < kPF; ++u) {
-          p.consume(base + q0 + u, e[u], win[u].r);
-          e[u] = ring[(half * kChunk + q0 + u + kPF) & (2 * kChunk - 1)];
-#pragma unroll
-          for (int w = 0; w < kRows; ++w) ln.gather(p.row(e[u], w), win[u].r[w]);
-        }
-      }
-    } else {
-      for (int q0 = 0; q0 < n; q0 += kPF) {
-#pragma unroll
-        for (int u = 0; u < kPF; ++u) {
-          if (q0 + u < n) p.consume(base + q0 + u, e[u], win[u].r);
-          e[u] = ring[(half * kChunk + q0 + u + kPF) & (2 * kChunk - 1)];
-#pragma unroll
-          for (int w = 0; w < kRows; ++w) ln.gather(p.row(e[u], w), win[u].r[w]);
-        }
-      }
-    }
+    const uint32_t cur = smem + half * (kChunk * 16), nxt = smem + (half ^ 1) * (kChunk * 16);
+    const uint32_t cur_aux = s_aux + half * (kChunk * 4), nxt_aux = s_aux + (half ^ 1) * (kChunk * 4);
+    p.begin_chunk(base);
+    const int n = j1 - base;
+    if (n >= kChunk) walk_chunk<L, Policy, false>(p, win, cur, nxt, cur_aux, nxt_aux, kChunk);
+    else walk_chunk<L, Policy, true>(p, win, cur, nxt, cur_aux, nxt_aux, n);
   }
 }
 
