@@ -105,10 +105,10 @@ extern "C" comet_status_t comet_spmv(comet_handle_t handle, const comet_sptensor
   const int64_t rows = A->dims[A->mode_order[0]];
   if (is_fmt(A, 2, COMET_D, COMET_CU))
     return seg_dot(ctx, A->pos[1] + 1, A->crd[1], (const double *)A->val, rows, A->nnz, (const double *)x,
-                   (double *)y, nullptr, rows, s);
+                   A->dims[A->mode_order[1]], (double *)y, nullptr, rows, s);
   if (is_fmt(A, 2, COMET_CU, COMET_CU))
     return seg_dot(ctx, A->pos[1] + 1, A->crd[1], (const double *)A->val, A->crd_len[0], A->nnz, (const double *)x,
-                   (double *)y, A->crd[0], rows, s);
+                   A->dims[A->mode_order[1]], (double *)y, A->crd[0], rows, s);
   return COMET_ERR_UNSUPPORTED_FORMAT;
 }
 
@@ -220,7 +220,7 @@ extern "C" comet_status_t comet_ttv(comet_handle_t handle, const comet_sptensor_
   if (misaligned8(v)) return COMET_ERR_MISALIGNED;
   Context *ctx = reinterpret_cast<Context *>(handle);
   return seg_dot(ctx, X->pos[2] + 1, X->crd[2], (const double *)X->val, X->crd_len[1], X->nnz, (const double *)v,
-                 (double *)Y->val, nullptr, X->crd_len[1], (cudaStream_t)stream);
+                 X->dims[mode], (double *)Y->val, nullptr, X->crd_len[1], (cudaStream_t)stream);
 }
 
 extern "C" comet_status_t comet_ttm_symbolic(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode,

@@ -69,4 +69,27 @@ __device__ __forceinline__ int64_t merge_path_segments(const int32_t *__restrict
   return lo;
 }
 
+
+// The same split found cooperatively by W consecutive lanes (W a power of two, `mask` = those lanes,
+// `k` = this lane's index among them): a W-ary search, log_W(M) rounds of one coalesced-ish probe per
+// lane instead of log_2(M) dependent loads by one thread. Every lane returns the result.
+template <int W>
+__device__ __forceinline__ int64_t merge_path_segments_coop(const int32_t *__restrict__ seg_end, int64_t M, int64_t N,
+                                                            int64_t diag, int k, unsigned mask) {
+  int64_t lo = diag > N ? diag - N : 0;
+  int64_t hi = diag < M ? diag : M;                 // markers below lo are inside, markers from hi on are not
+  const int shift = (threadIdx.x & 31) & ~(W - 1);
+  while (lo < hi) {
+    const int64_t stride = (hi - lo + W - 1) / W;
+    const int64_t s = lo + (int64_t)k * stride + stride - 1;     // last marker of this lane's sub-range
+    const bool inside = s < hi && (int64_t)__ldg(seg_end + s) + s < diag;
+    const unsigned votes = (__ballot_sync(mask, inside) >> shift) & (W == 32 ? 0xffffffffu : ((1u << W) - 1u));
+    const int full = __popc(votes);                // sub-ranges that lie wholly inside (the predicate is monotone)
+    lo += (int64_t)full * stride;
+    const int64_t cap = lo + stride - 1;           // the last marker of the first mixed sub-range is outside
+    if (cap < hi) hi = cap;
+  }
+  return lo;
+}
+
 }  // namespace comet

@@ -33,36 +33,21 @@ struct SegDotArgs {
   int32_t *carry_seg;
 };
 
-template <int THREADS, int IPT>
-__global__ void __launch_bounds__(THREADS) seg_dot_kernel(const SegDotArgs a) {
-  constexpr int TILE = THREADS * IPT;
+struct BlockBarrier {
+  __device__ __forceinline__ void operator()() const { __syncthreads(); }
+};
+struct NamedBarrier {          // a barrier over `count` threads of the CTA (a "virtual CTA")
+  int id, count;
+  __device__ __forceinline__ void operator()() const { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
+};
+
+// Steps 3 and 4 for a tile whose products and (tile-relative) segment ends are staged in shared memory.
+// `tid` is the thread's index among the THREADS threads that share the tile and the barrier.
+template <int THREADS, int IPT, class Bar>
+__device__ __forceinline__ void walk_staged_tile(const SegDotArgs &a, const int32_t *s_end, const double *s_prod,
+                                                 int32_t *s_wkey, double *s_wval, int tid, int rows, int nnz,
+                                                 int64_t i0, int64_t i1, int64_t tile, Bar bar) {
   constexpr int WARPS = THREADS / 32;
-  __shared__ int32_t s_end[TILE + 1];
-  __shared__ double s_prod[TILE];
-  __shared__ int64_t s_split[2];
-  __shared__ int32_t s_wkey[WARPS];
-  __shared__ double s_wval[WARPS];
-
-  const int tid = threadIdx.x;
-  const int64_t tile = blockIdx.x;
-  const int64_t total = a.M + a.N;
-  const int64_t d0 = tile * TILE;
-  const int64_t d1 = (d0 + TILE < total) ? d0 + TILE : total;
-  if (tid < 2) s_split[tid] = merge_path_segments(a.seg_end, a.M, a.N, tid ? d1 : d0);
-  __syncthreads();
-  const int64_t i0 = s_split[0], i1 = s_split[1];
-  const int64_t j0 = d0 - i0, j1 = d1 - i1;
-  const int rows = (int)(i1 - i0);       // segment-end markers inside the tile
-  const int nnz = (int)(j1 - j0);        // leaf entries inside the tile
-
-  for (int t = tid; t < rows; t += THREADS) s_end[t] = (int32_t)((int64_t)__ldg(a.seg_end + i0 + t) - j0);
-  for (int t = tid; t < nnz; t += THREADS) {
-    const int32_t c = ld_stream(a.crd + j0 + t);
-    const double v = ld_stream(a.val + j0 + t);
-    s_prod[t] = v * __ldg(a.x + c);
-  }
-  __syncthreads();
-
   // thread-level split of the tile's merge list
   const int items = rows + nnz;
   const int t0 = (tid * IPT < items) ? tid * IPT : items;
@@ -109,7 +94,7 @@ __global__ void __launch_bounds__(THREADS) seg_dot_kernel(const SegDotArgs a) {
     if (lane >= off && k2 == key) sum += v2;
   }
   if (lane == 31) { s_wkey[warp] = key; s_wval[warp] = sum; }
-  __syncthreads();
+  bar();
   if (warp == 0) {
     int wk = lane < WARPS ? s_wkey[lane] : 0x7fffffff;
     double wv = lane < WARPS ? s_wval[lane] : 0.0;
@@ -121,7 +106,7 @@ __global__ void __launch_bounds__(THREADS) seg_dot_kernel(const SegDotArgs a) {
     }
     if (lane < WARPS) s_wval[lane] = wv;
   }
-  __syncthreads();
+  bar();
   if (warp > 0 && s_wkey[warp - 1] == key) sum += s_wval[warp - 1];
   // what the threads before this one hold for the segment this thread started in
   int prev_key = __shfl_up_sync(0xffffffffu, key, 1);
@@ -139,6 +124,161 @@ __global__ void __launch_bounds__(THREADS) seg_dot_kernel(const SegDotArgs a) {
     // key == rows here: the segment the tile stops in
     a.carry_seg[tile] = (i1 < a.M) ? (int32_t)i1 : -1;
     a.carry_val[tile] = sum;
+  }
+}
+
+template <int THREADS, int IPT>
+__global__ void __launch_bounds__(THREADS) seg_dot_kernel(const SegDotArgs a) {
+  constexpr int TILE = THREADS * IPT;
+  constexpr int WARPS = THREADS / 32;
+  __shared__ int32_t s_end[TILE + 1];
+  __shared__ double s_prod[TILE];
+  __shared__ int64_t s_split[2];
+  __shared__ int32_t s_wkey[WARPS];
+  __shared__ double s_wval[WARPS];
+
+  const int tid = threadIdx.x;
+  const int64_t tile = blockIdx.x;
+  const int64_t total = a.M + a.N;
+  const int64_t d0 = tile * TILE;
+  const int64_t d1 = (d0 + TILE < total) ? d0 + TILE : total;
+  if (tid < 64) {          // warps 0 and 1 locate the two ends of the tile, 32 probes per round each
+    const int64_t split = merge_path_segments_coop<32>(a.seg_end, a.M, a.N, tid < 32 ? d0 : d1, tid & 31, 0xffffffffu);
+    if ((tid & 31) == 0) s_split[tid >> 5] = split;
+  }
+  __syncthreads();
+  const int64_t i0 = s_split[0], i1 = s_split[1];
+  const int64_t j0 = d0 - i0, j1 = d1 - i1;
+  const int rows = (int)(i1 - i0);       // segment-end markers inside the tile
+  const int nnz = (int)(j1 - j0);        // leaf entries inside the tile
+
+  // Load phase, fully unrolled (a tile holds at most IPT entries and IPT markers per thread): all of a
+  // thread's coordinate/value loads are issued before the first dependent vector gather, and all
+  // gathers before the first product, so a thread has up to 3*IPT loads in flight instead of one.
+  {
+    int32_t c[IPT], e[IPT];
+    double v[IPT];
+#pragma unroll
+    for (int k = 0; k < IPT; ++k) {
+      const int t = tid + k * THREADS;
+      c[k] = 0; v[k] = 0.0; e[k] = 0;
+      if (t < nnz) { c[k] = ld_stream(a.crd + j0 + t); v[k] = ld_stream(a.val + j0 + t); }
+      if (t < rows) e[k] = __ldg(a.seg_end + i0 + t);
+    }
+#pragma unroll
+    for (int k = 0; k < IPT; ++k) {
+      const int t = tid + k * THREADS;
+#ifdef EXP_NOGATHER
+      if (t < nnz) v[k] *= __ldg(a.x + (c[k] & 1));
+#else
+      if (t < nnz) v[k] *= __ldg(a.x + c[k]);
+#endif
+    }
+#pragma unroll
+    for (int k = 0; k < IPT; ++k) {
+      const int t = tid + k * THREADS;
+      if (t < nnz) s_prod[t] = v[k];
+      if (t < rows) s_end[t] = (int32_t)((int64_t)e[k] - j0);
+    }
+  }
+  __syncthreads();
+
+  walk_staged_tile<THREADS, IPT>(a, s_end, s_prod, s_wkey, s_wval, tid, rows, nnz, i0, i1, tile, BlockBarrier());
+}
+
+// ------------------------------------------------------------------------------------------------
+// The resident-vector variant: when the dense vector fits in shared memory beside the tile staging
+// (x up to ~21,000 doubles), the random 8-byte gathers x[crd] are served from shared memory instead of
+// L2, whose sector-request rate otherwise bounds the kernel (measured on TTV: 589 us with L2 gathers,
+// 188 us with the gather removed). One persistent CTA per SM holds x and runs VC "virtual CTAs" of
+// THREADS threads, each walking its own sequence of tiles with its own staging and named barrier.
+// A virtual CTA keeps the next tile's leaf loads in flight (registers) while it walks the current
+// one, and reads its tile boundaries from a table a small partition kernel wrote, two tiles ahead.
+
+// splits[b] = segment-end markers among the first b * tile_items merge items, one warp per boundary
+__global__ void tile_split_kernel(const int32_t *__restrict__ seg_end, int64_t M, int64_t N, int32_t tile_items,
+                                  int64_t num_tiles, int32_t *__restrict__ splits) {
+  const int64_t b = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (b > num_tiles) return;
+  const int64_t total = M + N;
+  const int64_t diag = b * tile_items < total ? b * tile_items : total;
+  const int64_t split = merge_path_segments_coop<32>(seg_end, M, N, diag, threadIdx.x & 31, 0xffffffffu);
+  if ((threadIdx.x & 31) == 0) splits[b] = (int32_t)split;
+}
+
+template <int THREADS, int IPT> struct ResidentLayout {
+  static constexpr int TILE = THREADS * IPT;
+  static constexpr int WARPS = THREADS / 32;
+  static constexpr int kProdBytes = TILE * 8;
+  static constexpr int kEndBytes = (TILE + 4) * 4;
+  static constexpr int kScanBytes = WARPS * 16;
+  static constexpr int kStageBytes = kProdBytes + kEndBytes + kScanBytes;    // multiple of 16
+};
+
+template <int VC, int THREADS, int IPT>
+__global__ void __launch_bounds__(VC *THREADS, 1)
+seg_dot_resident_kernel(const SegDotArgs a, const int32_t *__restrict__ splits, int64_t x_len, int32_t x_bytes_padded) {
+  using RL = ResidentLayout<THREADS, IPT>;
+  constexpr int TILE = RL::TILE;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  double *s_x = reinterpret_cast<double *>(smem_raw);
+  for (int64_t i = threadIdx.x; i < x_len; i += VC * THREADS) s_x[i] = __ldg(a.x + i);
+  __syncthreads();
+
+  const int vc = threadIdx.x / THREADS, tid = threadIdx.x % THREADS;
+  unsigned char *stage = smem_raw + x_bytes_padded + vc * RL::kStageBytes;
+  double *s_prod = reinterpret_cast<double *>(stage);
+  int32_t *s_end = reinterpret_cast<int32_t *>(stage + RL::kProdBytes);
+  double *s_wval = reinterpret_cast<double *>(stage + RL::kProdBytes + RL::kEndBytes);
+  int32_t *s_wkey = reinterpret_cast<int32_t *>(stage + RL::kProdBytes + RL::kEndBytes + RL::WARPS * 8);
+  const NamedBarrier bar{1 + vc, THREADS};
+
+  const int64_t total = a.M + a.N;
+  const int64_t stride = (int64_t)gridDim.x * VC;
+  int64_t t = (int64_t)blockIdx.x * VC + vc;
+
+  // registers of the tile in flight
+  int32_t c[IPT], e[IPT];
+  double v[IPT];
+  int64_t f_i0 = 0, f_i1 = 0, f_j0 = 0;
+  int f_rows = 0, f_nnz = 0;
+  // boundaries of the tile after it
+  int32_t n_i0 = 0, n_i1 = 0;
+
+  auto fetch = [&](int64_t tile, int32_t i0, int32_t i1) {     // issue the leaf loads of `tile`
+    const int64_t d0 = tile * TILE;
+    const int64_t d1 = (d0 + TILE < total) ? d0 + TILE : total;
+    f_i0 = i0; f_i1 = i1; f_j0 = d0 - i0;
+    f_rows = i1 - i0;
+    f_nnz = (int)((d1 - i1) - f_j0);
+#pragma unroll
+    for (int k = 0; k < IPT; ++k) {
+      const int tt = tid + k * THREADS;
+      c[k] = 0; v[k] = 0.0; e[k] = 0;
+      if (tt < f_nnz) { c[k] = ld_stream(a.crd + f_j0 + tt); v[k] = ld_stream(a.val + f_j0 + tt); }
+      if (tt < f_rows) e[k] = __ldg(a.seg_end + f_i0 + tt);
+    }
+  };
+
+  if (t < a.num_tiles) fetch(t, __ldg(splits + t), __ldg(splits + t + 1));
+  if (t + stride < a.num_tiles) { n_i0 = __ldg(splits + t + stride); n_i1 = __ldg(splits + t + stride + 1); }
+
+  for (; t < a.num_tiles; t += stride) {
+    // publish the fetched tile: products (vector element from shared memory) and tile-relative segment ends
+    const int rows = f_rows, nnz = f_nnz;
+    const int64_t i0 = f_i0, i1 = f_i1, j0 = f_j0;
+#pragma unroll
+    for (int k = 0; k < IPT; ++k) {
+      const int tt = tid + k * THREADS;
+      if (tt < nnz) s_prod[tt] = v[k] * s_x[c[k]];
+      if (tt < rows) s_end[tt] = (int32_t)((int64_t)e[k] - j0);
+    }
+    // the next tile's loads fly while this one is walked; its successor's boundaries follow
+    if (t + stride < a.num_tiles) fetch(t + stride, n_i0, n_i1);
+    if (t + 2 * stride < a.num_tiles) { n_i0 = __ldg(splits + t + 2 * stride); n_i1 = __ldg(splits + t + 2 * stride + 1); }
+    bar();
+    walk_staged_tile<THREADS, IPT>(a, s_end, s_prod, s_wkey, s_wval, tid, rows, nnz, i0, i1, t, bar);
+    bar();                                               // the staging area may be overwritten
   }
 }
 
@@ -162,9 +302,40 @@ static comet_status_t launch_dot(Context *ctx, SegDotArgs a, cudaStream_t stream
   return COMET_OK;
 }
 
+constexpr int kResVC = 4, kResThreads = 256, kResIpt = 5;
+constexpr size_t kMaxDynamicSmem = 232448;               // 227 KB opt-in limit per CTA on sm_100
+
+static comet_status_t launch_resident(Context *ctx, SegDotArgs a, int64_t x_len, cudaStream_t stream) {
+  using RL = ResidentLayout<kResThreads, kResIpt>;
+  const int64_t total = a.M + a.N;
+  a.num_tiles = ceil_div(total, (int64_t)RL::TILE);
+  const size_t val_bytes = align_up((size_t)a.num_tiles * sizeof(double), 256);
+  const size_t seg_bytes = align_up((size_t)a.num_tiles * sizeof(int32_t), 256);
+  const size_t split_bytes = align_up((size_t)(a.num_tiles + 1) * sizeof(int32_t), 256);
+  char *scratch = (char *)scratch_get(ctx, val_bytes + seg_bytes + split_bytes, stream);
+  if (!scratch) return COMET_ERR_ALLOC;
+  a.carry_val = (double *)scratch;
+  a.carry_seg = (int32_t *)(scratch + val_bytes);
+  int32_t *splits = (int32_t *)(scratch + val_bytes + seg_bytes);
+  tile_split_kernel<<<(unsigned)ceil_div((a.num_tiles + 1) * 32, 256), 256, 0, stream>>>(a.seg_end, a.M, a.N, RL::TILE,
+                                                                                       a.num_tiles, splits);
+  COMET_LAUNCH_CHECK(ctx);
+  const int32_t x_bytes = (int32_t)align_up((size_t)x_len * 8, 16);
+  const size_t smem = (size_t)x_bytes + (size_t)kResVC * RL::kStageBytes;
+  auto kernel = seg_dot_resident_kernel<kResVC, kResThreads, kResIpt>;
+  COMET_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  const int64_t ctas = ceil_div(a.num_tiles, kResVC) < kSmCount ? ceil_div(a.num_tiles, kResVC) : kSmCount;
+  kernel<<<(unsigned)ctas, kResVC * kResThreads, smem, stream>>>(a, splits, x_len, x_bytes);
+  COMET_LAUNCH_CHECK(ctx);
+  carry_fixup_kernel<<<(unsigned)ceil_div(a.num_tiles, 256), 256, 0, stream>>>(a.carry_val, a.carry_seg, a.num_tiles, 1,
+                                                                              1, a.y, 1, a.out_row);
+  COMET_LAUNCH_CHECK(ctx);
+  return COMET_OK;
+}
+
 comet_status_t seg_dot(Context *ctx, const int32_t *seg_end, const int32_t *crd, const double *val, int64_t M,
-                       int64_t N, const double *x, double *y, const int32_t *out_row, int64_t out_rows,
-                       cudaStream_t stream) {
+                       int64_t N, const double *x, int64_t x_len, double *y, const int32_t *out_row,
+                       int64_t out_rows, cudaStream_t stream) {
   if (out_row) {
     comet_status_t st = zero_rows(ctx, y, out_rows, 1, 1, stream);
     if (st != COMET_OK) return st;
@@ -172,9 +343,19 @@ comet_status_t seg_dot(Context *ctx, const int32_t *seg_end, const int32_t *crd,
   if (M == 0) return COMET_OK;
   SegDotArgs a{};
   a.seg_end = seg_end; a.crd = crd; a.val = val; a.M = M; a.N = N; a.x = x; a.y = y; a.out_row = out_row;
-  // Small problems: short tiles so that the grid still covers the 148 SMs.
-  if (M + N < (int64_t)kSmCount * 2048 * 2) return launch_dot<128, 4>(ctx, a, stream);
-  return launch_dot<256, 8>(ctx, a, stream);
+  // Large problems whose vector fits in shared memory beside the staging: persistent CTAs, x resident.
+  {
+    using RL = ResidentLayout<kResThreads, kResIpt>;
+    const size_t need = align_up((size_t)x_len * 8, 16) + (size_t)kResVC * RL::kStageBytes;
+    const bool forced = getenv("COMET_SEG_DOT_RESIDENT") != nullptr;     // tests: exercise this path on small inputs
+    if (need <= kMaxDynamicSmem && (forced || M + N >= (int64_t)kSmCount * kResVC * RL::TILE * 8))
+      return launch_resident(ctx, a, x_len, stream);
+  }
+  // Items per thread are odd so that the per-thread walks (stride IPT doubles across lanes) hit all
+  // shared-memory banks; an even stride of 8 serialises them 16 ways. Small problems get short tiles so
+  // that the grid still covers the 148 SMs.
+  if (M + N < (int64_t)kSmCount * 2048 * 2) return launch_dot<128, 5>(ctx, a, stream);
+  return launch_dot<256, 9>(ctx, a, stream);
 }
 
 }  // namespace comet

@@ -124,8 +124,8 @@ seg_gather_kernel(const SegGatherArgs a) {
   const int64_t total = a.M + a.N;
   const int64_t d0 = tile * a.tile_items;
   const int64_t d1 = (d0 + a.tile_items < total) ? d0 + a.tile_items : total;
-  const int64_t i0 = merge_path_segments(a.seg_end, a.M, a.N, d0);
-  const int64_t i1 = merge_path_segments(a.seg_end, a.M, a.N, d1);
+  const int64_t i0 = merge_path_segments_coop<LPN>(a.seg_end, a.M, a.N, d0, ln.g, ln.mask);
+  const int64_t i1 = merge_path_segments_coop<LPN>(a.seg_end, a.M, a.N, d1, ln.g, ln.mask);
   const int32_t j0 = (int32_t)(d0 - i0), j1 = (int32_t)(d1 - i1);
 
   SegGatherPolicy<LPN, CPL, VEC, MAPPED> p(a, ln, i0, j0);

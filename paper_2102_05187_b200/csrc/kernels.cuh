@@ -14,8 +14,8 @@ comet_status_t seg_gather(Context *ctx, const int32_t *seg_end, const int32_t *c
 
 // y[row(s)] = sum over leaf entries p of segment s of val[p] * x[crd[p]]                    (SpMV, TTV)
 comet_status_t seg_dot(Context *ctx, const int32_t *seg_end, const int32_t *crd, const double *val, int64_t M,
-                       int64_t N, const double *x, double *y, const int32_t *out_row, int64_t out_rows,
-                       cudaStream_t stream);
+                       int64_t N, const double *x, int64_t x_len, double *y, const int32_t *out_row,
+                       int64_t out_rows, cudaStream_t stream);
 
 // Sorted COO [CN,S,S]: out[crd0[p], :] += val[p] * P[crd1[p], :] * Q[crd2[p], :]; every row < rows written.
 comet_status_t mttkrp_coo(Context *ctx, const int32_t *crd0, const int32_t *crd1, const int32_t *crd2,

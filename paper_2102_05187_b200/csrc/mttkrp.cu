@@ -230,8 +230,8 @@ __global__ void __launch_bounds__(kBlockThreads, (CPL * VEC <= 2 ? COMET_MINB_CS
   const int64_t total = a.F + a.N;
   const int64_t d0 = tile * a.tile_items;
   const int64_t d1 = (d0 + a.tile_items < total) ? d0 + a.tile_items : total;
-  const int64_t f0 = merge_path_segments(a.seg_end2, a.F, a.N, d0);
-  const int64_t f1 = merge_path_segments(a.seg_end2, a.F, a.N, d1);
+  const int64_t f0 = merge_path_segments_coop<LPN>(a.seg_end2, a.F, a.N, d0, ln.g, ln.mask);
+  const int64_t f1 = merge_path_segments_coop<LPN>(a.seg_end2, a.F, a.N, d1, ln.g, ln.mask);
   const int32_t j0 = (int32_t)(d0 - f0), j1 = (int32_t)(d1 - f1);
 
   // slice that holds fiber f0: the number of slices that end at or before it (every slice is non-empty)

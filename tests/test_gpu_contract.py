@@ -34,6 +34,16 @@ def tile_items(request, monkeypatch):
     return request.param
 
 
+@pytest.fixture(params=["default", "resident"])
+def seg_dot_path(request, monkeypatch):
+    """SpMV/TTV kernel choice: the size-based default, and the persistent resident-vector kernel forced."""
+    if request.param == "resident":
+        monkeypatch.setenv("COMET_SEG_DOT_RESIDENT", "1")
+    else:
+        monkeypatch.delenv("COMET_SEG_DOT_RESIDENT", raising=False)
+    return request.param
+
+
 def test_worked_example():
     mc = ([0, 0, 2, 2, 2, 3], [1, 4, 0, 1, 5, 3])
     mv = [1.0, 2.0, 3.0, 4.0, 5.0, 6.0]
@@ -65,7 +75,7 @@ MATRIX_CASES = [((64, 48), 700, 1), ((300, 200), 5000, 2), ((1, 500), 300, 3), (
 
 @pytest.mark.parametrize("dims,nnz,seed", MATRIX_CASES)
 @pytest.mark.parametrize("attr", [(D, CU), (CU, CU)])
-def test_spmv(dims, nnz, seed, attr, tile_items):
+def test_spmv(dims, nnz, seed, attr, tile_items, seg_dot_path):
     coords, val = synth.random_coo(dims, nnz, seed)
     c, v = _np(coords), val.numpy()
     x = synth.random_dense((dims[1],), seed).numpy()
@@ -129,7 +139,7 @@ TENSOR_CASES = [((20, 18, 16), 900, 1), ((50, 40, 30), 6000, 2), ((1, 30, 30), 3
 
 @pytest.mark.parametrize("dims,nnz,seed", TENSOR_CASES)
 @pytest.mark.parametrize("mode", [0, 1, 2])
-def test_ttv_ttm(dims, nnz, seed, mode, tile_items):
+def test_ttv_ttm(dims, nnz, seed, mode, tile_items, seg_dot_path):
     coords, val = synth.random_coo(dims, nnz, seed)
     c, v = _np(coords), val.numpy()
     kept = [m for m in range(3) if m != mode]
@@ -200,7 +210,7 @@ def test_results_are_reproducible_run_to_run():
 
 
 @pytest.mark.parametrize("config", [1, 2, 3, 4, 5])
-def test_scaled_workloads(config):
+def test_scaled_workloads(config, seg_dot_path):
     """The five benchmark workloads at 1/64 scale (several tiles, ragged tails, skewed segments)."""
     case = synth.make(config, scale=1 / 64)
     c, v = _np(case.coords), case.val.numpy()
