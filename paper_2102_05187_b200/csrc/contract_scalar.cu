@@ -302,7 +302,12 @@ static comet_status_t launch_dot(Context *ctx, SegDotArgs a, cudaStream_t stream
   return COMET_OK;
 }
 
-constexpr int kResVC = 4, kResThreads = 256, kResIpt = 5;
+#ifndef COMET_RES_VC
+#define COMET_RES_VC 8          // virtual CTAs per persistent CTA (measured best: 8 x 128 threads x 5 items)
+#define COMET_RES_THREADS 128
+#define COMET_RES_IPT 5
+#endif
+constexpr int kResVC = COMET_RES_VC, kResThreads = COMET_RES_THREADS, kResIpt = COMET_RES_IPT;
 constexpr size_t kMaxDynamicSmem = 232448;               // 227 KB opt-in limit per CTA on sm_100
 
 static comet_status_t launch_resident(Context *ctx, SegDotArgs a, int64_t x_len, cudaStream_t stream) {
