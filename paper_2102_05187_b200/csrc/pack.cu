@@ -22,7 +22,7 @@
 namespace comet {
 
 constexpr int kSortThreads = 256;
-constexpr int kSortItems = 16;
+constexpr int kSortItems = 8;
 constexpr int kSortTile = kSortThreads * kSortItems;   // keys per CTA per pass
 constexpr int kSortWarps = kSortThreads / 32;
 
@@ -43,16 +43,22 @@ struct KeyLayout {
 struct CoordPtrs { const int32_t *p[COMET_MAX_ORDER]; };   // level order
 
 // ------------------------------------------------------------------------------------------------ keys
+// ORDER is a template parameter so that the per-level loops unroll and the by-value descriptor structs
+// are read with constant indices (a runtime index would push them into local memory).
+template <int ORDER>
 __global__ void make_keys_kernel(CoordPtrs c, KeyLayout k, int64_t n, uint64_t *__restrict__ keys,
                                  uint32_t *__restrict__ idx, int32_t *__restrict__ status) {
   const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (p >= n) return;
+  int32_t v[ORDER];
+#pragma unroll
+  for (int l = 0; l < ORDER; ++l) v[l] = __ldcs(c.p[l] + p);
   uint64_t key = 0;
   bool bad = false;
-  for (int l = 0; l < k.order; ++l) {
-    const int64_t v = c.p[l][p];
-    bad |= (v < 0) | (v >= k.dim[l]);
-    key |= (uint64_t)(v & ((1ll << k.bits[l]) - 1)) << k.shift[l];
+#pragma unroll
+  for (int l = 0; l < ORDER; ++l) {
+    bad |= (v[l] < 0) | ((int64_t)v[l] >= k.dim[l]);
+    key |= ((uint64_t)(uint32_t)v[l] & ((1ull << k.bits[l]) - 1)) << k.shift[l];
   }
   if (bad) atomicOr(status + kStatusRange, 1);
   keys[p] = key;
@@ -168,26 +174,34 @@ __global__ void __launch_bounds__(kSortThreads) radix_histogram_kernel(const uin
   table[(int64_t)threadIdx.x * tiles + blockIdx.x] = s_cnt[threadIdx.x];     // digit-major
 }
 
-__global__ void __launch_bounds__(kSortThreads) radix_scatter_kernel(
+__global__ void __launch_bounds__(kSortThreads, 4) radix_scatter_kernel(
     const uint64_t *__restrict__ kin, const uint32_t *__restrict__ pin, uint64_t *__restrict__ kout,
     uint32_t *__restrict__ pout, const uint32_t *__restrict__ table, int64_t n, int shift, int64_t tiles) {
-  __shared__ uint32_t s_cnt[kSortWarps][256];
+  __shared__ uint32_t s_cnt[kSortWarps][256];     // per-warp digit counts, then per-warp local offsets
+  __shared__ uint32_t s_start[256];               // where digit d starts inside the tile's sorted order
+  __shared__ uint32_t s_delta[256];               // global position of digit d's run minus s_start[d]
+  __shared__ uint64_t s_key[kSortTile];           // the tile in sorted order
+  __shared__ uint32_t s_pay[kSortTile];
+  __shared__ uint32_t s_warp[32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int w = 0; w < kSortWarps; ++w) s_cnt[w][tid] = 0;
-  __syncthreads();
 
   // Item r of lane l of warp w sits at tile_base + w*(32*ITEMS) + r*32 + l: memory order is (w, r, l).
-  const int64_t warp_base = (int64_t)blockIdx.x * kSortTile + (int64_t)warp * (32 * kSortItems);
+  const int64_t tile_base = (int64_t)blockIdx.x * kSortTile;
+  const int64_t warp_base = tile_base + (int64_t)warp * (32 * kSortItems);
   uint64_t key[kSortItems];
   uint32_t pay[kSortItems];
+#pragma unroll
+  for (int r = 0; r < kSortItems; ++r) {          // all loads first
+    const int64_t i = warp_base + r * 32 + lane;
+    key[r] = i < n ? __ldcs(kin + i) : ~0ull;     // slots past the end rank after every real key of the tile
+    pay[r] = i < n ? __ldcs(pin + i) : 0u;
+  }
+  __syncthreads();
   uint32_t rank[kSortItems];
   const unsigned lt = (1u << lane) - 1u;
 #pragma unroll
   for (int r = 0; r < kSortItems; ++r) {
-    const int64_t i = warp_base + r * 32 + lane;
-    const bool valid = i < n;
-    key[r] = valid ? kin[i] : ~0ull;          // slots past the end rank after every real key of the tile
-    pay[r] = valid ? pin[i] : 0u;
     const uint32_t d = (uint32_t)(key[r] >> shift) & 255u;
     const unsigned peers = __match_any_sync(0xffffffffu, d);
     const int leader = __ffs(peers) - 1;
@@ -202,24 +216,37 @@ __global__ void __launch_bounds__(kSortThreads) radix_scatter_kernel(
   }
   __syncthreads();
   {
-    // digit `tid`: where each warp's run of this digit starts in the output
-    uint32_t run = table[(int64_t)tid * tiles + blockIdx.x];
+    // digit `tid`: tile total, per-warp offsets inside the digit's run, start of the run inside the tile
+    uint32_t run = 0;
 #pragma unroll
     for (int w = 0; w < kSortWarps; ++w) {
       const uint32_t c = s_cnt[w][tid];
       s_cnt[w][tid] = run;
       run += c;
     }
+    const uint32_t start = block_exclusive_scan(run, s_warp, nullptr);
+    s_start[tid] = start;
+    s_delta[tid] = table[(int64_t)tid * tiles + blockIdx.x] - start;
   }
   __syncthreads();
 #pragma unroll
-  for (int r = 0; r < kSortItems; ++r) {
-    const int64_t i = warp_base + r * 32 + lane;
-    if (i < n) {
-      const uint32_t d = (uint32_t)(key[r] >> shift) & 255u;
-      const uint32_t dst = s_cnt[warp][d] + rank[r];
-      kout[dst] = key[r];
-      pout[dst] = pay[r];
+  for (int r = 0; r < kSortItems; ++r) {          // local sort: every item to its place in the tile's order
+    const uint32_t d = (uint32_t)(key[r] >> shift) & 255u;
+    const uint32_t at = s_start[d] + s_cnt[warp][d] + rank[r];
+    s_key[at] = key[r];
+    s_pay[at] = pay[r];
+  }
+  __syncthreads();
+  const int64_t left = n - tile_base;
+  const int valid = left < kSortTile ? (int)left : kSortTile;
+#pragma unroll
+  for (int r = 0; r < kSortItems; ++r) {          // coalesced: consecutive threads write a digit's run contiguously
+    const int at = r * kSortThreads + tid;
+    if (at < valid) {
+      const uint64_t k2 = s_key[at];
+      const uint32_t dst = s_delta[(uint32_t)(k2 >> shift) & 255u] + (uint32_t)at;
+      kout[dst] = k2;
+      pout[dst] = s_pay[at];
     }
   }
 }
@@ -243,6 +270,9 @@ constexpr int kLevelItems = 8;
 constexpr int kLevelTile = kLevelThreads * kLevelItems;
 
 // Per tile: how many nodes each counted level opens; duplicates (equal adjacent keys) are flagged.
+// Counters are indexed by level (slots of uncounted levels stay unused); ORDER is a template parameter
+// so that every per-level loop unrolls and the plan is read with constant indices.
+template <int ORDER>
 __global__ void __launch_bounds__(kLevelThreads) level_count_kernel(const uint64_t *__restrict__ keys, int64_t n,
                                                                     LevelPlan plan, int64_t tiles,
                                                                     uint32_t *__restrict__ counts,
@@ -251,7 +281,9 @@ __global__ void __launch_bounds__(kLevelThreads) level_count_kernel(const uint64
   if (threadIdx.x < COMET_MAX_ORDER) s_cnt[threadIdx.x] = 0;
   __syncthreads();
   const int64_t base = (int64_t)blockIdx.x * kLevelTile;
-  uint32_t mine[COMET_MAX_ORDER] = {0, 0, 0, 0};
+  uint32_t mine[ORDER];
+#pragma unroll
+  for (int l = 0; l < ORDER; ++l) mine[l] = 0;
   bool dup = false;
 #pragma unroll
   for (int t = 0; t < kLevelItems; ++t) {
@@ -260,19 +292,23 @@ __global__ void __launch_bounds__(kLevelThreads) level_count_kernel(const uint64
       const uint64_t k = keys[p];
       const uint64_t kp = p > 0 ? keys[p - 1] : 0;
       dup |= (p > 0) & (k == kp);
-      for (int l = 0; l < plan.order; ++l)
-        if (plan.counted[l] >= 0 && is_head(k, kp, p == 0, plan.shift[l])) mine[plan.counted[l]] += 1;
+#pragma unroll
+      for (int l = 0; l < ORDER; ++l)
+        if (plan.counted[l] >= 0 && is_head(k, kp, p == 0, plan.shift[l])) mine[l] += 1;
     }
   }
-  for (int c = 0; c < plan.ncounted; ++c) {
-    uint32_t v = mine[c];
+#pragma unroll
+  for (int l = 0; l < ORDER; ++l) {
+    if (plan.counted[l] < 0) continue;
+    uint32_t v = mine[l];
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) v += __shfl_down_sync(0xffffffffu, v, off);
-    if ((threadIdx.x & 31) == 0 && v) atomicAdd(&s_cnt[c], v);
+    if ((threadIdx.x & 31) == 0 && v) atomicAdd(&s_cnt[l], v);
   }
   if (dup) atomicOr(status + kStatusDuplicate, 1);
   __syncthreads();
-  if (threadIdx.x < plan.ncounted) counts[(int64_t)threadIdx.x * tiles + blockIdx.x] = s_cnt[threadIdx.x];
+  if (threadIdx.x < ORDER && plan.counted[threadIdx.x] >= 0)
+    counts[(int64_t)threadIdx.x * tiles + blockIdx.x] = s_cnt[threadIdx.x];
 }
 
 struct LevelOut {
@@ -280,10 +316,11 @@ struct LevelOut {
   int32_t *crd[COMET_MAX_ORDER];
   double *val;
   int64_t dim0;                // extent of level 0 (for a dense root)
-  uint32_t nodes[COMET_MAX_ORDER];   // node count of every counted level
+  uint32_t nodes[COMET_MAX_ORDER];   // node count of every counted level (indexed by level)
 };
 
 // Per tile: ranks of the heads (tile-local scan + the tile's scanned offset), then crd / pos / val.
+template <int ORDER>
 __global__ void __launch_bounds__(kLevelThreads) level_emit_kernel(const uint64_t *__restrict__ keys,
                                                                    const uint32_t *__restrict__ perm,
                                                                    const double *__restrict__ val_in, int64_t n,
@@ -293,84 +330,97 @@ __global__ void __launch_bounds__(kLevelThreads) level_emit_kernel(const uint64_
   __shared__ uint32_t s_warp[32];
   const int64_t base = (int64_t)blockIdx.x * kLevelTile + (int64_t)threadIdx.x * kLevelItems;   // blocked: 8 consecutive
   uint64_t k[kLevelItems + 1];
+  uint32_t src[kLevelItems];
   k[0] = (base > 0 && base - 1 < n) ? keys[base - 1] : 0;
 #pragma unroll
-  for (int t = 0; t < kLevelItems; ++t) k[t + 1] = (base + t < n) ? keys[base + t] : 0;
+  for (int t = 0; t < kLevelItems; ++t) {
+    k[t + 1] = (base + t < n) ? keys[base + t] : 0;
+    src[t] = (base + t < n) ? perm[base + t] : 0;
+  }
+  double vals[kLevelItems];
+#pragma unroll
+  for (int t = 0; t < kLevelItems; ++t) vals[t] = (base + t < n) ? __ldg(val_in + src[t]) : 0.0;   // the random gather, all in flight
 
   // rank[l] = nodes of level l opened before this thread's first entry
-  uint32_t rank[COMET_MAX_ORDER];
-  for (int l = 0; l < plan.order; ++l) {
+  uint32_t rank[ORDER];
+#pragma unroll
+  for (int l = 0; l < ORDER; ++l) {
     rank[l] = 0;
     if (plan.counted[l] < 0) continue;
     uint32_t mine = 0;
 #pragma unroll
     for (int t = 0; t < kLevelItems; ++t)
       if (base + t < n && is_head(k[t + 1], k[t], base + t == 0, plan.shift[l])) mine += 1;
-    rank[l] = offsets[(int64_t)plan.counted[l] * tiles + blockIdx.x] + block_exclusive_scan(mine, s_warp, nullptr);
+    rank[l] = offsets[(int64_t)l * tiles + blockIdx.x] + block_exclusive_scan(mine, s_warp, nullptr);
   }
 
 #pragma unroll
   for (int t = 0; t < kLevelItems; ++t) {
     const int64_t p = base + t;
-    if (p >= n) break;
-    const uint64_t key = k[t + 1], kp = k[t];
-    const bool first = p == 0;
-    // position of this entry's node at each level (entry rank where the level is not counted)
-    uint32_t parent_pos = 0;
-    bool parent_head = first;      // does this entry open a new node at the parent level?
-    for (int l = 0; l < plan.order; ++l) {
-      const int32_t coord = (int32_t)((key >> plan.shift[l]) & ((1ull << plan.bits[l]) - 1));
-      const int a = plan.attr[l];
-      if (a == COMET_D) {
-        parent_pos = (uint32_t)coord;
-        parent_head = is_head(key, kp, first, plan.shift[l]);
-      } else if (a == COMET_CU) {
-        const bool head = is_head(key, kp, first, plan.shift[l]);
-        const bool leaf = plan.counted[l] < 0;               // leaf level: one node per entry
-        const uint32_t node = leaf ? (uint32_t)p : (head ? rank[l] : rank[l] - 1);
-        if (head) {
-          out.crd[l][node] = coord;
-          if (l == 0) {
-            // root: pos = [0, nodes], written by the host-side finisher
-          } else if (plan.attr[l - 1] == COMET_D) {
-            // dense parent: every parent coordinate after the previous node's and up to this one starts here
-            if (parent_head) {
-              const int64_t prev = first ? -1 : (int64_t)((kp >> plan.shift[l - 1]) & ((1ull << plan.bits[l - 1]) - 1));
-              for (int64_t r = prev + 1; r <= (int64_t)parent_pos; ++r) out.pos[l][r] = (int32_t)node;
+    if (p < n) {
+      const uint64_t key = k[t + 1], kp = k[t];
+      const bool first = p == 0;
+      uint32_t parent_pos = 0;       // position of this entry's node at the level above
+      bool parent_head = first;      // does this entry open a new node at the level above?
+#pragma unroll
+      for (int l = 0; l < ORDER; ++l) {
+        const int32_t coord = (int32_t)((key >> plan.shift[l]) & ((1ull << plan.bits[l]) - 1));
+        const int a = plan.attr[l];
+        if (a == COMET_D) {
+          parent_pos = (uint32_t)coord;
+          parent_head = is_head(key, kp, first, plan.shift[l]);
+        } else if (a == COMET_CU) {
+          const bool head = is_head(key, kp, first, plan.shift[l]);
+          const bool leaf = plan.counted[l] < 0;               // leaf level: one node per entry
+          const uint32_t node = leaf ? (uint32_t)p : (head ? rank[l] : rank[l] - 1);
+          if (head) {
+            out.crd[l][node] = coord;
+            if (l == 0) {
+              // root: pos = [0, nodes], written by the finisher
+            } else if (plan.attr[l > 0 ? l - 1 : 0] == COMET_D) {
+              // dense parent: every parent coordinate after the previous node's and up to this one starts here
+              if (parent_head) {
+                const int sh = plan.shift[l > 0 ? l - 1 : 0], bt = plan.bits[l > 0 ? l - 1 : 0];
+                const int64_t prev = first ? -1 : (int64_t)((kp >> sh) & ((1ull << bt) - 1));
+                for (int64_t r = prev + 1; r <= (int64_t)parent_pos; ++r) out.pos[l][r] = (int32_t)node;
+              }
+            } else if (parent_head) {
+              out.pos[l][parent_pos] = (int32_t)node;           // first child of parent node parent_pos
             }
-          } else if (parent_head) {
-            out.pos[l][parent_pos] = (int32_t)node;           // first child of parent node parent_pos
           }
+          parent_pos = node;
+          parent_head = head;
+          if (!leaf && head) rank[l] += 1;
+        } else {                                                // CN, S: one position per entry
+          out.crd[l][p] = coord;
+          parent_pos = (uint32_t)p;
+          parent_head = true;
         }
-        parent_pos = node;
-        parent_head = head;
-        if (!leaf && head) rank[l] += 1;
-      } else {                                                // CN, S: one position per entry
-        out.crd[l][p] = coord;
-        parent_pos = (uint32_t)p;
-        parent_head = true;
       }
+      out.val[p] = vals[t];
     }
-    out.val[p] = val_in[perm[p]];
   }
 }
 
 // Closes the pos arrays: the terminal entry of every compressed level (and the empty tail of a CSR pos).
+template <int ORDER>
 __global__ void level_finish_kernel(const uint64_t *__restrict__ keys, int64_t n, LevelPlan plan, LevelOut out) {
   const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   uint32_t parents = 1;
-  for (int l = 0; l < plan.order; ++l) {
+#pragma unroll
+  for (int l = 0; l < ORDER; ++l) {
     const int a = plan.attr[l];
-    const uint32_t nodes = plan.counted[l] >= 0 ? out.nodes[plan.counted[l]] : (uint32_t)n;
+    const uint32_t nodes = plan.counted[l] >= 0 ? out.nodes[l] : (uint32_t)n;
     if (a == COMET_D) {
       if (tid == 0) out.pos[l][0] = (int32_t)out.dim0;
       parents = (uint32_t)out.dim0;
     } else if (a == COMET_CU) {
       if (l == 0) {
         if (tid == 0) { out.pos[0][0] = 0; out.pos[0][1] = (int32_t)nodes; }
-      } else if (plan.attr[l - 1] == COMET_D) {
+      } else if (plan.attr[l > 0 ? l - 1 : 0] == COMET_D) {
         // rows after the last stored one (all rows when the tensor is empty) start at `nodes`
-        const int64_t last = n > 0 ? (int64_t)((keys[n - 1] >> plan.shift[l - 1]) & ((1ull << plan.bits[l - 1]) - 1)) : -1;
+        const int sh = plan.shift[l > 0 ? l - 1 : 0], bt = plan.bits[l > 0 ? l - 1 : 0];
+        const int64_t last = n > 0 ? (int64_t)((keys[n - 1] >> sh) & ((1ull << bt) - 1)) : -1;
         for (int64_t r = last + 1 + tid; r <= (int64_t)out.dim0; r += (int64_t)gridDim.x * blockDim.x)
           out.pos[l][r] = (int32_t)nodes;
       } else if (tid == 0) {
@@ -514,7 +564,9 @@ extern "C" comet_status_t comet_pack(comet_handle_t handle, int32_t order, const
   uint32_t *d_nodes = reinterpret_cast<uint32_t *>(ctx->d_status) + 8;   // node counts live beside the status words
 
   if (n > 0) {
-    make_keys_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(coords, key, n, keys_a, perm_a, ctx->d_status);
+    if (order == 2) make_keys_kernel<2><<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(coords, key, n, keys_a, perm_a, ctx->d_status);
+    else if (order == 3) make_keys_kernel<3><<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(coords, key, n, keys_a, perm_a, ctx->d_status);
+    else make_keys_kernel<4><<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(coords, key, n, keys_a, perm_a, ctx->d_status);
     COMET_LAUNCH_CHECK(ctx);
     for (int shift = 0; shift < total_bits; shift += 8) {
       radix_histogram_kernel<<<(unsigned)sort_tiles, kSortThreads, 0, s>>>(keys_a, n, shift, sort_tiles, table);
@@ -528,12 +580,14 @@ extern "C" comet_status_t comet_pack(comet_handle_t handle, int32_t order, const
       uint32_t *tp = perm_a; perm_a = perm_b; perm_b = tp;
     }
     // node counts of the counted levels: per-tile counts -> scanned offsets (kept in `table`) + totals
-    level_count_kernel<<<(unsigned)level_tiles, kLevelThreads, 0, s>>>(keys_a, n, plan, level_tiles, table,
-                                                                       ctx->d_status);
+    if (order == 2) level_count_kernel<2><<<(unsigned)level_tiles, kLevelThreads, 0, s>>>(keys_a, n, plan, level_tiles, table, ctx->d_status);
+    else if (order == 3) level_count_kernel<3><<<(unsigned)level_tiles, kLevelThreads, 0, s>>>(keys_a, n, plan, level_tiles, table, ctx->d_status);
+    else level_count_kernel<4><<<(unsigned)level_tiles, kLevelThreads, 0, s>>>(keys_a, n, plan, level_tiles, table, ctx->d_status);
     COMET_LAUNCH_CHECK(ctx);
-    for (int c = 0; c < plan.ncounted; ++c) {
-      comet_status_t st = exclusive_scan(ctx, table + (int64_t)c * level_tiles, table + (int64_t)c * level_tiles,
-                                         level_tiles, scan_tmp, d_nodes + c, s);
+    for (int l = 0; l < order; ++l) {
+      if (plan.counted[l] < 0) continue;
+      comet_status_t st = exclusive_scan(ctx, table + (int64_t)l * level_tiles, table + (int64_t)l * level_tiles,
+                                         level_tiles, scan_tmp, d_nodes + l, s);
       if (st != COMET_OK) return st;
     }
   }
@@ -556,8 +610,8 @@ extern "C" comet_status_t comet_pack(comet_handle_t handle, int32_t order, const
     out->dims[l] = h_dims[l];
     out->mode_order[l] = h_mode_order[l];
     out->attr[l] = h_attr[l];
-    const int64_t nodes = plan.counted[l] >= 0 ? (int64_t)reinterpret_cast<uint32_t *>(ctx->h_pinned)[8 + plan.counted[l]] : n;
-    if (plan.counted[l] >= 0) lo.nodes[plan.counted[l]] = (uint32_t)nodes;
+    const int64_t nodes = plan.counted[l] >= 0 ? (int64_t)reinterpret_cast<uint32_t *>(ctx->h_pinned)[8 + l] : n;
+    if (plan.counted[l] >= 0) lo.nodes[l] = (uint32_t)nodes;
     int64_t pos_len = 0, crd_len = 0;
     if (h_attr[l] == COMET_D) { pos_len = 1; parents = key.dim[l]; }
     else if (h_attr[l] == COMET_CU) { pos_len = parents + 1; crd_len = nodes; parents = nodes; }
@@ -575,10 +629,15 @@ extern "C" comet_status_t comet_pack(comet_handle_t handle, int32_t order, const
   lo.dim0 = key.dim[0];
   if (!alloc_ok) { owner_release(ctx, owner, s); memset(out, 0, sizeof(*out)); return COMET_ERR_ALLOC; }
 
-  if (n > 0)
-    level_emit_kernel<<<(unsigned)level_tiles, kLevelThreads, 0, s>>>(keys_a, perm_a, (const double *)coo_val, n, plan,
-                                                                      level_tiles, table, lo);
-  level_finish_kernel<<<kSmCount, 256, 0, s>>>(keys_a, n, plan, lo);
+  const double *vin = (const double *)coo_val;
+  if (n > 0) {
+    if (order == 2) level_emit_kernel<2><<<(unsigned)level_tiles, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
+    else if (order == 3) level_emit_kernel<3><<<(unsigned)level_tiles, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
+    else level_emit_kernel<4><<<(unsigned)level_tiles, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
+  }
+  if (order == 2) level_finish_kernel<2><<<kSmCount, 256, 0, s>>>(keys_a, n, plan, lo);
+  else if (order == 3) level_finish_kernel<3><<<kSmCount, 256, 0, s>>>(keys_a, n, plan, lo);
+  else level_finish_kernel<4><<<kSmCount, 256, 0, s>>>(keys_a, n, plan, lo);
   ctx->launches += n > 0 ? 2 : 1;
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { owner_release(ctx, owner, s); memset(out, 0, sizeof(*out)); return cuda_fail(ctx, e); }
