@@ -152,7 +152,9 @@ template <int LPN_, int CPL_, int VEC_> struct Lanes {
 // Shared memory of one worker: the entry ring, then (when the policy stages an aux word) the side ring.
 template <class L, bool AUX> struct RingLayout {
   static constexpr int kEntryBytes = 2 * L::kChunk * 16;
-  static constexpr int kWorkerBytes = kEntryBytes + (AUX ? 2 * L::kChunk * 4 : 0);
+  // +16: the workers of one warp read the same ring position in the same instruction; without the skew
+  // their rings are a multiple of 128 bytes apart and every broadcast read is a 2- to 8-way bank conflict
+  static constexpr int kWorkerBytes = kEntryBytes + (AUX ? 2 * L::kChunk * 4 : 0) + 16;
   static constexpr size_t kBlockBytes = (size_t)L::kWorkers * kWorkerBytes;
 };
 
