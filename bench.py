@@ -134,6 +134,20 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(value, dist, device):
+    """The job-wide time of a measurement: the slowest rank's (identity when not distributed)."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(step_bytes, ms_per_step, world):
+    """Whole-job throughput in GB/s of `world` independent replicas that each move step_bytes per step."""
+    return world * step_bytes / ms_per_step / 1e6
+
+
 def cuda_time(fn, reps, warm):
     """Median and min device time (ms) of fn over `reps` runs after `warm` untimed ones (CUDA events on the
     current stream)."""
@@ -326,11 +340,9 @@ def run_ours(args):
     launches = handle.kernel_launches() - launches0
     clocks = sampler.stop()
     total_ms = t_start.elapsed_time(t_end)
+    total_ms = max_over_ranks(total_ms, dist, "cuda")
     if dist:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
         dist.barrier()
-        total_ms = float(t.item())
     ms_per_step = total_ms / args.steps
 
     A = step()
@@ -338,7 +350,7 @@ def run_ours(args):
     spmm_bytes, spmm_flops = model("spmm", "csr", case, A)
     pack_bytes = bytes_pack(n, 2, index_bytes(A))
     step_bytes = pack_bytes + spmm_bytes
-    value = world * step_bytes / ms_per_step / 1e6
+    value = aggregate_value(step_bytes, ms_per_step, world)
 
     # end to end through the host-buffer call: pinned COO + B in, C out, every step
     h_coords = [c.cpu().pin_memory() for c in coords]
@@ -356,10 +368,7 @@ def run_ours(args):
     e1.record()
     torch.cuda.synchronize()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    if dist:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, dist, "cuda")
     h2d = n * 16 + B.numel() * 8
     d2h = C.numel() * 8
     A.free()
@@ -387,7 +396,7 @@ def run_ours(args):
         "pack_ms_median": round(statistics.median(pack_ms), 4), "spmm_ms_median": round(spmm_med, 4),
         "spmm_GBps": round(spmm_bytes / spmm_med / 1e6, 1), "spmm_GFLOPs": round(spmm_flops / spmm_med / 1e6, 1),
         "clocks": clocks,
-        "e2e": {"value": round(world * step_bytes / e2e_ms / 1e6, 2), "unit": "GB/s", "ms_per_step": round(e2e_ms, 3),
+        "e2e": {"value": round(aggregate_value(step_bytes, e2e_ms, world), 2), "unit": "GB/s", "ms_per_step": round(e2e_ms, 3),
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(launches),
         "roofline": roofline,

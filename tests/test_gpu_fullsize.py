@@ -1,0 +1,166 @@
+"""Full-size checks, in the launch configuration bench.py times: every workload at scale 1.
+
+Packing: the packed arrays are expanded back to coordinate lists (Table 1's loops, vectorised) and must
+equal the lexicographically sorted input bit for bit; pos arrays must be monotone and end at the next
+level's length. Contractions: a seeded sample of output rows / fibers is recomputed one by one by the
+CPU oracle over the raw COO entries and compared with the normalised fp64 tolerance.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+from oracle import D, CU, CN, S
+
+pytestmark = pytest.mark.gpu
+
+comet = pytest.importorskip("paper_2102_05187_b200")
+from gpu_util import FP64_TOL, assert_close  # noqa: E402
+
+SAMPLES = 48
+
+
+@pytest.fixture(autouse=True)
+def _need_gpu(cuda_device):
+    yield
+
+
+def _expand(pos, n_children):
+    """parent index of every child position from a pos array (the CU loop of Table 1, vectorised)."""
+    counts = (pos[1:] - pos[:-1]).long()
+    assert int(counts.min()) >= 0 and int(pos[0]) == 0 and int(pos[-1]) == n_children
+    return torch.repeat_interleave(torch.arange(counts.numel(), device=pos.device), counts)
+
+
+def check_packed_against_sorted_input(case, T, mode_order, attr):
+    """Rebuild the coordinate list from the packed levels and compare with the sorted input."""
+    n = case.nnz
+    key = torch.zeros(n, dtype=torch.int64, device="cuda")
+    for m in mode_order:
+        key = key * case.dims[m] + case.coords[m].long()
+    order = torch.sort(key, stable=True).indices
+    want = [case.coords[m][order] for m in mode_order]
+    assert torch.equal(T.val, case.val[order]), "values are not the input values in sorted order"
+    # walk from the leaf upwards: position of each leaf entry at each level
+    levels = len(mode_order)
+    positions = [None] * levels
+    positions[levels - 1] = torch.arange(n, device="cuda")
+    for l in range(levels - 1, 0, -1):
+        a = attr[l]
+        if a == CU:
+            up = _expand(T.pos(l), T.c.crd_len[l])           # parent position of every node of level l
+            positions[l - 1] = up[positions[l]]
+        else:                                                # S: same position as the level above
+            positions[l - 1] = positions[l]
+    for l in range(levels):
+        a = attr[l]
+        if a == D:
+            got = positions[l].to(torch.int32)               # under a dense root the position IS the coordinate
+            assert T.pos(l).tolist() == [case.dims[mode_order[l]]]
+        else:
+            crd = T.crd(l)
+            assert int(crd.min()) >= 0 and int(crd.max()) < case.dims[mode_order[l]]
+            got = crd[positions[l]]
+            if a == CN:
+                assert T.pos(l).tolist() == [0, n]
+            if a == CU and l == 0:
+                assert T.pos(0).tolist() == [0, T.c.crd_len[0]]
+        assert torch.equal(got, want[l]), f"level {l}: coordinates differ from the sorted input"
+    # CU coordinates strictly ascend inside each parent: follows from equality with the sorted distinct input
+    return order
+
+
+def sample_rows(n_rows, seed, always=()):
+    g = np.random.default_rng(seed)
+    rows = set(int(r) for r in g.integers(0, n_rows, SAMPLES))
+    rows.update(int(r) for r in always if 0 <= r < n_rows)
+    return np.array(sorted(rows), dtype=np.int64)
+
+
+def host(case):
+    return [c.cpu().numpy() for c in case.coords], case.val.cpu().numpy()
+
+
+def test_full_c1_spmv():
+    case = synth.make(1, device="cuda")
+    A = comet.pack(case.coords, case.val, case.dims, (0, 1), (D, CU))
+    check_packed_against_sorted_input(case, A, (0, 1), (D, CU))
+    y = comet.spmv(A, case.dense["x"])
+    c, v = host(case)
+    want, norm = oracle.spmv(c, v, case.dims, case.dense["x"].cpu().numpy())      # small enough for every row
+    assert_close(y, want, norm, what="C1 spmv")
+
+
+def test_full_c2_spmm():
+    case = synth.make(2, device="cuda")
+    A = comet.pack(case.coords, case.val, case.dims, (0, 1), (D, CU))
+    check_packed_against_sorted_input(case, A, (0, 1), (D, CU))
+    C = comet.spmm(A, case.dense["B"])
+    lengths = torch.bincount(case.coords[0].long(), minlength=case.dims[0])
+    heavy = torch.topk(lengths, 4).indices.tolist()                                # rows that span many tiles
+    rows = sample_rows(case.dims[0], 2, always=heavy + [0, case.dims[0] - 1])
+    c, v = host(case)
+    want, norm = oracle.spmm(c, v, case.dims, case.dense["B"].cpu().numpy(), rows=rows)
+    rel = assert_close(C[torch.from_numpy(rows).cuda()], want, norm, what="C2 spmm")
+    print(f"C2 worst normalised error {rel:.2e}")
+
+
+def test_full_c3_ttv():
+    case = synth.make(3, device="cuda")
+    X = comet.pack(case.coords, case.val, case.dims, (0, 1, 2), (CU, CU, CU))
+    check_packed_against_sorted_input(case, X, (0, 1, 2), (CU, CU, CU))
+    Y = comet.ttv(X, 2, case.dense["v"])
+    F = X.c.crd_len[1]
+    fib = sample_rows(F, 3, always=[0, F - 1])
+    # the (i, j) key of sampled fiber f: crd1[f] and the slice that holds it
+    slice_of = _expand(X.pos(1), F)
+    fi = X.crd(0)[slice_of[torch.from_numpy(fib).cuda()]].long()
+    fj = X.crd(1)[torch.from_numpy(fib).cuda()].long()
+    keys = (fi * case.dims[1] + fj).cpu().numpy()
+    assert np.all(np.diff(keys) > 0)
+    c, v = host(case)
+    _, want, norm = oracle.ttv(c, v, case.dims, 2, case.dense["v"].cpu().numpy(), keys=keys)
+    rel = assert_close(Y.val[torch.from_numpy(fib).cuda()], want, norm, what="C3 ttv")
+    print(f"C3 worst normalised error {rel:.2e}")
+    # output structure: CSR over (I, J) whose rows are the slices
+    pos = Y.pos(1)
+    assert pos.numel() == case.dims[0] + 1 and int(pos[-1]) == F and bool((pos[1:] >= pos[:-1]).all())
+    assert torch.equal(Y.crd(1), X.crd(1))
+
+
+def test_full_c4_ttm():
+    case = synth.make(4, device="cuda")
+    X = comet.pack(case.coords, case.val, case.dims, (0, 1, 2), (CU, CU, CU))
+    check_packed_against_sorted_input(case, X, (0, 1, 2), (CU, CU, CU))
+    Y = comet.ttm(X, 2, case.dense["U"])
+    F = X.c.crd_len[1]
+    fib = sample_rows(F, 4, always=[0, F - 1])
+    sel = torch.from_numpy(fib).cuda()
+    slice_of = _expand(X.pos(1), F)
+    keys = (X.crd(0)[slice_of[sel]].long() * case.dims[1] + X.crd(1)[sel].long()).cpu().numpy()
+    c, v = host(case)
+    _, want, norm = oracle.ttm(c, v, case.dims, 2, case.dense["U"].cpu().numpy(), keys=keys)
+    rel = assert_close(Y.val.reshape(F, case.R)[sel], want, norm, what="C4 ttm")
+    print(f"C4 worst normalised error {rel:.2e}")
+
+
+@pytest.mark.parametrize("attr", [(CN, S, S), (CU, CU, CU)])
+def test_full_c5_mttkrp(attr):
+    case = synth.make(5, device="cuda")
+    X = comet.pack(case.coords, case.val, case.dims, (0, 1, 2), attr)
+    check_packed_against_sorted_input(case, X, (0, 1, 2), attr)
+    Fd = [None, case.dense["B"], case.dense["C"]]
+    out = torch.full((case.dims[0], case.R), float("nan"), dtype=torch.float64, device="cuda")
+    comet.mttkrp(X, 0, Fd, out)
+    assert not bool(torch.isnan(out).any()), "an output row was not written"
+    counts = torch.bincount(case.coords[0].long(), minlength=case.dims[0])
+    heavy = torch.topk(counts, 4).indices.tolist()                                 # slices spanning thousands of tiles
+    empty = torch.nonzero(counts == 0)[:4, 0].tolist()
+    rows = sample_rows(case.dims[0], 5, always=heavy + empty + [0, case.dims[0] - 1])
+    del X
+    c, v = host(case)
+    want, norm = oracle.mttkrp(c, v, case.dims, 0, [None, Fd[1].cpu().numpy(), Fd[2].cpu().numpy()], rows=rows)
+    rel = assert_close(out[torch.from_numpy(rows).cuda()], want, norm, what=f"C5 mttkrp {attr}")
+    print(f"C5 {attr} worst normalised error {rel:.2e}")
+    assert bool((out[counts == 0] == 0).all())                                     # rows without entries are +0
