@@ -420,7 +420,7 @@ def run_ours(args):
 
 # DRAM bytes per launch of the SpMM gather kernel at full size, from the ncu capture summarised in
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum).
-TRAFFIC_SPMM_C2 = 9.55e9
+TRAFFIC_SPMM_C2 = 9.47e9
 
 
 # --------------------------------------------------------------------------------------------- reference arm
