@@ -16,6 +16,8 @@
 #include "common.cuh"
 #include "kernels.cuh"
 
+#include <string.h>
+
 #include <mutex>
 
 namespace comet {
@@ -282,6 +284,133 @@ seg_dot_resident_kernel(const SegDotArgs a, const int32_t *__restrict__ splits, 
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// The warp-stream variant: every warp owns a span of consecutive leaf entries and walks it 32 entries
+// per step with fully coalesced loads; nothing is staged in shared memory except (optionally) the dense
+// vector. Lanes accumulate private partial sums while no segment ends inside a step -- one DADD per 32
+// entries, which is where the long fibers of a power-law tensor spend their time -- and only a step in
+// which a segment ends pays for a segmented warp scan (shuffles) and the stores. The warp keeps the ends
+// of the next 32 segments in registers (one per lane) and finds the ends that fall into a step with one
+// REDUX.OR; a lane that owns a closing segment fetches that segment's sum from the lane holding its last
+// entry. Segments are closed by the span that holds their last entry; the open partial of a span goes to
+// a carry slot as in the other kernels (deterministic, no atomics).
+template <bool XSMEM>
+__global__ void __launch_bounds__(1024, 1)
+seg_dot_stream_kernel(const SegDotArgs a, int64_t x_len, int32_t span, unsigned long long *next_tile) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const double *s_x = reinterpret_cast<const double *>(smem_raw);
+  if (XSMEM) {
+    double *w = reinterpret_cast<double *>(smem_raw);
+    for (int64_t i = threadIdx.x; i < x_len; i += blockDim.x) w[i] = __ldg(a.x + i);
+    __syncthreads();
+  }
+  const unsigned full = 0xffffffffu;
+  const int lane = threadIdx.x & 31;
+  auto xval = [&](int32_t c) -> double { return XSMEM ? s_x[c] : __ldg(a.x + c); };
+  auto warp_sum = [&](double v) -> double {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(full, v, off);
+    return v;
+  };
+
+  // Spans are handed out dynamically (one atomic per span): spans full of short segments take several times
+  // longer than spans inside one long segment, and a static assignment leaves warps idle at the end.
+  while (true) {
+    int64_t tile = 0;
+    if (lane == 0) tile = atomicAdd(next_tile, 1ull);
+    tile = __shfl_sync(full, tile, 0);
+    if (tile >= a.num_tiles) break;
+    const int32_t w0 = (int32_t)(tile * span);
+    const int32_t w1 = (int64_t)w0 + span < a.N ? w0 + span : (int32_t)a.N;
+    const bool whole = w1 - w0 == span;                  // span is a multiple of 128: no bounds checks inside
+
+    // open segment: the first one whose end lies beyond w0 (segments ending at w0 closed in the previous span)
+    int64_t lo = 0, hi = a.M;
+    while (lo < hi) {
+      const int64_t stride = (hi - lo + 31) / 32;
+      const int64_t q = lo + (int64_t)lane * stride + stride - 1;
+      const bool inside = q < hi && __ldg(a.seg_end + q) <= w0;
+      const int fullr = __popc(__ballot_sync(full, inside));
+      lo += (int64_t)fullr * stride;
+      const int64_t cap = lo + stride - 1;
+      if (cap < hi) hi = cap;
+    }
+    int64_t s = lo;
+    if (tile == 0)                                       // leading empty segments (end == 0) belong to nobody else
+      for (int64_t q = lane; q < s; q += 32) a.y[a.out_row ? (int64_t)__ldg(a.out_row + q) : q] = 0.0;
+
+    int32_t ew = (s + lane < a.M) ? __ldg(a.seg_end + s + lane) : 0x7fffffff;   // ends of the next 32 segments
+    int32_t last_end = w0;                               // end of the most recently closed segment
+    double run = 0.0;                                    // this lane's share of the open segment's sum
+
+    for (int32_t j0 = w0; j0 < w1; j0 += 128) {          // four steps per round: their loads are issued together
+      int32_t c[4];
+      double v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int32_t jj = j0 + u * 32 + lane;
+        c[u] = 0; v[u] = 0.0;
+        if (whole || jj < w1) { c[u] = ld_stream(a.crd + jj); v[u] = ld_stream(a.val + jj); }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int32_t j = j0 + u * 32;
+        if (!whole && j >= w1) break;
+        const double p = (whole || j + lane < w1) ? v[u] * xval(c[u]) : 0.0;
+        const int32_t top = (whole || j + 32 < w1) ? j + 32 : w1;   // segments with an end in (j, top] close in this step
+        if (!__any_sync(full, ew <= top)) { run += p; continue; }
+
+        // every end that falls into this step, as a bit per position (more than the 32 cached ends may)
+        unsigned endbits = __reduce_or_sync(full, ew <= top ? 1u << (ew - j - 1) : 0u);
+        if (__all_sync(full, ew <= top)) {
+          for (int64_t more = s + 32;; more += 32) {
+            const int32_t e2 = (more + lane < a.M) ? __ldg(a.seg_end + more + lane) : 0x7fffffff;
+            endbits |= __reduce_or_sync(full, e2 <= top ? 1u << (e2 - j - 1) : 0u);
+            if (!__all_sync(full, e2 <= top)) break;
+          }
+        }
+        // inclusive segmented scan of p; a new sub-sum starts after every end position
+        const unsigned heads = (endbits << 1) | 1u;
+        const int dist = lane - (31 - __clz(heads & (0xffffffffu >> (31 - lane))));   // entries since the sub-sum started
+        double sc = p;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const double t = __shfl_up_sync(full, sc, off);
+          if (off <= dist) sc += t;
+        }
+        const int firstb = __ffs(endbits) - 1, lastb = 31 - __clz(endbits);
+        const double tot = warp_sum(run);                // what earlier steps hold for the segment closed first
+        run = lane > lastb ? p : 0.0;                    // entries behind the last end open the next segment
+
+        while (true) {                                   // emit: each lane owns the segment whose end it caches
+          const bool closing = ew <= top;
+          const unsigned cm = __ballot_sync(full, closing);
+          if (cm == 0) break;
+          const int src = closing ? ew - j - 1 : 0;
+          double val = __shfl_sync(full, sc, src);
+          int32_t prev = __shfl_up_sync(full, ew, 1);
+          if (lane == 0) prev = last_end;
+          if (closing) {
+            if (ew == prev) val = 0.0;                   // an empty segment: its end repeats its predecessor's
+            else if (src == firstb) val += tot;
+            const int64_t seg = s + lane;
+            a.y[a.out_row ? (int64_t)__ldg(a.out_row + seg) : seg] = val;
+          }
+          const int k = __popc(cm);                      // closing lanes are a prefix: ends are sorted
+          last_end = __shfl_sync(full, ew, k - 1);
+          s += k;
+          ew = (s + lane < a.M) ? __ldg(a.seg_end + s + lane) : 0x7fffffff;
+        }
+      }
+    }
+    const double open = warp_sum(run);
+    if (lane == 0) {
+      a.carry_seg[tile] = s < a.M ? (int32_t)s : -1;
+      a.carry_val[tile] = open;
+    }
+  }
+}
+
 template <int THREADS, int IPT>
 static comet_status_t launch_dot(Context *ctx, SegDotArgs a, cudaStream_t stream) {
   const int64_t total = a.M + a.N;
@@ -338,6 +467,39 @@ static comet_status_t launch_resident(Context *ctx, SegDotArgs a, int64_t x_len,
   return COMET_OK;
 }
 
+static comet_status_t launch_stream(Context *ctx, SegDotArgs a, int64_t x_len, cudaStream_t stream) {
+  const size_t x_bytes = align_up((size_t)x_len * 8, 16);
+  const bool xsmem = x_bytes <= kMaxDynamicSmem - 1024;
+  // spans: a multiple of 128 entries, several per warp of the 148 persistent CTAs so that the tail is short
+  const int64_t warps = (int64_t)kSmCount * 32;
+  int64_t span = ceil_div(ceil_div(a.N, warps * 10), 128) * 128;
+  if (span < 512) span = 512;
+  if (span > 2048) span = 2048;
+  if (const char *e = getenv("COMET_STREAM_SPAN")) { const int v = atoi(e); if (v >= 128 && v % 128 == 0) span = v; }
+  a.num_tiles = ceil_div(a.N, span);
+  const size_t val_bytes = align_up((size_t)a.num_tiles * sizeof(double), 256);
+  const size_t seg_bytes = align_up((size_t)a.num_tiles * sizeof(int32_t), 256);
+  char *scratch = (char *)scratch_get(ctx, val_bytes + seg_bytes + 256, stream);
+  if (!scratch) return COMET_ERR_ALLOC;
+  a.carry_val = (double *)scratch;
+  a.carry_seg = (int32_t *)(scratch + val_bytes);
+  unsigned long long *next_tile = (unsigned long long *)(scratch + val_bytes + seg_bytes);
+  COMET_CUDA_TRY(ctx, cudaMemsetAsync(next_tile, 0, sizeof(unsigned long long), stream));
+  const int64_t ctas = ceil_div(a.num_tiles, 32) < kSmCount ? ceil_div(a.num_tiles, 32) : kSmCount;
+  if (xsmem) {
+    auto kernel = seg_dot_stream_kernel<true>;
+    COMET_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)x_bytes));
+    kernel<<<(unsigned)ctas, 1024, x_bytes, stream>>>(a, x_len, (int32_t)span, next_tile);
+  } else {
+    seg_dot_stream_kernel<false><<<(unsigned)ctas, 1024, 0, stream>>>(a, x_len, (int32_t)span, next_tile);
+  }
+  COMET_LAUNCH_CHECK(ctx);
+  carry_fixup_kernel<<<(unsigned)ceil_div(a.num_tiles, 256), 256, 0, stream>>>(a.carry_val, a.carry_seg, a.num_tiles, 1,
+                                                                              1, a.y, 1, a.out_row);
+  COMET_LAUNCH_CHECK(ctx);
+  return COMET_OK;
+}
+
 comet_status_t seg_dot(Context *ctx, const int32_t *seg_end, const int32_t *crd, const double *val, int64_t M,
                        int64_t N, const double *x, int64_t x_len, double *y, const int32_t *out_row,
                        int64_t out_rows, cudaStream_t stream) {
@@ -348,11 +510,18 @@ comet_status_t seg_dot(Context *ctx, const int32_t *seg_end, const int32_t *crd,
   if (M == 0) return COMET_OK;
   SegDotArgs a{};
   a.seg_end = seg_end; a.crd = crd; a.val = val; a.M = M; a.N = N; a.x = x; a.y = y; a.out_row = out_row;
-  // Large problems whose vector fits in shared memory beside the staging: persistent CTAs, x resident.
+  // Large problems: the warp-stream kernel (x in shared memory when it fits).
+  {
+    const char *force = getenv("COMET_SEG_DOT_KERNEL");   // tests: "stream", "resident" or "tile" on any input
+    const bool want_stream = force ? !strcmp(force, "stream") : (N >= (int64_t)kSmCount * 32 * 512 && N > 0);
+    if (want_stream && N > 0) return launch_stream(ctx, a, x_len, stream);
+  }
+  // Mid-size problems whose vector fits in shared memory beside the staging: persistent CTAs, x resident.
   {
     using RL = ResidentLayout<kResThreads, kResIpt>;
     const size_t need = align_up((size_t)x_len * 8, 16) + (size_t)kResVC * RL::kStageBytes;
-    const bool forced = getenv("COMET_SEG_DOT_RESIDENT") != nullptr;     // tests: exercise this path on small inputs
+    const char *force = getenv("COMET_SEG_DOT_KERNEL");
+    const bool forced = force && !strcmp(force, "resident");
     if (need <= kMaxDynamicSmem && (forced || M + N >= (int64_t)kSmCount * kResVC * RL::TILE * 8))
       return launch_resident(ctx, a, x_len, stream);
   }

@@ -34,13 +34,18 @@ def tile_items(request, monkeypatch):
     return request.param
 
 
-@pytest.fixture(params=["default", "resident"])
+@pytest.fixture(params=["default", "resident", "stream", "stream-short-spans"])
 def seg_dot_path(request, monkeypatch):
-    """SpMV/TTV kernel choice: the size-based default, and the persistent resident-vector kernel forced."""
+    """SpMV/TTV kernel choice: the size-based default, then each large-input kernel forced on small inputs
+    (the warp-stream kernel also with 128-entry spans, so that segments straddle many spans)."""
+    monkeypatch.delenv("COMET_SEG_DOT_KERNEL", raising=False)
+    monkeypatch.delenv("COMET_STREAM_SPAN", raising=False)
     if request.param == "resident":
-        monkeypatch.setenv("COMET_SEG_DOT_RESIDENT", "1")
-    else:
-        monkeypatch.delenv("COMET_SEG_DOT_RESIDENT", raising=False)
+        monkeypatch.setenv("COMET_SEG_DOT_KERNEL", "resident")
+    elif request.param.startswith("stream"):
+        monkeypatch.setenv("COMET_SEG_DOT_KERNEL", "stream")
+        if request.param.endswith("short-spans"):
+            monkeypatch.setenv("COMET_STREAM_SPAN", "128")
     return request.param
 
 
