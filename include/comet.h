@@ -125,7 +125,8 @@ comet_status_t comet_sptensor_free(comet_handle_t handle, comet_sptensor_t *tens
 comet_status_t comet_validate(comet_handle_t handle, const comet_sptensor_t *tensor, void *stream);
 
 /* SpMV  y_i = sum_j A_ij x_j  (SpMV definition in the Sparse Tensor Operations subsection).
- * A: 2 levels, [D,CU] (CSR), [CU,CU] (DCSR) or [CN,S] (COO). x: dims[mode_order[1]] values;
+ * A: 2 levels, [D,CU] (CSR), [CU,CU] (DCSR) or [CN,S] (COO; its row structure is rebuilt into a
+ * temporary obtained from the handle's allocator). x: dims[mode_order[1]] values;
  * y: dims[mode_order[0]] values, every entry written. */
 comet_status_t comet_spmv(comet_handle_t handle, const comet_sptensor_t *A, const void *x, void *y, void *stream);
 

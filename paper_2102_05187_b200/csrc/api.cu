@@ -75,6 +75,31 @@ __global__ void expand_root_pos_kernel(const int32_t *__restrict__ crd0, const i
 
 __global__ void set_word_kernel(int32_t *p, int32_t v) { *p = v; }
 
+// CSR pos of a sorted COO matrix: pos[i] = number of entries whose root coordinate is below i
+__global__ void coo_row_pos_kernel(const int32_t *__restrict__ crd0, int64_t n, int64_t rows, int32_t *__restrict__ pos) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i > rows) return;
+  int64_t lo = 0, hi = n;
+  while (lo < hi) {
+    const int64_t mid = (lo + hi) >> 1;
+    if ((int64_t)__ldg(crd0 + mid) < i) lo = mid + 1; else hi = mid;
+  }
+  pos[i] = (int32_t)lo;
+}
+
+// [CN,S] matrices go through the CSR kernels: the row structure the compressed level would store is
+// rebuilt from the sorted root coordinates into scratch that sits in front of the kernels' own scratch.
+comet_status_t coo_rows(Context *ctx, const comet_sptensor_t *A, int64_t rows, cudaStream_t s, int32_t **pos_out) {
+  int32_t *pos = (int32_t *)ctx_alloc(ctx, (size_t)(rows + 1) * sizeof(int32_t), s);
+  if (!pos) return COMET_ERR_ALLOC;
+  coo_row_pos_kernel<<<(unsigned)ceil_div(rows + 1, 256), 256, 0, s>>>(A->crd[0], A->nnz, rows, pos);
+  ctx->launches += 1;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { ctx_free(ctx, pos, s); return cuda_fail(ctx, e); }
+  *pos_out = pos;
+  return COMET_OK;
+}
+
 }  // namespace
 
 namespace comet {
@@ -109,6 +134,15 @@ extern "C" comet_status_t comet_spmv(comet_handle_t handle, const comet_sptensor
   if (is_fmt(A, 2, COMET_CU, COMET_CU))
     return seg_dot(ctx, A->pos[1] + 1, A->crd[1], (const double *)A->val, A->crd_len[0], A->nnz, (const double *)x,
                    A->dims[A->mode_order[1]], (double *)y, A->crd[0], rows, s);
+  if (is_fmt(A, 2, COMET_CN, COMET_S)) {
+    int32_t *pos = nullptr;
+    st = coo_rows(ctx, A, rows, s, &pos);
+    if (st != COMET_OK) return st;
+    st = seg_dot(ctx, pos + 1, A->crd[1], (const double *)A->val, rows, A->nnz, (const double *)x,
+                 A->dims[A->mode_order[1]], (double *)y, nullptr, rows, s);
+    ctx_free(ctx, pos, s);          // stream-ordered allocators release after the queued work
+    return st;
+  }
   return COMET_ERR_UNSUPPORTED_FORMAT;
 }
 
@@ -128,6 +162,15 @@ extern "C" comet_status_t comet_spmm(comet_handle_t handle, const comet_sptensor
     if (A->crd_len[0] == 0) return zero_rows(ctx, (double *)C, rows, R, ldc, s);
     return seg_gather(ctx, A->pos[1] + 1, A->crd[1], (const double *)A->val, A->crd_len[0], A->nnz,
                       (const double *)B, ldb, R, (double *)C, ldc, A->crd[0], rows, s);
+  }
+  if (is_fmt(A, 2, COMET_CN, COMET_S)) {
+    int32_t *pos = nullptr;
+    st = coo_rows(ctx, A, rows, s, &pos);
+    if (st != COMET_OK) return st;
+    st = seg_gather(ctx, pos + 1, A->crd[1], (const double *)A->val, rows, A->nnz, (const double *)B, ldb, R,
+                    (double *)C, ldc, nullptr, rows, s);
+    ctx_free(ctx, pos, s);
+    return st;
   }
   return COMET_ERR_UNSUPPORTED_FORMAT;
 }

@@ -52,7 +52,7 @@ def seg_dot_path(request, monkeypatch):
 def test_worked_example():
     mc = ([0, 0, 2, 2, 2, 3], [1, 4, 0, 1, 5, 3])
     mv = [1.0, 2.0, 3.0, 4.0, 5.0, 6.0]
-    for attr in [(D, CU), (CU, CU)]:
+    for attr in [(D, CU), (CU, CU), (CN, S)]:
         A = upload_packed(oracle.pack(mc, mv, (4, 6), (0, 1), attr))
         y = comet.spmv(A, dev([1.0, 2, 3, 4, 5, 6]))
         assert y.tolist() == [12.0, 0.0, 41.0, 24.0]
@@ -79,7 +79,7 @@ MATRIX_CASES = [((64, 48), 700, 1), ((300, 200), 5000, 2), ((1, 500), 300, 3), (
 
 
 @pytest.mark.parametrize("dims,nnz,seed", MATRIX_CASES)
-@pytest.mark.parametrize("attr", [(D, CU), (CU, CU)])
+@pytest.mark.parametrize("attr", [(D, CU), (CU, CU), (CN, S)])
 def test_spmv(dims, nnz, seed, attr, tile_items, seg_dot_path):
     coords, val = synth.random_coo(dims, nnz, seed)
     c, v = _np(coords), val.numpy()
@@ -92,7 +92,7 @@ def test_spmv(dims, nnz, seed, attr, tile_items, seg_dot_path):
 
 
 @pytest.mark.parametrize("dims,nnz,seed", MATRIX_CASES)
-@pytest.mark.parametrize("attr", [(D, CU), (CU, CU)])
+@pytest.mark.parametrize("attr", [(D, CU), (CU, CU), (CN, S)])
 @pytest.mark.parametrize("R", [1, 2, 3, 8, 16, 17, 32, 64, 100, 128, 130])
 def test_spmm(dims, nnz, seed, attr, R, tile_items):
     if tile_items == 37 and R not in (2, 17, 64):
