@@ -29,7 +29,8 @@
  *   - A handle caches scratch memory and may be used from one stream at a time.
  *   - Errors are return codes; nothing aborts, throws or traps. Errors detectable on the host are
  *     returned before anything is launched.
- *   - Limits: nnz, every extent and every pos value must be < 2^31 - 1 (int32 indices).
+ *   - Limits: nnz, every extent and every pos value must be < 2^31 - 1 (int32 indices); leading
+ *     dimensions of gathered dense operands must be < 2^28 elements (COMET_ERR_INDEX_OVERFLOW).
  *   - Values are fp64 (COMET_F64). COMET_F32 is reserved and reported as unsupported.
  */
 #ifndef COMET_H
@@ -138,11 +139,12 @@ comet_status_t comet_spmm(comet_handle_t handle, const comet_sptensor_t *A, cons
                           void *C, int64_t ldc, void *stream);
 
 /* TTV  Y = X x_n v  (SpTTV definition; `mode` = n, 0-based, must be the mode of X's LAST level).
- * X: 3 levels, [CU,CU,CU] (CSF) or [CN,S,S] (COO). The result is sparse, one order lower:
+ * X: 3 levels, [CU,CU,CU] (CSF; a COO tensor is first re-packed with comet_pack). The result is sparse,
+ * one order lower:
  * comet_ttv_symbolic builds its structure over (mode_order[0], mode_order[1]) with level attributes
  * h_out_attr = {D,CU} (CSR) or {CU,CU} (DCSR); values are then (re)computed by comet_ttv, which
  * writes only Y->val. The structure depends on X's structure alone, never on values. Y owns its
- * arrays; X need not outlive it. comet_ttv_symbolic synchronises `stream` once for COO inputs. */
+ * arrays; X need not outlive it. */
 comet_status_t comet_ttv_symbolic(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode,
                                   const int32_t *h_out_attr, void *stream, comet_sptensor_t *Y);
 comet_status_t comet_ttv(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode, const void *v,

@@ -225,6 +225,7 @@ static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 comet_status_t seg_gather(Context *ctx, const int32_t *seg_end, const int32_t *crd, const double *val, int64_t M,
                           int64_t N, const double *B, int64_t ldb, int64_t R, double *C, int64_t ldc,
                           const int32_t *out_row, int64_t out_rows, cudaStream_t stream) {
+  if (ldb >= (1ll << 28)) return COMET_ERR_INDEX_OVERFLOW;      // row offsets are formed as int32 bytes * int32 index
   if (M == 0) return out_row ? zero_rows(ctx, C, out_rows, R, ldc, stream) : COMET_OK;
   const bool vec_ok = aligned16(B) && aligned16(C) && (ldb % 2 == 0) && (ldc % 2 == 0);
   int64_t done = 0;

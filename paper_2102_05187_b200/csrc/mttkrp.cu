@@ -312,6 +312,7 @@ static comet_status_t mttkrp_chunks(Context *ctx, MttkrpArgs base, int64_t R, cu
 comet_status_t mttkrp_coo(Context *ctx, const int32_t *crd0, const int32_t *crd1, const int32_t *crd2,
                           const double *val, int64_t N, int64_t rows, const double *P, int64_t ldp, const double *Q,
                           int64_t ldq, int64_t R, double *out, int64_t ldo, cudaStream_t stream) {
+  if (ldp >= (1ll << 28) || ldq >= (1ll << 28)) return COMET_ERR_INDEX_OVERFLOW;
   if (N == 0) return zero_rows(ctx, out, rows, R, ldo, stream);
   MttkrpArgs a{};
   a.crd0 = crd0; a.crd1 = crd1; a.crd2 = crd2; a.val = val; a.N = N; a.rows = rows;
@@ -323,6 +324,7 @@ comet_status_t mttkrp_csf(Context *ctx, const int32_t *pos1, const int32_t *crd0
                           const int32_t *pos2, const int32_t *crd2, const double *val, int64_t S, int64_t F,
                           int64_t N, int64_t rows, const double *P, int64_t ldp, const double *Q, int64_t ldq,
                           int64_t R, double *out, int64_t ldo, cudaStream_t stream) {
+  if (ldp >= (1ll << 28) || ldq >= (1ll << 28)) return COMET_ERR_INDEX_OVERFLOW;
   if (N == 0 || S == 0) return zero_rows(ctx, out, rows, R, ldo, stream);
   MttkrpArgs a{};
   a.pos1 = pos1; a.crd0 = crd0; a.crd1 = crd1; a.seg_end2 = pos2 + 1; a.crd2 = crd2; a.val = val;
