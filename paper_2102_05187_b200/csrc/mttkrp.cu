@@ -148,15 +148,20 @@ struct CsfPolicy {
   double *ocol;
   double tac[CPL][VEC], aac[CPL][VEC];   // open fiber sum, open slice sum
   double prow[CPL][VEC];                 // P row of the open fiber, fetched when the fiber opened
-  int64_t f, s;                          // open fiber, open slice
+  // cursors instead of indices: the per-fiber path is executed once per fiber and per worker (divergently),
+  // so it is kept to pointer bumps and 32-bit compares
+  const int32_t *endp;                   // seg_end2 + open fiber
+  const int32_t *c1p;                    // crd1 + open fiber
+  int32_t fibers_left;                   // fibers from the open one to the last
+  int32_t to_slice_end;                  // fibers from the open one to the end of the open slice
+  int32_t s;                             // open slice
   int32_t next_end;                      // leaf position where the open fiber ends
   int32_t base, rel_end;
-  int64_t slice_end;                     // fiber index where the open slice ends
   int32_t last_fold;                     // leaf position of the latest fold (entries at or after it are in tac)
   bool a_dirty;
 
   __device__ __forceinline__ CsfPolicy(const MttkrpArgs &args, const L &lanes, int64_t f0, int64_t s0, int32_t j0)
-      : a(args), ln(lanes), f(f0), s(s0), base(j0), last_fold(j0), a_dirty(false) {
+      : a(args), ln(lanes), s((int32_t)s0), base(j0), last_fold(j0), a_dirty(false) {
     ln.zero(tac);
     ln.zero(aac);
     ln.zero(prow);
@@ -165,13 +170,17 @@ struct CsfPolicy {
     ldp_bytes = (int32_t)(a.ldp * 8);
     ldq_bytes = (int32_t)(a.ldq * 8);
     ocol = a.out + ln.col0;
-    next_end = f < a.F ? __ldg(a.seg_end2 + f) : -1;
+    endp = a.seg_end2 + f0;
+    c1p = a.crd1 + f0;
+    fibers_left = (int32_t)(a.F - f0);
+    next_end = fibers_left > 0 ? __ldg(endp) : -1;
     rel_end = next_end - base;
-    slice_end = s < a.S ? (int64_t)__ldg(a.pos1 + s + 1) : -1;
+    to_slice_end = s < a.S ? (int32_t)(__ldg(a.pos1 + s + 1) - f0) : -1;
     open_fiber();
   }
+  __device__ __forceinline__ int64_t fiber() const { return a.F - fibers_left; }
   __device__ __forceinline__ void open_fiber() {         // start fetching the P row the fiber will be folded with
-    if (f < a.F) ln.gather(reinterpret_cast<const double *>(pcol + (int64_t)__ldg(a.crd1 + f) * ldp_bytes), prow);
+    if (fibers_left > 0) ln.gather(reinterpret_cast<const double *>(pcol + (int64_t)__ldg(c1p) * ldp_bytes), prow);
   }
   __device__ __forceinline__ void fetch(int32_t j, Entry16 &e, int32_t &) const {
     e.v = ld_stream(a.val + j);
@@ -191,23 +200,26 @@ struct CsfPolicy {
     a_dirty = true;
     last_fold = j;
   }
+  __device__ __forceinline__ void close_slice() {        // the slice is complete: this worker owns its row
+    const int64_t row = __ldg(a.crd0 + s);
+    const int64_t lo = s > 0 ? (int64_t)__ldg(a.crd0 + s - 1) + 1 : 0;
+    ln.zero_rows(ocol, a.ldo, lo, row);
+    ln.store_row(ocol + row * a.ldo, aac);
+    if (s == a.S - 1) ln.zero_rows(ocol, a.ldo, row + 1, a.rows);
+    ln.zero(aac);
+    a_dirty = false;
+    ++s;
+    to_slice_end = s < a.S ? __ldg(a.pos1 + s + 1) - __ldg(a.pos1 + s) : -1;
+  }
   __device__ __forceinline__ void end_fiber(int32_t j) {
     fold(j);
-    ++f;
-    next_end = f < a.F ? __ldg(a.seg_end2 + f) : -1;
+    ++endp;
+    ++c1p;
+    --fibers_left;
+    next_end = fibers_left > 0 ? __ldg(endp) : -1;
     rel_end = next_end - base;
     open_fiber();
-    if (f == slice_end) {                                // the slice is complete: this worker owns its row
-      const int64_t row = __ldg(a.crd0 + s);
-      const int64_t lo = s > 0 ? (int64_t)__ldg(a.crd0 + s - 1) + 1 : 0;
-      ln.zero_rows(ocol, a.ldo, lo, row);
-      ln.store_row(ocol + row * a.ldo, aac);
-      if (s == a.S - 1) ln.zero_rows(ocol, a.ldo, row + 1, a.rows);
-      ln.zero(aac);
-      a_dirty = false;
-      ++s;
-      slice_end = s < a.S ? (int64_t)__ldg(a.pos1 + s + 1) : -1;
-    }
+    if (--to_slice_end == 0) close_slice();
   }
   __device__ __forceinline__ void consume(int q, double v, int32_t, Slot &sl) {
     while (rel_end == q) end_fiber(base + q);
@@ -243,7 +255,7 @@ __global__ void __launch_bounds__(kBlockThreads, (CPL * VEC <= 2 ? COMET_MINB_CS
 
   P p(a, ln, f0, lo, j0);
   walk_tile(ln, p, j0, j1, smem);
-  while (p.f < f1) p.end_fiber(j1);
+  while (p.fiber() < f1) p.end_fiber(j1);
   if (j1 > p.last_fold) p.fold(j1);                      // an unfinished fiber contributes through distributivity
   const bool carry = p.a_dirty && p.s < a.S;
   if (ln.g == 0) a.carry_seg[tile] = carry ? (int32_t)p.s : -1;
