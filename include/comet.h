@@ -31,7 +31,12 @@
  *     returned before anything is launched.
  *   - Limits: nnz, every extent and every pos value must be < 2^31 - 1 (int32 indices); leading
  *     dimensions of gathered dense operands must be < 2^28 elements (COMET_ERR_INDEX_OVERFLOW).
- *   - Values are fp64 (COMET_F64). COMET_F32 is reserved and reported as unsupported.
+ *   - Values are fp64 (COMET_F64) or fp32 (COMET_F32); a tensor's dtype is also the type of every dense
+ *     operand and output of a call on it (no mixing: the library cannot see a dense buffer's type, so the
+ *     caller must get this right; a sparse OUTPUT of another dtype is COMET_ERR_INVALID_ARG). Products and
+ *     sums are formed in double for both types and rounded once when stored; with fp32 a row that spans
+ *     several tiles is rounded once more when its carry is added. Dense pointers must be aligned to one
+ *     element (COMET_ERR_MISALIGNED).
  */
 #ifndef COMET_H
 #define COMET_H
@@ -133,8 +138,8 @@ comet_status_t comet_spmv(comet_handle_t handle, const comet_sptensor_t *A, cons
 
 /* SpMM  C_ir = sum_j A_ij B_jr  (SpMM definition). B: dims[mode_order[1]] x R, leading dimension
  * ldb >= R; C: dims[mode_order[0]] x R, leading dimension ldc >= R; every row of C is written.
- * Formats as for comet_spmv. Any R >= 1; R in {2,4,8,16,32,64,128} with 16-byte-aligned rows takes
- * the vectorised path. */
+ * Formats as for comet_spmv. Any R >= 1; columns are processed in chunks of up to 128, and a chunk of
+ * 2^k 16-byte pieces (fp64: 2..128 columns, fp32: 4..128) on 16-byte-aligned rows takes the vectorised path. */
 comet_status_t comet_spmm(comet_handle_t handle, const comet_sptensor_t *A, const void *B, int64_t R, int64_t ldb,
                           void *C, int64_t ldc, void *stream);
 
@@ -179,7 +184,7 @@ comet_status_t comet_mttkrp(comet_handle_t handle, const comet_sptensor_t *X, in
  * scratch from an allocator; this entry point needs neither. It calls no cudaMalloc, cudaFree or
  * any other allocating routine, directly or through a library.
  *
- * Same result as comet_spmv for A = [D,CU] (other formats: COMET_ERR_UNSUPPORTED_FORMAT). The caller
+ * Same result as comet_spmv for A = [D,CU] with fp64 values (other formats or fp32: COMET_ERR_UNSUPPORTED_FORMAT). The caller
  * still passes the inputs and the output (device pointers, y has dims[mode_order[0]] entries and is
  * fully overwritten). The per-tile carry slots live in a fixed 768 KiB device array that is part of
  * the library image: every GPU that loads the library holds it until the process exits.

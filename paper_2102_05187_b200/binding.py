@@ -15,6 +15,25 @@ import torch
 
 D, CU, CN, S = 0, 1, 2, 3
 F64 = 0
+F32 = 1
+_TORCH_DTYPE = {F64: torch.float64, F32: torch.float32}
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    """comet_dtype_t of a value tensor (fp64 or fp32; anything else is refused here)."""
+    if t.dtype == torch.float64:
+        return F64
+    if t.dtype == torch.float32:
+        return F32
+    raise TypeError(f"values must be float64 or float32, got {t.dtype}")
+
+
+def _same_dtype(A, *tensors):
+    want = _TORCH_DTYPE[A.c.dtype]
+    for t in tensors:
+        if t is not None and t.dtype != want:
+            raise TypeError(f"dense operand is {t.dtype}, the sparse tensor's values are {want}")
+    return want
 MAX_ORDER = 4
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -204,7 +223,7 @@ class SpTensor:
 
     @property
     def val(self):
-        return _from_ptr(self.c.val, self.c.nnz, torch.float64, self)
+        return _from_ptr(self.c.val, self.c.nnz, _TORCH_DTYPE[self.c.dtype], self)
 
     def free(self):
         if self.c.owner:
@@ -219,11 +238,12 @@ class SpTensor:
 
     @staticmethod
     def from_arrays(dims, mode_order, attr, pos, crd, val, handle: Handle | None = None) -> "SpTensor":
-        """Describe caller-built level arrays (torch CUDA int32 / float64 tensors; None where a level has none)."""
+        """Describe caller-built level arrays (torch CUDA int32 tensors, float64 or float32 values; None where a
+        level has none)."""
         handle = handle or default_handle()
         s = SpTensorStruct()
         order = len(dims)
-        s.order, s.dtype = order, F64
+        s.order, s.dtype = order, _dtype_code(val)
         keep = []
         for m in range(order):
             s.dims[m] = int(dims[m])
@@ -241,7 +261,7 @@ class SpTensor:
             s.crd[m] = 0 if c is None else c.data_ptr()
             s.crd_len[m] = 0 if c is None else c.numel()
         _require_cuda(val)
-        assert val.dtype == torch.float64 and val.is_contiguous()
+        assert val.is_contiguous()
         keep.append(val)
         s.val = val.data_ptr() if val.numel() else 0
         s.nnz = val.numel()
@@ -259,7 +279,7 @@ def _from_ptr(ptr, n, dtype, owner):
         pass
 
     iface = _Iface()
-    typestr = {torch.int32: "<i4", torch.float64: "<f8", torch.uint8: "|u1"}[dtype]
+    typestr = {torch.int32: "<i4", torch.float64: "<f8", torch.float32: "<f4", torch.uint8: "|u1"}[dtype]
     iface.__cuda_array_interface__ = {"shape": (int(n),), "typestr": typestr, "data": (int(ptr), False),
                                       "version": 3, "strides": (itemsize,)}
     iface._owner = owner
@@ -275,14 +295,14 @@ def pack(coords, val, dims, mode_order, attr, handle: Handle | None = None) -> S
     _require_cuda(val, *coords)
     coords = [c.contiguous() for c in coords]
     val = val.contiguous()
-    assert all(c.dtype == torch.int32 for c in coords) and val.dtype == torch.float64
+    assert all(c.dtype == torch.int32 for c in coords)
     h_dims = (C.c_int64 * order)(*[int(d) for d in dims])
     h_crd = (C.c_void_p * order)(*[c.data_ptr() for c in coords])
     h_mo = (C.c_int32 * order)(*[int(m) for m in mode_order])
     h_at = (C.c_int32 * order)(*[int(a) for a in attr])
     out = SpTensorStruct()
     st = handle.lib.comet_pack(handle._h, C.c_int32(order), h_dims, C.c_int64(val.numel()), h_crd, _ptr(val),
-                               C.c_int(F64), h_mo, h_at, _stream_ptr(), C.byref(out))
+                               C.c_int(_dtype_code(val)), h_mo, h_at, _stream_ptr(), C.byref(out))
     handle.check(st, "comet_pack")
     return SpTensor(handle, out)
 
@@ -294,8 +314,9 @@ def validate(t: SpTensor):
 def spmv(A: SpTensor, x: torch.Tensor, y: torch.Tensor | None = None) -> torch.Tensor:
     _require_cuda(x)
     rows = A.c.dims[A.c.mode_order[0]]
+    dt = _same_dtype(A, x, y)
     if y is None:
-        y = torch.empty(rows, dtype=torch.float64, device=x.device)
+        y = torch.empty(rows, dtype=dt, device=x.device)
     st = A.handle.lib.comet_spmv(A.handle._h, C.byref(A.c), _ptr(x), _ptr(y), _stream_ptr())
     A.handle.check(st, "comet_spmv")
     return y
@@ -306,8 +327,9 @@ def spmm(A: SpTensor, B: torch.Tensor, out: torch.Tensor | None = None) -> torch
     assert B.dim() == 2 and B.stride(1) == 1
     rows = A.c.dims[A.c.mode_order[0]]
     R = B.shape[1]
+    dt = _same_dtype(A, B, out)
     if out is None:
-        out = torch.empty((rows, R), dtype=torch.float64, device=B.device)
+        out = torch.empty((rows, R), dtype=dt, device=B.device)
     st = A.handle.lib.comet_spmm(A.handle._h, C.byref(A.c), _ptr(B), C.c_int64(R), C.c_int64(B.stride(0)),
                                  _ptr(out), C.c_int64(out.stride(0)), _stream_ptr())
     A.handle.check(st, "comet_spmm")
@@ -324,6 +346,7 @@ def ttv_symbolic(X: SpTensor, mode: int, out_attr=(D, CU)) -> SpTensor:
 
 def ttv(X: SpTensor, mode: int, v: torch.Tensor, Y: SpTensor | None = None) -> SpTensor:
     _require_cuda(v)
+    _same_dtype(X, v)
     if Y is None:
         Y = ttv_symbolic(X, mode)
     st = X.handle.lib.comet_ttv(X.handle._h, C.byref(X.c), C.c_int32(mode), _ptr(v), C.byref(Y.c), _stream_ptr())
@@ -343,6 +366,7 @@ def ttm(X: SpTensor, mode: int, U: torch.Tensor, Y: SpTensor | None = None) -> S
     _require_cuda(U)
     assert U.dim() == 2 and U.stride(1) == 1
     R = U.shape[1]
+    _same_dtype(X, U)
     if Y is None:
         Y = ttm_symbolic(X, mode, R)
     st = X.handle.lib.comet_ttm(X.handle._h, C.byref(X.c), C.c_int32(mode), _ptr(U), C.c_int64(R),
@@ -358,8 +382,9 @@ def mttkrp(X: SpTensor, mode: int, factors, out: torch.Tensor | None = None) -> 
     R = live[0].shape[1]
     assert all(f.dim() == 2 and f.stride(1) == 1 and f.shape[1] == R for f in live)
     rows = X.c.dims[mode]
+    dt = _same_dtype(X, out, *live)
     if out is None:
-        out = torch.empty((rows, R), dtype=torch.float64, device=live[0].device)
+        out = torch.empty((rows, R), dtype=dt, device=live[0].device)
     h_f = (C.c_void_p * 3)(*[0 if (m == mode or f is None) else f.data_ptr() for m, f in enumerate(factors)])
     h_ld = (C.c_int64 * 3)(*[0 if (m == mode or f is None) else f.stride(0) for m, f in enumerate(factors)])
     st = X.handle.lib.comet_mttkrp(X.handle._h, C.byref(X.c), C.c_int32(mode), h_f, h_ld, C.c_int64(R), _ptr(out),

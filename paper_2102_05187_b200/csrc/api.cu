@@ -22,7 +22,7 @@ bool is_fmt(const comet_sptensor_t *t, int order, int a0, int a1, int a2 = -1) {
 comet_status_t check_tensor(const comet_sptensor_t *t, int order) {
   if (!t) return COMET_ERR_INVALID_ARG;
   if (t->order != order) return COMET_ERR_UNSUPPORTED_FORMAT;
-  if (t->dtype != COMET_F64) return COMET_ERR_UNSUPPORTED_FORMAT;
+  if (t->dtype != COMET_F64 && t->dtype != COMET_F32) return COMET_ERR_UNSUPPORTED_FORMAT;
   if (t->nnz < 0) return COMET_ERR_INVALID_ARG;
   if (t->nnz > kIndexLimit) return COMET_ERR_INDEX_OVERFLOW;
   bool seen[COMET_MAX_ORDER] = {false, false, false, false};
@@ -41,7 +41,9 @@ comet_status_t check_tensor(const comet_sptensor_t *t, int order) {
   return COMET_OK;
 }
 
-bool misaligned8(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 7) != 0; }
+// Dense operands and outputs carry the tensor's value type and must be aligned to one element of it.
+size_t elem_size(int dtype) { return dtype == COMET_F32 ? 4 : 8; }
+bool misaligned(const void *p, int dtype) { return (reinterpret_cast<uintptr_t>(p) & (elem_size(dtype) - 1)) != 0; }
 
 struct Owner {           // bookkeeping of a library-owned tensor: the blocks to release
   int count;
@@ -124,22 +126,21 @@ extern "C" comet_status_t comet_spmv(comet_handle_t handle, const comet_sptensor
   if (!handle || !x || !y) return COMET_ERR_INVALID_ARG;
   comet_status_t st = check_tensor(A, 2);
   if (st != COMET_OK) return st;
-  if (misaligned8(x) || misaligned8(y)) return COMET_ERR_MISALIGNED;
+  if (misaligned(x, A->dtype) || misaligned(y, A->dtype)) return COMET_ERR_MISALIGNED;
   Context *ctx = reinterpret_cast<Context *>(handle);
   cudaStream_t s = (cudaStream_t)stream;
   const int64_t rows = A->dims[A->mode_order[0]];
   if (is_fmt(A, 2, COMET_D, COMET_CU))
-    return seg_dot(ctx, A->pos[1] + 1, A->crd[1], (const double *)A->val, rows, A->nnz, (const double *)x,
-                   A->dims[A->mode_order[1]], (double *)y, nullptr, rows, s);
+    return seg_dot(ctx, A->dtype, A->pos[1] + 1, A->crd[1], A->val, rows, A->nnz, x, A->dims[A->mode_order[1]], y, nullptr,
+                   rows, s);
   if (is_fmt(A, 2, COMET_CU, COMET_CU))
-    return seg_dot(ctx, A->pos[1] + 1, A->crd[1], (const double *)A->val, A->crd_len[0], A->nnz, (const double *)x,
-                   A->dims[A->mode_order[1]], (double *)y, A->crd[0], rows, s);
+    return seg_dot(ctx, A->dtype, A->pos[1] + 1, A->crd[1], A->val, A->crd_len[0], A->nnz, x, A->dims[A->mode_order[1]], y,
+                   A->crd[0], rows, s);
   if (is_fmt(A, 2, COMET_CN, COMET_S)) {
     int32_t *pos = nullptr;
     st = coo_rows(ctx, A, rows, s, &pos);
     if (st != COMET_OK) return st;
-    st = seg_dot(ctx, pos + 1, A->crd[1], (const double *)A->val, rows, A->nnz, (const double *)x,
-                 A->dims[A->mode_order[1]], (double *)y, nullptr, rows, s);
+    st = seg_dot(ctx, A->dtype, pos + 1, A->crd[1], A->val, rows, A->nnz, x, A->dims[A->mode_order[1]], y, nullptr, rows, s);
     ctx_free(ctx, pos, s);          // stream-ordered allocators release after the queued work
     return st;
   }
@@ -151,24 +152,22 @@ extern "C" comet_status_t comet_spmm(comet_handle_t handle, const comet_sptensor
   if (!handle || !B || !C || R < 1 || ldb < R || ldc < R) return COMET_ERR_INVALID_ARG;
   comet_status_t st = check_tensor(A, 2);
   if (st != COMET_OK) return st;
-  if (misaligned8(B) || misaligned8(C)) return COMET_ERR_MISALIGNED;
+  if (misaligned(B, A->dtype) || misaligned(C, A->dtype)) return COMET_ERR_MISALIGNED;
   Context *ctx = reinterpret_cast<Context *>(handle);
   cudaStream_t s = (cudaStream_t)stream;
   const int64_t rows = A->dims[A->mode_order[0]];
   if (is_fmt(A, 2, COMET_D, COMET_CU))
-    return seg_gather(ctx, A->pos[1] + 1, A->crd[1], (const double *)A->val, rows, A->nnz, (const double *)B, ldb, R,
-                      (double *)C, ldc, nullptr, rows, s);
+    return seg_gather(ctx, A->dtype, A->pos[1] + 1, A->crd[1], A->val, rows, A->nnz, B, ldb, R, C, ldc, nullptr, rows, s);
   if (is_fmt(A, 2, COMET_CU, COMET_CU)) {
-    if (A->crd_len[0] == 0) return zero_rows(ctx, (double *)C, rows, R, ldc, s);
-    return seg_gather(ctx, A->pos[1] + 1, A->crd[1], (const double *)A->val, A->crd_len[0], A->nnz,
-                      (const double *)B, ldb, R, (double *)C, ldc, A->crd[0], rows, s);
+    if (A->crd_len[0] == 0) return zero_rows(ctx, C, A->dtype, rows, R, ldc, s);
+    return seg_gather(ctx, A->dtype, A->pos[1] + 1, A->crd[1], A->val, A->crd_len[0], A->nnz, B, ldb, R, C, ldc, A->crd[0],
+                      rows, s);
   }
   if (is_fmt(A, 2, COMET_CN, COMET_S)) {
     int32_t *pos = nullptr;
     st = coo_rows(ctx, A, rows, s, &pos);
     if (st != COMET_OK) return st;
-    st = seg_gather(ctx, pos + 1, A->crd[1], (const double *)A->val, rows, A->nnz, (const double *)B, ldb, R,
-                    (double *)C, ldc, nullptr, rows, s);
+    st = seg_gather(ctx, A->dtype, pos + 1, A->crd[1], A->val, rows, A->nnz, B, ldb, R, C, ldc, nullptr, rows, s);
     ctx_free(ctx, pos, s);
     return st;
   }
@@ -218,7 +217,7 @@ extern "C" comet_status_t comet_ttv_symbolic(comet_handle_t handle, const comet_
   const int64_t S = X->crd_len[0], F = X->crd_len[1];
   const int64_t rows = X->dims[X->mode_order[0]];
   Y->order = 2;
-  Y->dtype = COMET_F64;
+  Y->dtype = X->dtype;
   Y->dims[0] = rows;
   Y->dims[1] = X->dims[X->mode_order[1]];
   Y->mode_order[0] = 0;
@@ -246,7 +245,7 @@ extern "C" comet_status_t comet_ttv_symbolic(comet_handle_t handle, const comet_
     }
   }
   if (st == COMET_OK) {
-    Y->val = owned_alloc(ctx, o, (size_t)F * sizeof(double), s);
+    Y->val = owned_alloc(ctx, o, (size_t)F * elem_size(X->dtype), s);
     if (!Y->val) st = COMET_ERR_ALLOC;
   }
   if (st != COMET_OK) { release(ctx, o, s); memset(Y, 0, sizeof(*Y)); return st; }
@@ -260,10 +259,11 @@ extern "C" comet_status_t comet_ttv(comet_handle_t handle, const comet_sptensor_
   comet_status_t st = check_last_mode(X, mode);
   if (st != COMET_OK) return st;
   if (Y->order != 2 || Y->nnz != X->crd_len[1] || (Y->nnz > 0 && !Y->val)) return COMET_ERR_INVALID_ARG;
-  if (misaligned8(v)) return COMET_ERR_MISALIGNED;
+  if (Y->dtype != X->dtype) return COMET_ERR_INVALID_ARG;
+  if (misaligned(v, X->dtype)) return COMET_ERR_MISALIGNED;
   Context *ctx = reinterpret_cast<Context *>(handle);
-  return seg_dot(ctx, X->pos[2] + 1, X->crd[2], (const double *)X->val, X->crd_len[1], X->nnz, (const double *)v,
-                 X->dims[mode], (double *)Y->val, nullptr, X->crd_len[1], (cudaStream_t)stream);
+  return seg_dot(ctx, X->dtype, X->pos[2] + 1, X->crd[2], X->val, X->crd_len[1], X->nnz, v, X->dims[mode], Y->val, nullptr,
+                 X->crd_len[1], (cudaStream_t)stream);
 }
 
 extern "C" comet_status_t comet_ttm_symbolic(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode,
@@ -279,7 +279,7 @@ extern "C" comet_status_t comet_ttm_symbolic(comet_handle_t handle, const comet_
   if (!o) return COMET_ERR_ALLOC;
   const int64_t F = X->crd_len[1];
   Y->order = 3;
-  Y->dtype = COMET_F64;
+  Y->dtype = X->dtype;
   for (int m = 0; m < 3; ++m) { Y->dims[m] = X->dims[m]; Y->mode_order[m] = X->mode_order[m]; }
   Y->dims[mode] = R;                      // mode n is replaced by r in place
   Y->attr[0] = COMET_CU; Y->attr[1] = COMET_CU; Y->attr[2] = COMET_D;
@@ -288,7 +288,7 @@ extern "C" comet_status_t comet_ttm_symbolic(comet_handle_t handle, const comet_
   if (st == COMET_OK) {
     Y->pos_len[2] = 1;
     Y->pos[2] = (int32_t *)owned_alloc(ctx, o, 4, s);
-    Y->val = owned_alloc(ctx, o, (size_t)F * R * sizeof(double), s);
+    Y->val = owned_alloc(ctx, o, (size_t)F * R * elem_size(X->dtype), s);
     if (!Y->pos[2] || !Y->val) st = COMET_ERR_ALLOC;
     else {
       set_word_kernel<<<1, 1, 0, s>>>(Y->pos[2], (int32_t)R);
@@ -309,10 +309,11 @@ extern "C" comet_status_t comet_ttm(comet_handle_t handle, const comet_sptensor_
   if (st != COMET_OK) return st;
   const int64_t F = X->crd_len[1];
   if (Y->order != 3 || Y->nnz != F * R || (Y->nnz > 0 && !Y->val)) return COMET_ERR_INVALID_ARG;
-  if (misaligned8(U)) return COMET_ERR_MISALIGNED;
+  if (Y->dtype != X->dtype) return COMET_ERR_INVALID_ARG;
+  if (misaligned(U, X->dtype)) return COMET_ERR_MISALIGNED;
   Context *ctx = reinterpret_cast<Context *>(handle);
-  return seg_gather(ctx, X->pos[2] + 1, X->crd[2], (const double *)X->val, F, X->nnz, (const double *)U, ldu, R,
-                    (double *)Y->val, R, nullptr, F, (cudaStream_t)stream);
+  return seg_gather(ctx, X->dtype, X->pos[2] + 1, X->crd[2], X->val, F, X->nnz, U, ldu, R, Y->val, R, nullptr, F,
+                    (cudaStream_t)stream);
 }
 
 // ------------------------------------------------------------------------------------------ MTTKRP
@@ -326,16 +327,16 @@ extern "C" comet_status_t comet_mttkrp(comet_handle_t handle, const comet_sptens
   if (X->mode_order[0] != mode) return COMET_ERR_UNSUPPORTED_FORMAT;   // re-pack with the output mode first
   const int m1 = X->mode_order[1], m2 = X->mode_order[2];
   if (!h_factors[m1] || !h_factors[m2] || h_ld[m1] < R || h_ld[m2] < R) return COMET_ERR_INVALID_ARG;
-  if (misaligned8(h_factors[m1]) || misaligned8(h_factors[m2]) || misaligned8(out)) return COMET_ERR_MISALIGNED;
+  if (misaligned(h_factors[m1], X->dtype) || misaligned(h_factors[m2], X->dtype) || misaligned(out, X->dtype)) return COMET_ERR_MISALIGNED;
   Context *ctx = reinterpret_cast<Context *>(handle);
   cudaStream_t s = (cudaStream_t)stream;
   const int64_t rows = X->dims[mode];
-  const double *P = (const double *)h_factors[m1], *Q = (const double *)h_factors[m2];
+  const void *P = h_factors[m1], *Q = h_factors[m2];
   if (is_fmt(X, 3, COMET_CN, COMET_S, COMET_S))
-    return mttkrp_coo(ctx, X->crd[0], X->crd[1], X->crd[2], (const double *)X->val, X->nnz, rows, P, h_ld[m1], Q,
-                      h_ld[m2], R, (double *)out, ldo, s);
+    return mttkrp_coo(ctx, X->dtype, X->crd[0], X->crd[1], X->crd[2], X->val, X->nnz, rows, P, h_ld[m1], Q, h_ld[m2], R, out,
+                      ldo, s);
   if (is_fmt(X, 3, COMET_CU, COMET_CU, COMET_CU))
-    return mttkrp_csf(ctx, X->pos[1], X->crd[0], X->crd[1], X->pos[2], X->crd[2], (const double *)X->val,
-                      X->crd_len[0], X->crd_len[1], X->nnz, rows, P, h_ld[m1], Q, h_ld[m2], R, (double *)out, ldo, s);
+    return mttkrp_csf(ctx, X->dtype, X->pos[1], X->crd[0], X->crd[1], X->pos[2], X->crd[2], X->val, X->crd_len[0],
+                      X->crd_len[1], X->nnz, rows, P, h_ld[m1], Q, h_ld[m2], R, out, ldo, s);
   return COMET_ERR_UNSUPPORTED_FORMAT;
 }

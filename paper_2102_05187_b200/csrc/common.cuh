@@ -53,6 +53,7 @@ inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 // operand rows that are re-used out of L2.
 __device__ __forceinline__ int32_t ld_stream(const int32_t *p) { return __ldcs(p); }
 __device__ __forceinline__ double ld_stream(const double *p) { return __ldcs(p); }
+__device__ __forceinline__ float ld_stream(const float *p) { return __ldcs(p); }
 
 // Merge-path split: the merge list interleaves segment-end markers (segment s ends at leaf position
 // seg_end[s]) with the leaf positions 0..N-1; at state (i, j) the next item is leaf j if

@@ -25,10 +25,10 @@ namespace comet {
 struct SegDotArgs {
   const int32_t *seg_end;
   const int32_t *crd;
-  const double *val;
+  const void *val;          // values, vector and output are T (double or float); sums are kept in double
   int64_t M, N;
-  const double *x;
-  double *y;
+  const void *x;
+  void *y;
   const int32_t *out_row;   // NULL: segment s -> y[s]; else y[out_row[s]] (y pre-zeroed by the launcher)
   int64_t num_tiles;
   double *carry_val;
@@ -45,11 +45,12 @@ struct NamedBarrier {          // a barrier over `count` threads of the CTA (a "
 
 // Steps 3 and 4 for a tile whose products and (tile-relative) segment ends are staged in shared memory.
 // `tid` is the thread's index among the THREADS threads that share the tile and the barrier.
-template <int THREADS, int IPT, class Bar>
+template <class T, int THREADS, int IPT, class Bar>
 __device__ __forceinline__ void walk_staged_tile(const SegDotArgs &a, const int32_t *s_end, const double *s_prod,
                                                  int32_t *s_wkey, double *s_wval, int tid, int rows, int nnz,
                                                  int64_t i0, int64_t i1, int64_t tile, Bar bar) {
   constexpr int WARPS = THREADS / 32;
+  T *const y = static_cast<T *>(a.y);
   // thread-level split of the tile's merge list
   const int items = rows + nnz;
   const int t0 = (tid * IPT < items) ? tid * IPT : items;
@@ -74,7 +75,7 @@ __device__ __forceinline__ void walk_staged_tile(const SegDotArgs &a, const int3
         first_val = running;             // completed once the earlier threads' part is known
       } else {
         const int64_t s = i0 + i;
-        a.y[a.out_row ? (int64_t)__ldg(a.out_row + s) : s] = running;
+        y[a.out_row ? (int64_t)__ldg(a.out_row + s) : s] = (T)running;
       }
       running = 0.0;
       ++i;
@@ -120,7 +121,7 @@ __device__ __forceinline__ void walk_staged_tile(const SegDotArgs &a, const int3
   if (have_first) {
     const double carry_in = (tid > 0 && prev_key == first_row) ? prev_sum : 0.0;
     const int64_t s = i0 + first_row;
-    a.y[a.out_row ? (int64_t)__ldg(a.out_row + s) : s] = first_val + carry_in;
+    y[a.out_row ? (int64_t)__ldg(a.out_row + s) : s] = (T)(first_val + carry_in);
   }
   if (tid == THREADS - 1) {
     // key == rows here: the segment the tile stops in
@@ -129,7 +130,7 @@ __device__ __forceinline__ void walk_staged_tile(const SegDotArgs &a, const int3
   }
 }
 
-template <int THREADS, int IPT>
+template <class T, int THREADS, int IPT>
 __global__ void __launch_bounds__(THREADS) seg_dot_kernel(const SegDotArgs a) {
   constexpr int TILE = THREADS * IPT;
   constexpr int WARPS = THREADS / 32;
@@ -153,6 +154,7 @@ __global__ void __launch_bounds__(THREADS) seg_dot_kernel(const SegDotArgs a) {
   const int64_t j0 = d0 - i0, j1 = d1 - i1;
   const int rows = (int)(i1 - i0);       // segment-end markers inside the tile
   const int nnz = (int)(j1 - j0);        // leaf entries inside the tile
+  const T *const val = static_cast<const T *>(a.val), *const x = static_cast<const T *>(a.x);
 
   // Load phase, fully unrolled (a tile holds at most IPT entries and IPT markers per thread): all of a
   // thread's coordinate/value loads are issued before the first dependent vector gather, and all
@@ -164,17 +166,13 @@ __global__ void __launch_bounds__(THREADS) seg_dot_kernel(const SegDotArgs a) {
     for (int k = 0; k < IPT; ++k) {
       const int t = tid + k * THREADS;
       c[k] = 0; v[k] = 0.0; e[k] = 0;
-      if (t < nnz) { c[k] = ld_stream(a.crd + j0 + t); v[k] = ld_stream(a.val + j0 + t); }
+      if (t < nnz) { c[k] = ld_stream(a.crd + j0 + t); v[k] = (double)ld_stream(val + j0 + t); }
       if (t < rows) e[k] = __ldg(a.seg_end + i0 + t);
     }
 #pragma unroll
     for (int k = 0; k < IPT; ++k) {
       const int t = tid + k * THREADS;
-#ifdef EXP_NOGATHER
-      if (t < nnz) v[k] *= __ldg(a.x + (c[k] & 1));
-#else
-      if (t < nnz) v[k] *= __ldg(a.x + c[k]);
-#endif
+      if (t < nnz) v[k] *= (double)__ldg(x + c[k]);
     }
 #pragma unroll
     for (int k = 0; k < IPT; ++k) {
@@ -185,7 +183,7 @@ __global__ void __launch_bounds__(THREADS) seg_dot_kernel(const SegDotArgs a) {
   }
   __syncthreads();
 
-  walk_staged_tile<THREADS, IPT>(a, s_end, s_prod, s_wkey, s_wval, tid, rows, nnz, i0, i1, tile, BlockBarrier());
+  walk_staged_tile<T, THREADS, IPT>(a, s_end, s_prod, s_wkey, s_wval, tid, rows, nnz, i0, i1, tile, BlockBarrier());
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -217,14 +215,15 @@ template <int THREADS, int IPT> struct ResidentLayout {
   static constexpr int kStageBytes = kProdBytes + kEndBytes + kScanBytes;    // multiple of 16
 };
 
-template <int VC, int THREADS, int IPT>
+template <class T, int VC, int THREADS, int IPT>
 __global__ void __launch_bounds__(VC *THREADS, 1)
 seg_dot_resident_kernel(const SegDotArgs a, const int32_t *__restrict__ splits, int64_t x_len, int32_t x_bytes_padded) {
   using RL = ResidentLayout<THREADS, IPT>;
   constexpr int TILE = RL::TILE;
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  double *s_x = reinterpret_cast<double *>(smem_raw);
-  for (int64_t i = threadIdx.x; i < x_len; i += VC * THREADS) s_x[i] = __ldg(a.x + i);
+  T *s_x = reinterpret_cast<T *>(smem_raw);
+  const T *const val = static_cast<const T *>(a.val), *const x = static_cast<const T *>(a.x);
+  for (int64_t i = threadIdx.x; i < x_len; i += VC * THREADS) s_x[i] = __ldg(x + i);
   __syncthreads();
 
   const int vc = threadIdx.x / THREADS, tid = threadIdx.x % THREADS;
@@ -257,7 +256,7 @@ seg_dot_resident_kernel(const SegDotArgs a, const int32_t *__restrict__ splits, 
     for (int k = 0; k < IPT; ++k) {
       const int tt = tid + k * THREADS;
       c[k] = 0; v[k] = 0.0; e[k] = 0;
-      if (tt < f_nnz) { c[k] = ld_stream(a.crd + f_j0 + tt); v[k] = ld_stream(a.val + f_j0 + tt); }
+      if (tt < f_nnz) { c[k] = ld_stream(a.crd + f_j0 + tt); v[k] = (double)ld_stream(val + f_j0 + tt); }
       if (tt < f_rows) e[k] = __ldg(a.seg_end + f_i0 + tt);
     }
   };
@@ -272,14 +271,14 @@ seg_dot_resident_kernel(const SegDotArgs a, const int32_t *__restrict__ splits, 
 #pragma unroll
     for (int k = 0; k < IPT; ++k) {
       const int tt = tid + k * THREADS;
-      if (tt < nnz) s_prod[tt] = v[k] * s_x[c[k]];
+      if (tt < nnz) s_prod[tt] = v[k] * (double)s_x[c[k]];
       if (tt < rows) s_end[tt] = (int32_t)((int64_t)e[k] - j0);
     }
     // the next tile's loads fly while this one is walked; its successor's boundaries follow
     if (t + stride < a.num_tiles) fetch(t + stride, n_i0, n_i1);
     if (t + 2 * stride < a.num_tiles) { n_i0 = __ldg(splits + t + 2 * stride); n_i1 = __ldg(splits + t + 2 * stride + 1); }
     bar();
-    walk_staged_tile<THREADS, IPT>(a, s_end, s_prod, s_wkey, s_wval, tid, rows, nnz, i0, i1, t, bar);
+    walk_staged_tile<T, THREADS, IPT>(a, s_end, s_prod, s_wkey, s_wval, tid, rows, nnz, i0, i1, t, bar);
     bar();                                               // the staging area may be overwritten
   }
 }
@@ -294,19 +293,21 @@ seg_dot_resident_kernel(const SegDotArgs a, const int32_t *__restrict__ splits, 
 // REDUX.OR; a lane that owns a closing segment fetches that segment's sum from the lane holding its last
 // entry. Segments are closed by the span that holds their last entry; the open partial of a span goes to
 // a carry slot as in the other kernels (deterministic, no atomics).
-template <bool XSMEM>
+template <class T, bool XSMEM>
 __global__ void __launch_bounds__(1024, 1)
 seg_dot_stream_kernel(const SegDotArgs a, int64_t x_len, int32_t span, unsigned long long *next_tile) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  const double *s_x = reinterpret_cast<const double *>(smem_raw);
+  const T *s_x = reinterpret_cast<const T *>(smem_raw);
+  const T *const val = static_cast<const T *>(a.val), *const x = static_cast<const T *>(a.x);
+  T *const y = static_cast<T *>(a.y);
   if (XSMEM) {
-    double *w = reinterpret_cast<double *>(smem_raw);
-    for (int64_t i = threadIdx.x; i < x_len; i += blockDim.x) w[i] = __ldg(a.x + i);
+    T *w = reinterpret_cast<T *>(smem_raw);
+    for (int64_t i = threadIdx.x; i < x_len; i += blockDim.x) w[i] = __ldg(x + i);
     __syncthreads();
   }
   const unsigned full = 0xffffffffu;
   const int lane = threadIdx.x & 31;
-  auto xval = [&](int32_t c) -> double { return XSMEM ? s_x[c] : __ldg(a.x + c); };
+  auto xval = [&](int32_t c) -> double { return XSMEM ? (double)s_x[c] : (double)__ldg(x + c); };
   auto warp_sum = [&](double v) -> double {
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(full, v, off);
@@ -337,7 +338,7 @@ seg_dot_stream_kernel(const SegDotArgs a, int64_t x_len, int32_t span, unsigned 
     }
     int64_t s = lo;
     if (tile == 0)                                       // leading empty segments (end == 0) belong to nobody else
-      for (int64_t q = lane; q < s; q += 32) a.y[a.out_row ? (int64_t)__ldg(a.out_row + q) : q] = 0.0;
+      for (int64_t q = lane; q < s; q += 32) y[a.out_row ? (int64_t)__ldg(a.out_row + q) : q] = (T)0;
 
     int32_t ew = (s + lane < a.M) ? __ldg(a.seg_end + s + lane) : 0x7fffffff;   // ends of the next 32 segments
     int32_t last_end = w0;                               // end of the most recently closed segment
@@ -350,7 +351,7 @@ seg_dot_stream_kernel(const SegDotArgs a, int64_t x_len, int32_t span, unsigned 
       for (int u = 0; u < 4; ++u) {
         const int32_t jj = j0 + u * 32 + lane;
         c[u] = 0; v[u] = 0.0;
-        if (whole || jj < w1) { c[u] = ld_stream(a.crd + jj); v[u] = ld_stream(a.val + jj); }
+        if (whole || jj < w1) { c[u] = ld_stream(a.crd + jj); v[u] = (double)ld_stream(val + jj); }
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
@@ -387,14 +388,14 @@ seg_dot_stream_kernel(const SegDotArgs a, int64_t x_len, int32_t span, unsigned 
           const unsigned cm = __ballot_sync(full, closing);
           if (cm == 0) break;
           const int src = closing ? ew - j - 1 : 0;
-          double val = __shfl_sync(full, sc, src);
+          double segsum = __shfl_sync(full, sc, src);
           int32_t prev = __shfl_up_sync(full, ew, 1);
           if (lane == 0) prev = last_end;
           if (closing) {
-            if (ew == prev) val = 0.0;                   // an empty segment: its end repeats its predecessor's
-            else if (src == firstb) val += tot;
+            if (ew == prev) segsum = 0.0;                // an empty segment: its end repeats its predecessor's
+            else if (src == firstb) segsum += tot;
             const int64_t seg = s + lane;
-            a.y[a.out_row ? (int64_t)__ldg(a.out_row + seg) : seg] = val;
+            y[a.out_row ? (int64_t)__ldg(a.out_row + seg) : seg] = (T)segsum;
           }
           const int k = __popc(cm);                      // closing lanes are a prefix: ends are sorted
           last_end = __shfl_sync(full, ew, k - 1);
@@ -411,7 +412,7 @@ seg_dot_stream_kernel(const SegDotArgs a, int64_t x_len, int32_t span, unsigned 
   }
 }
 
-template <int THREADS, int IPT>
+template <class T, int THREADS, int IPT>
 static comet_status_t launch_dot(Context *ctx, SegDotArgs a, cudaStream_t stream) {
   const int64_t total = a.M + a.N;
   a.num_tiles = ceil_div(total, (int64_t)THREADS * IPT);
@@ -421,11 +422,11 @@ static comet_status_t launch_dot(Context *ctx, SegDotArgs a, cudaStream_t stream
   if (!scratch) return COMET_ERR_ALLOC;
   a.carry_val = (double *)scratch;
   a.carry_seg = (int32_t *)(scratch + val_bytes);
-  seg_dot_kernel<THREADS, IPT><<<(unsigned)a.num_tiles, THREADS, 0, stream>>>(a);
+  seg_dot_kernel<T, THREADS, IPT><<<(unsigned)a.num_tiles, THREADS, 0, stream>>>(a);
   COMET_LAUNCH_CHECK(ctx);
   if (a.num_tiles > 1) {
-    carry_fixup_kernel<<<(unsigned)ceil_div(a.num_tiles, 256), 256, 0, stream>>>(
-        a.carry_val, a.carry_seg, a.num_tiles, 1, 1, a.y, 1, a.out_row);
+    carry_fixup_launch(sizeof(T) == 4 ? COMET_F32 : COMET_F64, a.carry_val, a.carry_seg, a.num_tiles, 1, 1, a.y, 1,
+                       a.out_row, stream);
     COMET_LAUNCH_CHECK(ctx);
   }
   return COMET_OK;
@@ -439,6 +440,7 @@ static comet_status_t launch_dot(Context *ctx, SegDotArgs a, cudaStream_t stream
 constexpr int kResVC = COMET_RES_VC, kResThreads = COMET_RES_THREADS, kResIpt = COMET_RES_IPT;
 constexpr size_t kMaxDynamicSmem = 232448;               // 227 KB opt-in limit per CTA on sm_100
 
+template <class T>
 static comet_status_t launch_resident(Context *ctx, SegDotArgs a, int64_t x_len, cudaStream_t stream) {
   using RL = ResidentLayout<kResThreads, kResIpt>;
   const int64_t total = a.M + a.N;
@@ -454,21 +456,22 @@ static comet_status_t launch_resident(Context *ctx, SegDotArgs a, int64_t x_len,
   tile_split_kernel<<<(unsigned)ceil_div((a.num_tiles + 1) * 32, 256), 256, 0, stream>>>(a.seg_end, a.M, a.N, RL::TILE,
                                                                                        a.num_tiles, splits);
   COMET_LAUNCH_CHECK(ctx);
-  const int32_t x_bytes = (int32_t)align_up((size_t)x_len * 8, 16);
+  const int32_t x_bytes = (int32_t)align_up((size_t)x_len * sizeof(T), 16);
   const size_t smem = (size_t)x_bytes + (size_t)kResVC * RL::kStageBytes;
-  auto kernel = seg_dot_resident_kernel<kResVC, kResThreads, kResIpt>;
+  auto kernel = seg_dot_resident_kernel<T, kResVC, kResThreads, kResIpt>;
   COMET_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   const int64_t ctas = ceil_div(a.num_tiles, kResVC) < kSmCount ? ceil_div(a.num_tiles, kResVC) : kSmCount;
   kernel<<<(unsigned)ctas, kResVC * kResThreads, smem, stream>>>(a, splits, x_len, x_bytes);
   COMET_LAUNCH_CHECK(ctx);
-  carry_fixup_kernel<<<(unsigned)ceil_div(a.num_tiles, 256), 256, 0, stream>>>(a.carry_val, a.carry_seg, a.num_tiles, 1,
-                                                                              1, a.y, 1, a.out_row);
+  carry_fixup_launch(sizeof(T) == 4 ? COMET_F32 : COMET_F64, a.carry_val, a.carry_seg, a.num_tiles, 1, 1, a.y, 1,
+                     a.out_row, stream);
   COMET_LAUNCH_CHECK(ctx);
   return COMET_OK;
 }
 
+template <class T>
 static comet_status_t launch_stream(Context *ctx, SegDotArgs a, int64_t x_len, cudaStream_t stream) {
-  const size_t x_bytes = align_up((size_t)x_len * 8, 16);
+  const size_t x_bytes = align_up((size_t)x_len * sizeof(T), 16);
   const bool xsmem = x_bytes <= kMaxDynamicSmem - 1024;
   // spans: a multiple of 128 entries, several per warp of the 148 persistent CTAs so that the tail is short
   const int64_t warps = (int64_t)kSmCount * 32;
@@ -487,24 +490,25 @@ static comet_status_t launch_stream(Context *ctx, SegDotArgs a, int64_t x_len, c
   COMET_CUDA_TRY(ctx, cudaMemsetAsync(next_tile, 0, sizeof(unsigned long long), stream));
   const int64_t ctas = ceil_div(a.num_tiles, 32) < kSmCount ? ceil_div(a.num_tiles, 32) : kSmCount;
   if (xsmem) {
-    auto kernel = seg_dot_stream_kernel<true>;
+    auto kernel = seg_dot_stream_kernel<T, true>;
     COMET_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)x_bytes));
     kernel<<<(unsigned)ctas, 1024, x_bytes, stream>>>(a, x_len, (int32_t)span, next_tile);
   } else {
-    seg_dot_stream_kernel<false><<<(unsigned)ctas, 1024, 0, stream>>>(a, x_len, (int32_t)span, next_tile);
+    seg_dot_stream_kernel<T, false><<<(unsigned)ctas, 1024, 0, stream>>>(a, x_len, (int32_t)span, next_tile);
   }
   COMET_LAUNCH_CHECK(ctx);
-  carry_fixup_kernel<<<(unsigned)ceil_div(a.num_tiles, 256), 256, 0, stream>>>(a.carry_val, a.carry_seg, a.num_tiles, 1,
-                                                                              1, a.y, 1, a.out_row);
+  carry_fixup_launch(sizeof(T) == 4 ? COMET_F32 : COMET_F64, a.carry_val, a.carry_seg, a.num_tiles, 1, 1, a.y, 1,
+                     a.out_row, stream);
   COMET_LAUNCH_CHECK(ctx);
   return COMET_OK;
 }
 
-comet_status_t seg_dot(Context *ctx, const int32_t *seg_end, const int32_t *crd, const double *val, int64_t M,
-                       int64_t N, const double *x, int64_t x_len, double *y, const int32_t *out_row,
-                       int64_t out_rows, cudaStream_t stream) {
+template <class T>
+static comet_status_t seg_dot_typed(Context *ctx, int dtype, const int32_t *seg_end, const int32_t *crd, const void *val,
+                                    int64_t M, int64_t N, const void *x, int64_t x_len, void *y, const int32_t *out_row,
+                                    int64_t out_rows, cudaStream_t stream) {
   if (out_row) {
-    comet_status_t st = zero_rows(ctx, y, out_rows, 1, 1, stream);
+    comet_status_t st = zero_rows(ctx, y, dtype, out_rows, 1, 1, stream);
     if (st != COMET_OK) return st;
   }
   if (M == 0) return COMET_OK;
@@ -514,22 +518,30 @@ comet_status_t seg_dot(Context *ctx, const int32_t *seg_end, const int32_t *crd,
   {
     const char *force = getenv("COMET_SEG_DOT_KERNEL");   // tests: "stream", "resident" or "tile" on any input
     const bool want_stream = force ? !strcmp(force, "stream") : (N >= (int64_t)kSmCount * 32 * 512 && N > 0);
-    if (want_stream && N > 0) return launch_stream(ctx, a, x_len, stream);
+    if (want_stream && N > 0) return launch_stream<T>(ctx, a, x_len, stream);
   }
   // Mid-size problems whose vector fits in shared memory beside the staging: persistent CTAs, x resident.
   {
     using RL = ResidentLayout<kResThreads, kResIpt>;
-    const size_t need = align_up((size_t)x_len * 8, 16) + (size_t)kResVC * RL::kStageBytes;
+    const size_t need = align_up((size_t)x_len * sizeof(T), 16) + (size_t)kResVC * RL::kStageBytes;
     const char *force = getenv("COMET_SEG_DOT_KERNEL");
     const bool forced = force && !strcmp(force, "resident");
     if (need <= kMaxDynamicSmem && (forced || M + N >= (int64_t)kSmCount * kResVC * RL::TILE * 8))
-      return launch_resident(ctx, a, x_len, stream);
+      return launch_resident<T>(ctx, a, x_len, stream);
   }
   // Items per thread are odd so that the per-thread walks (stride IPT doubles across lanes) hit all
   // shared-memory banks; an even stride of 8 serialises them 16 ways. Small problems get short tiles so
   // that the grid still covers the 148 SMs.
-  if (M + N < (int64_t)kSmCount * 2048 * 2) return launch_dot<128, 5>(ctx, a, stream);
-  return launch_dot<256, 9>(ctx, a, stream);
+  if (M + N < (int64_t)kSmCount * 2048 * 2) return launch_dot<T, 128, 5>(ctx, a, stream);
+  return launch_dot<T, 256, 9>(ctx, a, stream);
+}
+
+comet_status_t seg_dot(Context *ctx, int dtype, const int32_t *seg_end, const int32_t *crd, const void *val, int64_t M,
+                       int64_t N, const void *x, int64_t x_len, void *y, const int32_t *out_row, int64_t out_rows,
+                       cudaStream_t stream) {
+  if (dtype == COMET_F32)
+    return seg_dot_typed<float>(ctx, dtype, seg_end, crd, val, M, N, x, x_len, y, out_row, out_rows, stream);
+  return seg_dot_typed<double>(ctx, dtype, seg_end, crd, val, M, N, x, x_len, y, out_row, out_rows, stream);
 }
 
 }  // namespace comet
@@ -594,16 +606,15 @@ extern "C" comet_status_t comet_spmv_static(const comet_sptensor_t *A, const voi
   if (st != COMET_OK) return st;
 
   SegDotArgs a{};
-  a.seg_end = A->pos[1] + 1; a.crd = A->crd[1]; a.val = (const double *)A->val;
-  a.M = M; a.N = N; a.x = (const double *)x; a.y = (double *)y; a.out_row = nullptr;
+  a.seg_end = A->pos[1] + 1; a.crd = A->crd[1]; a.val = A->val;
+  a.M = M; a.N = N; a.x = x; a.y = y; a.out_row = nullptr;
   a.num_tiles = ceil_div(M + N, (int64_t)kStaticThreads * kStaticIpt);
   a.carry_val = (double *)scratch;                               // every tile writes its slot before the
   a.carry_seg = (int32_t *)((char *)scratch + kStaticValBytes);  // fix-up reads it: nothing to clear
   cudaStream_t s = (cudaStream_t)stream;
-  seg_dot_kernel<kStaticThreads, kStaticIpt><<<(unsigned)a.num_tiles, kStaticThreads, 0, s>>>(a);
+  seg_dot_kernel<double, kStaticThreads, kStaticIpt><<<(unsigned)a.num_tiles, kStaticThreads, 0, s>>>(a);
   if (a.num_tiles > 1)
-    carry_fixup_kernel<<<(unsigned)ceil_div(a.num_tiles, 256), 256, 0, s>>>(a.carry_val, a.carry_seg, a.num_tiles, 1, 1,
-                                                                            a.y, 1, nullptr);
+    carry_fixup_launch(COMET_F64, a.carry_val, a.carry_seg, a.num_tiles, 1, 1, y, 1, nullptr, s);
   if (cudaGetLastError() != cudaSuccess) return COMET_ERR_CUDA;
   return COMET_OK;
 }

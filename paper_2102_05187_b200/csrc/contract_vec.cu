@@ -25,11 +25,11 @@ namespace comet {
 struct SegGatherArgs {
   const int32_t *seg_end;   // M entries: leaf position where segment s ends (= pos + 1)
   const int32_t *crd;       // N leaf coordinates (row index into B)
-  const double *val;        // N values
+  const void *val;          // N values (T)
   int64_t M, N;
-  const double *B;
+  const void *B;            // dense operand (T), already offset to this launch's first column
   int64_t ldb;
-  double *C;                // output rows
+  void *C;                  // output rows (T), already offset to this launch's first column
   int64_t ldc;
   const int32_t *out_row;   // NULL: segment s -> row s. Else segment s -> row out_row[s] (ascending) and the
   int64_t out_rows;         //   rows in between (and up to out_rows) are zero-filled by the flushing worker
@@ -42,20 +42,22 @@ struct SegGatherArgs {
 };
 
 // What the walker does with one leaf entry: close the segments that end in front of it, accumulate.
-template <int LPN, int CPL, int VEC, bool MAPPED>
+template <class T, int LPN, int CPL, int VEC, bool MAPPED>
 struct SegGatherPolicy {
-  using L = Lanes<LPN, CPL, VEC>;
+  using L = Lanes<T, LPN, CPL, VEC>;
   static constexpr int kPF = COMET_PF_GATHER;
   static constexpr bool kAux = false;
   static constexpr bool kFullUnroll = true;
-  struct Slot { double r[CPL][VEC]; };
+  struct Slot { T r[CPL][VEC]; };
 
   const SegGatherArgs &a;
   const L &ln;
+  const T *val;
+  T *cmat;                  // this lane's piece 0 of row 0 of C
   const char *bcol;         // this lane's piece 0 of row 0 of B
   int32_t ldb_bytes;
   double acc[CPL][VEC];
-  double *out;              // this lane's piece 0 of the open segment's output row (identity mapping)
+  T *out;                   // this lane's piece 0 of the open segment's output row (identity mapping)
   const int32_t *endp;      // seg_end + open segment
   int32_t segs_left;        // segments from the open one to the last
   int32_t next_end;         // leaf position where the open segment ends (-1: no segment left)
@@ -65,9 +67,11 @@ struct SegGatherPolicy {
   __device__ __forceinline__ SegGatherPolicy(const SegGatherArgs &args, const L &lanes, int64_t i0, int32_t j0)
       : a(args), ln(lanes), base(j0), last_flush(j0) {
     ln.zero(acc);
-    bcol = reinterpret_cast<const char *>(a.B + ln.col0);
-    ldb_bytes = (int32_t)(a.ldb * 8);
-    out = a.C + i0 * a.ldc + ln.col0;
+    val = static_cast<const T *>(a.val);
+    bcol = reinterpret_cast<const char *>(static_cast<const T *>(a.B) + ln.col0);
+    ldb_bytes = (int32_t)(a.ldb * sizeof(T));
+    cmat = static_cast<T *>(a.C) + ln.col0;
+    out = cmat + i0 * a.ldc;
     endp = a.seg_end + i0;
     segs_left = (int32_t)(a.M - i0);
     next_end = segs_left > 0 ? __ldg(endp) : -1;
@@ -75,11 +79,11 @@ struct SegGatherPolicy {
   }
   __device__ __forceinline__ int64_t segment() const { return a.M - segs_left; }
   __device__ __forceinline__ void fetch(int32_t j, Entry16 &e, int32_t &) const {
-    e.v = ld_stream(a.val + j);
+    e.v = (double)ld_stream(val + j);
     e.a = ld_stream(a.crd + j);
   }
   __device__ __forceinline__ void prefetch(int32_t c, int32_t, Slot &s) const {
-    ln.gather(reinterpret_cast<const double *>(bcol + (int64_t)c * ldb_bytes), s.r);
+    ln.gather(reinterpret_cast<const T *>(bcol + (int64_t)c * ldb_bytes), s.r);
   }
   __device__ __forceinline__ void begin_chunk(int32_t b) { base = b; rel_end = next_end - b; }
 
@@ -89,10 +93,9 @@ struct SegGatherPolicy {
       const int64_t i = segment();
       const int64_t r = __ldg(a.out_row + i);
       const int64_t lo = (i > 0) ? (int64_t)__ldg(a.out_row + i - 1) + 1 : 0;
-      double *c0 = a.C + ln.col0;
-      ln.zero_rows(c0, a.ldc, lo, r);
-      if (i == a.M - 1) ln.zero_rows(c0, a.ldc, r + 1, a.out_rows);
-      ln.store_row(c0 + r * a.ldc, acc);
+      ln.zero_rows(cmat, a.ldc, lo, r);
+      if (i == a.M - 1) ln.zero_rows(cmat, a.ldc, r + 1, a.out_rows);
+      ln.store_row(cmat + r * a.ldc, acc);
     } else {
       ln.store_row(out, acc);
       out += a.ldc;
@@ -110,10 +113,10 @@ struct SegGatherPolicy {
   }
 };
 
-template <int LPN, int CPL, int VEC, bool MAPPED>
-__global__ void __launch_bounds__(kBlockThreads, (CPL * VEC <= 2 ? COMET_MINB_GATHER : 2))
+template <class T, int LPN, int CPL, int VEC, bool MAPPED>
+__global__ void __launch_bounds__(kBlockThreads, (CPL * VEC * sizeof(T) <= 16 ? COMET_MINB_GATHER : 2))
 seg_gather_kernel(const SegGatherArgs a) {
-  using L = Lanes<LPN, CPL, VEC>;
+  using L = Lanes<T, LPN, CPL, VEC>;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int worker = threadIdx.x / LPN;
   const int64_t tile = (int64_t)blockIdx.x * L::kWorkers + worker;
@@ -128,7 +131,7 @@ seg_gather_kernel(const SegGatherArgs a) {
   const int64_t i1 = merge_path_segments_coop<LPN>(a.seg_end, a.M, a.N, d1, ln.g, ln.mask);
   const int32_t j0 = (int32_t)(d0 - i0), j1 = (int32_t)(d1 - i1);
 
-  SegGatherPolicy<LPN, CPL, VEC, MAPPED> p(a, ln, i0, j0);
+  SegGatherPolicy<T, LPN, CPL, VEC, MAPPED> p(a, ln, i0, j0);
   walk_tile(ln, p, j0, j1, smem);
   while (p.segment() < i1) p.flush(j1);                  // end markers that close the tile
 
@@ -140,8 +143,9 @@ seg_gather_kernel(const SegGatherArgs a) {
 
 // Adds the carries onto the stored rows. Tiles that stopped inside the same segment are consecutive;
 // the first of such a run sums the run in tile order and updates the row (the only writer of it now).
+template <class T>
 __global__ void carry_fixup_kernel(const double *__restrict__ carry_val, const int32_t *__restrict__ carry_seg,
-                                   int64_t num_tiles, int32_t R, int32_t carry_ld, double *__restrict__ C,
+                                   int64_t num_tiles, int32_t R, int32_t carry_ld, T *__restrict__ C,
                                    int64_t ldc, const int32_t *__restrict__ out_row) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t tile = idx / R;
@@ -153,19 +157,30 @@ __global__ void carry_fixup_kernel(const double *__restrict__ carry_val, const i
   double sum = 0.0;
   for (int64_t t = tile; t < num_tiles && carry_seg[t] == seg; ++t) sum += carry_val[t * carry_ld + c];
   const int64_t row = out_row ? (int64_t)out_row[seg] : (int64_t)seg;
-  C[row * ldc + c] += sum;
+  C[row * ldc + c] = (T)((double)C[row * ldc + c] + sum);
 }
 
-__global__ void zero_rows_kernel(double *__restrict__ C, int64_t rows, int32_t R, int64_t ldc) {
+void carry_fixup_launch(int dtype, const double *carry_val, const int32_t *carry_seg, int64_t num_tiles, int32_t R,
+                        int32_t carry_ld, void *C, int64_t ldc, const int32_t *out_row, cudaStream_t stream) {
+  const unsigned blocks = (unsigned)ceil_div(num_tiles * R, 256);
+  if (dtype == COMET_F32)
+    carry_fixup_kernel<float><<<blocks, 256, 0, stream>>>(carry_val, carry_seg, num_tiles, R, carry_ld, (float *)C, ldc, out_row);
+  else
+    carry_fixup_kernel<double><<<blocks, 256, 0, stream>>>(carry_val, carry_seg, num_tiles, R, carry_ld, (double *)C, ldc, out_row);
+}
+
+template <class T>
+__global__ void zero_rows_kernel(T *__restrict__ C, int64_t rows, int32_t R, int64_t ldc) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t r = idx / R;
-  if (r < rows) C[r * ldc + (idx - r * R)] = 0.0;
+  if (r < rows) C[r * ldc + (idx - r * R)] = (T)0;
 }
 
-comet_status_t zero_rows(Context *ctx, double *C, int64_t rows, int64_t R, int64_t ldc, cudaStream_t stream) {
+comet_status_t zero_rows(Context *ctx, void *C, int dtype, int64_t rows, int64_t R, int64_t ldc, cudaStream_t stream) {
   if (rows <= 0 || R <= 0) return COMET_OK;
   const int64_t n = rows * R;
-  zero_rows_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, stream>>>(C, rows, (int32_t)R, ldc);
+  if (dtype == COMET_F32) zero_rows_kernel<float><<<(unsigned)ceil_div(n, 256), 256, 0, stream>>>((float *)C, rows, (int32_t)R, ldc);
+  else zero_rows_kernel<double><<<(unsigned)ceil_div(n, 256), 256, 0, stream>>>((double *)C, rows, (int32_t)R, ldc);
   COMET_LAUNCH_CHECK(ctx);
   return COMET_OK;
 }
@@ -184,11 +199,11 @@ int32_t choose_tile_items(int64_t total_items, int workers_per_block) {
   return (int32_t)t;
 }
 
-template <int LPN, int CPL, int VEC, bool MAPPED>
+template <class T, int LPN, int CPL, int VEC, bool MAPPED>
 static comet_status_t launch_mapped(Context *ctx, const SegGatherArgs &a, int64_t blocks, cudaStream_t stream) {
-  using L = Lanes<LPN, CPL, VEC>;
+  using L = Lanes<T, LPN, CPL, VEC>;
   constexpr size_t smem = RingLayout<L, false>::kBlockBytes;
-  auto kernel = seg_gather_kernel<LPN, CPL, VEC, MAPPED>;
+  auto kernel = seg_gather_kernel<T, LPN, CPL, VEC, MAPPED>;
   if (smem > 48 * 1024)
     COMET_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   kernel<<<(unsigned)blocks, kBlockThreads, smem, stream>>>(a);
@@ -196,7 +211,7 @@ static comet_status_t launch_mapped(Context *ctx, const SegGatherArgs &a, int64_
   return COMET_OK;
 }
 
-template <int LPN, int CPL, int VEC>
+template <class T, int LPN, int CPL, int VEC>
 static comet_status_t launch_one(Context *ctx, SegGatherArgs a, cudaStream_t stream) {
   constexpr int WORKERS = kBlockThreads / LPN;
   const int64_t total = a.M + a.N;
@@ -210,51 +225,63 @@ static comet_status_t launch_one(Context *ctx, SegGatherArgs a, cudaStream_t str
   a.carry_val = (double *)scratch;
   a.carry_seg = (int32_t *)(scratch + val_bytes);
   const int64_t blocks = ceil_div(a.num_tiles, WORKERS);
-  comet_status_t st = a.out_row ? launch_mapped<LPN, CPL, VEC, true>(ctx, a, blocks, stream)
-                                : launch_mapped<LPN, CPL, VEC, false>(ctx, a, blocks, stream);
+  comet_status_t st = a.out_row ? launch_mapped<T, LPN, CPL, VEC, true>(ctx, a, blocks, stream)
+                                : launch_mapped<T, LPN, CPL, VEC, false>(ctx, a, blocks, stream);
   if (st != COMET_OK) return st;
-  const int64_t fix_threads = a.num_tiles * a.R;
-  carry_fixup_kernel<<<(unsigned)ceil_div(fix_threads, 256), 256, 0, stream>>>(
-      a.carry_val, a.carry_seg, a.num_tiles, a.R, a.carry_ld, a.C, a.ldc, a.out_row);
+  carry_fixup_launch(sizeof(T) == 4 ? COMET_F32 : COMET_F64, a.carry_val, a.carry_seg, a.num_tiles, a.R, a.carry_ld, a.C,
+                     a.ldc, a.out_row, stream);
   COMET_LAUNCH_CHECK(ctx);
   return COMET_OK;
 }
 
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
-comet_status_t seg_gather(Context *ctx, const int32_t *seg_end, const int32_t *crd, const double *val, int64_t M,
-                          int64_t N, const double *B, int64_t ldb, int64_t R, double *C, int64_t ldc,
-                          const int32_t *out_row, int64_t out_rows, cudaStream_t stream) {
-  if (ldb >= (1ll << 28)) return COMET_ERR_INDEX_OVERFLOW;      // row offsets are formed as int32 bytes * int32 index
-  if (M == 0) return out_row ? zero_rows(ctx, C, out_rows, R, ldc, stream) : COMET_OK;
-  const bool vec_ok = aligned16(B) && aligned16(C) && (ldb % 2 == 0) && (ldc % 2 == 0);
+// One launch per chunk of up to 128 columns. A power-of-two chunk on 16-byte-aligned rows takes the
+// 128-bit path (LPN lanes x 16 bytes); anything else takes the scalar path (32 lanes, ragged).
+template <class T>
+static comet_status_t seg_gather_typed(Context *ctx, const int32_t *seg_end, const int32_t *crd, const T *val,
+                                       int64_t M, int64_t N, const T *B, int64_t ldb, int64_t R, T *C, int64_t ldc,
+                                       const int32_t *out_row, int64_t out_rows, cudaStream_t stream) {
+  constexpr int PER = 16 / sizeof(T);                      // elements per 128-bit piece
+  const bool vec_ok = aligned16(B) && aligned16(C) && (ldb % PER == 0) && (ldc % PER == 0);
   int64_t done = 0;
   while (done < R) {
-    int64_t rem = R - done;
+    const int64_t rem = R - done;
     SegGatherArgs a{};
     a.seg_end = seg_end; a.crd = crd; a.val = val; a.M = M; a.N = N;
     a.B = B + done; a.ldb = ldb; a.C = C + done; a.ldc = ldc;
     a.out_row = out_row; a.out_rows = out_rows;
     comet_status_t st;
-    // One launch per chunk of up to 128 columns. A power-of-two chunk on 16-byte-aligned rows takes the
-    // 128-bit path (LPN lanes x 2 columns); anything else takes the scalar path (32 lanes, ragged).
     const int64_t chunk = rem < 128 ? rem : 128;
     a.R = (int32_t)chunk;
-    const bool v = vec_ok && done % 2 == 0;
-    if (v && chunk == 128) st = launch_one<32, 2, 2>(ctx, a, stream);
-    else if (v && chunk == 64) st = launch_one<32, 1, 2>(ctx, a, stream);
-    else if (v && chunk == 32) st = launch_one<16, 1, 2>(ctx, a, stream);
-    else if (v && chunk == 16) st = launch_one<8, 1, 2>(ctx, a, stream);
-    else if (v && chunk == 8) st = launch_one<4, 1, 2>(ctx, a, stream);
-    else if (v && chunk == 4) st = launch_one<2, 1, 2>(ctx, a, stream);
-    else if (v && chunk == 2) st = launch_one<1, 1, 2>(ctx, a, stream);
-    else if (chunk > 64) st = launch_one<32, 4, 1>(ctx, a, stream);
-    else if (chunk > 32) st = launch_one<32, 2, 1>(ctx, a, stream);
-    else st = launch_one<32, 1, 1>(ctx, a, stream);
+    const bool v = vec_ok && done % PER == 0;
+    const int64_t pieces = chunk / PER;                    // 128-bit pieces per row when chunk is a multiple
+    if (v && chunk % PER == 0 && pieces == 64) st = launch_one<T, 32, 2, PER>(ctx, a, stream);
+    else if (v && chunk % PER == 0 && pieces == 32) st = launch_one<T, 32, 1, PER>(ctx, a, stream);
+    else if (v && chunk % PER == 0 && pieces == 16) st = launch_one<T, 16, 1, PER>(ctx, a, stream);
+    else if (v && chunk % PER == 0 && pieces == 8) st = launch_one<T, 8, 1, PER>(ctx, a, stream);
+    else if (v && chunk % PER == 0 && pieces == 4) st = launch_one<T, 4, 1, PER>(ctx, a, stream);
+    else if (v && chunk % PER == 0 && pieces == 2) st = launch_one<T, 2, 1, PER>(ctx, a, stream);
+    else if (v && chunk % PER == 0 && pieces == 1) st = launch_one<T, 1, 1, PER>(ctx, a, stream);
+    else if (chunk > 64) st = launch_one<T, 32, 4, 1>(ctx, a, stream);
+    else if (chunk > 32) st = launch_one<T, 32, 2, 1>(ctx, a, stream);
+    else st = launch_one<T, 32, 1, 1>(ctx, a, stream);
     if (st != COMET_OK) return st;
     done += a.R;
   }
   return COMET_OK;
+}
+
+comet_status_t seg_gather(Context *ctx, int dtype, const int32_t *seg_end, const int32_t *crd, const void *val,
+                          int64_t M, int64_t N, const void *B, int64_t ldb, int64_t R, void *C, int64_t ldc,
+                          const int32_t *out_row, int64_t out_rows, cudaStream_t stream) {
+  if (ldb >= (1ll << 28)) return COMET_ERR_INDEX_OVERFLOW;      // row offsets are formed as int32 bytes * int32 index
+  if (M == 0) return out_row ? zero_rows(ctx, C, dtype, out_rows, R, ldc, stream) : COMET_OK;
+  if (dtype == COMET_F32)
+    return seg_gather_typed<float>(ctx, seg_end, crd, (const float *)val, M, N, (const float *)B, ldb, R, (float *)C, ldc,
+                                   out_row, out_rows, stream);
+  return seg_gather_typed<double>(ctx, seg_end, crd, (const double *)val, M, N, (const double *)B, ldb, R, (double *)C,
+                                  ldc, out_row, out_rows, stream);
 }
 
 }  // namespace comet

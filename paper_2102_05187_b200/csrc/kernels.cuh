@@ -8,27 +8,27 @@ namespace comet {
 // out[row(s), 0..R) = sum over leaf entries p of segment s of val[p] * B[crd[p], 0..R)   (SpMM, TTM)
 // seg_end[s] = leaf position where segment s ends. out_row == NULL: row(s) = s; otherwise row(s) =
 // out_row[s] (ascending) and all other rows below out_rows are zero-filled.
-comet_status_t seg_gather(Context *ctx, const int32_t *seg_end, const int32_t *crd, const double *val, int64_t M,
-                          int64_t N, const double *B, int64_t ldb, int64_t R, double *C, int64_t ldc,
+comet_status_t seg_gather(Context *ctx, int dtype, const int32_t *seg_end, const int32_t *crd, const void *val,
+                          int64_t M, int64_t N, const void *B, int64_t ldb, int64_t R, void *C, int64_t ldc,
                           const int32_t *out_row, int64_t out_rows, cudaStream_t stream);
 
 // y[row(s)] = sum over leaf entries p of segment s of val[p] * x[crd[p]]                    (SpMV, TTV)
-comet_status_t seg_dot(Context *ctx, const int32_t *seg_end, const int32_t *crd, const double *val, int64_t M,
-                       int64_t N, const double *x, int64_t x_len, double *y, const int32_t *out_row,
+comet_status_t seg_dot(Context *ctx, int dtype, const int32_t *seg_end, const int32_t *crd, const void *val, int64_t M,
+                       int64_t N, const void *x, int64_t x_len, void *y, const int32_t *out_row,
                        int64_t out_rows, cudaStream_t stream);
 
 // Sorted COO [CN,S,S]: out[crd0[p], :] += val[p] * P[crd1[p], :] * Q[crd2[p], :]; every row < rows written.
-comet_status_t mttkrp_coo(Context *ctx, const int32_t *crd0, const int32_t *crd1, const int32_t *crd2,
-                          const double *val, int64_t N, int64_t rows, const double *P, int64_t ldp, const double *Q,
-                          int64_t ldq, int64_t R, double *out, int64_t ldo, cudaStream_t stream);
+comet_status_t mttkrp_coo(Context *ctx, int dtype, const int32_t *crd0, const int32_t *crd1, const int32_t *crd2,
+                          const void *val, int64_t N, int64_t rows, const void *P, int64_t ldp, const void *Q,
+                          int64_t ldq, int64_t R, void *out, int64_t ldo, cudaStream_t stream);
 
 // CSF [CU,CU,CU]: per fiber t = sum val * Q[crd2]; out[crd0[slice], :] += t * P[crd1[fiber], :].
-comet_status_t mttkrp_csf(Context *ctx, const int32_t *pos1, const int32_t *crd0, const int32_t *crd1,
-                          const int32_t *pos2, const int32_t *crd2, const double *val, int64_t S, int64_t F,
-                          int64_t N, int64_t rows, const double *P, int64_t ldp, const double *Q, int64_t ldq,
-                          int64_t R, double *out, int64_t ldo, cudaStream_t stream);
+comet_status_t mttkrp_csf(Context *ctx, int dtype, const int32_t *pos1, const int32_t *crd0, const int32_t *crd1,
+                          const int32_t *pos2, const int32_t *crd2, const void *val, int64_t S, int64_t F,
+                          int64_t N, int64_t rows, const void *P, int64_t ldp, const void *Q, int64_t ldq,
+                          int64_t R, void *out, int64_t ldo, cudaStream_t stream);
 
-comet_status_t zero_rows(Context *ctx, double *C, int64_t rows, int64_t R, int64_t ldc, cudaStream_t stream);
+comet_status_t zero_rows(Context *ctx, void *C, int dtype, int64_t rows, int64_t R, int64_t ldc, cudaStream_t stream);
 int32_t choose_tile_items(int64_t total_items, int workers_per_block);
 
 // Block list of a library-owned tensor (what comet_sptensor_free releases).
@@ -36,9 +36,10 @@ void *owner_new();
 void *owner_alloc(Context *ctx, void *owner, size_t bytes, cudaStream_t stream);
 void owner_release(Context *ctx, void *owner, cudaStream_t stream);
 
-// Carry fix-up shared by the vector kernels (see contract_vec.cu).
-__global__ void carry_fixup_kernel(const double *__restrict__ carry_val, const int32_t *__restrict__ carry_seg,
-                                   int64_t num_tiles, int32_t R, int32_t carry_ld, double *__restrict__ C,
-                                   int64_t ldc, const int32_t *__restrict__ out_row);
+// Carry fix-up shared by all contraction kernels (defined in contract_vec.cu): adds the per-tile open sums
+// carry_val[tile, 0..R) onto row carry_seg[tile] of C (mapped through out_row when given). One launch of
+// num_tiles * R threads on `stream`; the caller checks the launch.
+void carry_fixup_launch(int dtype, const double *carry_val, const int32_t *carry_seg, int64_t num_tiles, int32_t R,
+                        int32_t carry_ld, void *C, int64_t ldc, const int32_t *out_row, cudaStream_t stream);
 
 }  // namespace comet

@@ -30,13 +30,13 @@ namespace comet {
 struct MttkrpArgs {
   // COO: crd0/crd1/crd2/val over N entries. CSF: pos1 (S+1), crd0 (S), crd1 (F), seg_end2 (= pos2+1, F), crd2, val.
   const int32_t *pos1, *crd0, *crd1, *seg_end2, *crd2;
-  const double *val;
+  const void *val;   // values, factors and output are T (double or float)
   int64_t S, F, N, rows;
-  const double *P;   // factor gathered by the level-1 coordinate
+  const void *P;     // factor gathered by the level-1 coordinate
   int64_t ldp;
-  const double *Q;   // factor gathered by the level-2 (leaf) coordinate
+  const void *Q;     // factor gathered by the level-2 (leaf) coordinate
   int64_t ldq;
-  double *out;
+  void *out;
   int64_t ldo;
   int32_t R;
   int32_t tile_items;
@@ -47,40 +47,42 @@ struct MttkrpArgs {
 };
 
 // ------------------------------------------------------------------------------------------- COO
-template <int LPN, int CPL, int VEC>
+template <class T, int LPN, int CPL, int VEC>
 struct CooPolicy {
-  using L = Lanes<LPN, CPL, VEC>;
+  using L = Lanes<T, LPN, CPL, VEC>;
   static constexpr int kPF = COMET_PF_COO;   // two rows per entry
   static constexpr bool kAux = true;         // the root coordinate rides in the side ring
   static constexpr bool kFullUnroll = true;
-  struct Slot { double r[2][CPL][VEC]; };
+  struct Slot { T r[2][CPL][VEC]; };
 
   const MttkrpArgs &a;
   const L &ln;
   const char *pcol, *qcol;               // this lane's piece 0 of row 0 of P and of Q
   int32_t ldp_bytes, ldq_bytes;
-  double *ocol;                          // this lane's piece 0 of row 0 of the output
+  T *ocol;                               // this lane's piece 0 of row 0 of the output
+  const T *val;
   double acc[CPL][VEC];
   int32_t cur;                           // output row being accumulated
 
   __device__ __forceinline__ CooPolicy(const MttkrpArgs &args, const L &lanes, int32_t first_row)
       : a(args), ln(lanes), cur(first_row) {
     ln.zero(acc);
-    pcol = reinterpret_cast<const char *>(a.P + ln.col0);
-    qcol = reinterpret_cast<const char *>(a.Q + ln.col0);
-    ldp_bytes = (int32_t)(a.ldp * 8);
-    ldq_bytes = (int32_t)(a.ldq * 8);
-    ocol = a.out + ln.col0;
+    pcol = reinterpret_cast<const char *>(static_cast<const T *>(a.P) + ln.col0);
+    qcol = reinterpret_cast<const char *>(static_cast<const T *>(a.Q) + ln.col0);
+    ldp_bytes = (int32_t)(a.ldp * sizeof(T));
+    ldq_bytes = (int32_t)(a.ldq * sizeof(T));
+    ocol = static_cast<T *>(a.out) + ln.col0;
+    val = static_cast<const T *>(a.val);
   }
   __device__ __forceinline__ void fetch(int32_t j, Entry16 &e, int32_t &aux) const {
-    e.v = ld_stream(a.val + j);
+    e.v = (double)ld_stream(val + j);
     e.a = ld_stream(a.crd1 + j);
     e.b = ld_stream(a.crd2 + j);
     aux = ld_stream(a.crd0 + j);
   }
   __device__ __forceinline__ void prefetch(int32_t cj, int32_t ck, Slot &s) const {
-    ln.gather(reinterpret_cast<const double *>(pcol + (int64_t)cj * ldp_bytes), s.r[0]);
-    ln.gather(reinterpret_cast<const double *>(qcol + (int64_t)ck * ldq_bytes), s.r[1]);
+    ln.gather(reinterpret_cast<const T *>(pcol + (int64_t)cj * ldp_bytes), s.r[0]);
+    ln.gather(reinterpret_cast<const T *>(qcol + (int64_t)ck * ldq_bytes), s.r[1]);
   }
   __device__ __forceinline__ void begin_chunk(int32_t) {}
   // The run of `cur` ends here: store it, zero-fill the rows up to the next stored row.
@@ -96,18 +98,18 @@ struct CooPolicy {
     for (int t = 0; t < CPL; ++t)
       if (ln.ok[t])
 #pragma unroll
-        for (int k = 0; k < VEC; ++k) acc[t][k] = fma(v * s.r[0][t][k], s.r[1][t][k], acc[t][k]);
+        for (int k = 0; k < VEC; ++k) acc[t][k] = fma(v * (double)s.r[0][t][k], (double)s.r[1][t][k], acc[t][k]);
   }
 };
 
-template <int LPN, int CPL, int VEC>
-__global__ void __launch_bounds__(kBlockThreads, (CPL * VEC <= 2 ? COMET_MINB_COO : 1)) mttkrp_coo_kernel(const MttkrpArgs a) {
-  using L = Lanes<LPN, CPL, VEC>;
+template <class T, int LPN, int CPL, int VEC>
+__global__ void __launch_bounds__(kBlockThreads, (CPL * VEC * sizeof(T) <= 16 ? COMET_MINB_COO : 1)) mttkrp_coo_kernel(const MttkrpArgs a) {
+  using L = Lanes<T, LPN, CPL, VEC>;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int worker = threadIdx.x / LPN;
   const int64_t tile = (int64_t)blockIdx.x * L::kWorkers + worker;
   if (tile >= a.num_tiles) return;
-  using P = CooPolicy<LPN, CPL, VEC>;
+  using P = CooPolicy<T, LPN, CPL, VEC>;
   const uint32_t smem = smem_u32(smem_raw) + worker * RingLayout<L, true>::kWorkerBytes;
   const L ln(a.R);
 
@@ -133,21 +135,22 @@ __global__ void __launch_bounds__(kBlockThreads, (CPL * VEC <= 2 ? COMET_MINB_CO
 }
 
 // ------------------------------------------------------------------------------------------- CSF
-template <int LPN, int CPL, int VEC>
+template <class T, int LPN, int CPL, int VEC>
 struct CsfPolicy {
-  using L = Lanes<LPN, CPL, VEC>;
+  using L = Lanes<T, LPN, CPL, VEC>;
   static constexpr int kPF = COMET_PF_CSF;
   static constexpr bool kAux = false;
   static constexpr bool kFullUnroll = false;   // the fiber/slice epilogue is long: keep the body small
-  struct Slot { double r[CPL][VEC]; };
+  struct Slot { T r[CPL][VEC]; };
 
   const MttkrpArgs &a;
   const L &ln;
   const char *pcol, *qcol;
   int32_t ldp_bytes, ldq_bytes;
-  double *ocol;
+  T *ocol;
+  const T *val;
   double tac[CPL][VEC], aac[CPL][VEC];   // open fiber sum, open slice sum
-  double prow[CPL][VEC];                 // P row of the open fiber, fetched when the fiber opened
+  T prow[CPL][VEC];                      // P row of the open fiber, fetched when the fiber opened
   // cursors instead of indices: the per-fiber path is executed once per fiber and per worker (divergently),
   // so it is kept to pointer bumps and 32-bit compares
   const int32_t *endp;                   // seg_end2 + open fiber
@@ -164,12 +167,16 @@ struct CsfPolicy {
       : a(args), ln(lanes), s((int32_t)s0), base(j0), last_fold(j0), a_dirty(false) {
     ln.zero(tac);
     ln.zero(aac);
-    ln.zero(prow);
-    pcol = reinterpret_cast<const char *>(a.P + ln.col0);
-    qcol = reinterpret_cast<const char *>(a.Q + ln.col0);
-    ldp_bytes = (int32_t)(a.ldp * 8);
-    ldq_bytes = (int32_t)(a.ldq * 8);
-    ocol = a.out + ln.col0;
+#pragma unroll
+    for (int t = 0; t < CPL; ++t)
+#pragma unroll
+      for (int k = 0; k < VEC; ++k) prow[t][k] = (T)0;
+    pcol = reinterpret_cast<const char *>(static_cast<const T *>(a.P) + ln.col0);
+    qcol = reinterpret_cast<const char *>(static_cast<const T *>(a.Q) + ln.col0);
+    ldp_bytes = (int32_t)(a.ldp * sizeof(T));
+    ldq_bytes = (int32_t)(a.ldq * sizeof(T));
+    ocol = static_cast<T *>(a.out) + ln.col0;
+    val = static_cast<const T *>(a.val);
     endp = a.seg_end2 + f0;
     c1p = a.crd1 + f0;
     fibers_left = (int32_t)(a.F - f0);
@@ -180,14 +187,14 @@ struct CsfPolicy {
   }
   __device__ __forceinline__ int64_t fiber() const { return a.F - fibers_left; }
   __device__ __forceinline__ void open_fiber() {         // start fetching the P row the fiber will be folded with
-    if (fibers_left > 0) ln.gather(reinterpret_cast<const double *>(pcol + (int64_t)__ldg(c1p) * ldp_bytes), prow);
+    if (fibers_left > 0) ln.gather(reinterpret_cast<const T *>(pcol + (int64_t)__ldg(c1p) * ldp_bytes), prow);
   }
   __device__ __forceinline__ void fetch(int32_t j, Entry16 &e, int32_t &) const {
-    e.v = ld_stream(a.val + j);
+    e.v = (double)ld_stream(val + j);
     e.a = ld_stream(a.crd2 + j);
   }
   __device__ __forceinline__ void prefetch(int32_t ck, int32_t, Slot &sl) const {
-    ln.gather(reinterpret_cast<const double *>(qcol + (int64_t)ck * ldq_bytes), sl.r);
+    ln.gather(reinterpret_cast<const T *>(qcol + (int64_t)ck * ldq_bytes), sl.r);
   }
   __device__ __forceinline__ void begin_chunk(int32_t b) { base = b; rel_end = next_end - b; }
 
@@ -196,7 +203,7 @@ struct CsfPolicy {
     for (int t = 0; t < CPL; ++t)
       if (ln.ok[t])
 #pragma unroll
-        for (int k = 0; k < VEC; ++k) { aac[t][k] = fma(tac[t][k], prow[t][k], aac[t][k]); tac[t][k] = 0.0; }
+        for (int k = 0; k < VEC; ++k) { aac[t][k] = fma(tac[t][k], (double)prow[t][k], aac[t][k]); tac[t][k] = 0.0; }
     a_dirty = true;
     last_fold = j;
   }
@@ -227,14 +234,14 @@ struct CsfPolicy {
   }
 };
 
-template <int LPN, int CPL, int VEC>
-__global__ void __launch_bounds__(kBlockThreads, (CPL * VEC <= 2 ? COMET_MINB_CSF : 2)) mttkrp_csf_kernel(const MttkrpArgs a) {
-  using L = Lanes<LPN, CPL, VEC>;
+template <class T, int LPN, int CPL, int VEC>
+__global__ void __launch_bounds__(kBlockThreads, (CPL * VEC * sizeof(T) <= 16 ? COMET_MINB_CSF : 2)) mttkrp_csf_kernel(const MttkrpArgs a) {
+  using L = Lanes<T, LPN, CPL, VEC>;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int worker = threadIdx.x / LPN;
   const int64_t tile = (int64_t)blockIdx.x * L::kWorkers + worker;
   if (tile >= a.num_tiles) return;
-  using P = CsfPolicy<LPN, CPL, VEC>;
+  using P = CsfPolicy<T, LPN, CPL, VEC>;
   const uint32_t smem = smem_u32(smem_raw) + worker * RingLayout<L, false>::kWorkerBytes;
   const L ln(a.R);
 
@@ -265,7 +272,7 @@ __global__ void __launch_bounds__(kBlockThreads, (CPL * VEC <= 2 ? COMET_MINB_CS
 // ------------------------------------------------------------------------------------------- host
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
-template <bool CSF, int LPN, int CPL, int VEC>
+template <bool CSF, class T, int LPN, int CPL, int VEC>
 static comet_status_t launch_mttkrp(Context *ctx, MttkrpArgs a, cudaStream_t stream) {
   constexpr int WORKERS = kBlockThreads / LPN;
   const int64_t total = CSF ? a.F + a.N : a.N;
@@ -279,70 +286,74 @@ static comet_status_t launch_mttkrp(Context *ctx, MttkrpArgs a, cudaStream_t str
   a.carry_val = (double *)scratch;
   a.carry_seg = (int32_t *)(scratch + val_bytes);
   const unsigned blocks = (unsigned)ceil_div(a.num_tiles, WORKERS);
-  using L = Lanes<LPN, CPL, VEC>;
+  using L = Lanes<T, LPN, CPL, VEC>;
   constexpr size_t smem = CSF ? RingLayout<L, false>::kBlockBytes : RingLayout<L, true>::kBlockBytes;
-  auto kernel = CSF ? mttkrp_csf_kernel<LPN, CPL, VEC> : mttkrp_coo_kernel<LPN, CPL, VEC>;
+  auto kernel = CSF ? mttkrp_csf_kernel<T, LPN, CPL, VEC> : mttkrp_coo_kernel<T, LPN, CPL, VEC>;
   if (smem > 48 * 1024)
     COMET_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   kernel<<<blocks, kBlockThreads, smem, stream>>>(a);
   COMET_LAUNCH_CHECK(ctx);
-  carry_fixup_kernel<<<(unsigned)ceil_div(a.num_tiles * a.R, 256), 256, 0, stream>>>(
-      a.carry_val, a.carry_seg, a.num_tiles, a.R, a.carry_ld, a.out, a.ldo, CSF ? a.crd0 : nullptr);
+  carry_fixup_launch(sizeof(T) == 4 ? COMET_F32 : COMET_F64, a.carry_val, a.carry_seg, a.num_tiles, a.R, a.carry_ld, a.out,
+                     a.ldo, CSF ? a.crd0 : nullptr, stream);
   COMET_LAUNCH_CHECK(ctx);
   return COMET_OK;
 }
 
-template <bool CSF>
+template <bool CSF, class T>
 static comet_status_t mttkrp_chunks(Context *ctx, MttkrpArgs base, int64_t R, cudaStream_t stream) {
-  const bool vec_ok = aligned16(base.P) && aligned16(base.Q) && aligned16(base.out) && base.ldp % 2 == 0 &&
-                      base.ldq % 2 == 0 && base.ldo % 2 == 0;
+  constexpr int PER = 16 / sizeof(T);
+  const bool vec_ok = aligned16(base.P) && aligned16(base.Q) && aligned16(base.out) && base.ldp % PER == 0 &&
+                      base.ldq % PER == 0 && base.ldo % PER == 0;
   int64_t done = 0;
   while (done < R) {
     const int64_t rem = R - done;
     const int64_t chunk = rem < 128 ? rem : 128;
     MttkrpArgs a = base;
-    a.P += done; a.Q += done; a.out += done;
+    a.P = static_cast<const T *>(base.P) + done;
+    a.Q = static_cast<const T *>(base.Q) + done;
+    a.out = static_cast<T *>(base.out) + done;
     a.R = (int32_t)chunk;
-    const bool v = vec_ok && done % 2 == 0;
+    const bool v = vec_ok && done % PER == 0 && chunk % PER == 0;
+    const int64_t pieces = chunk / PER;
     comet_status_t st;
-    if (v && chunk == 128) st = launch_mttkrp<CSF, 32, 2, 2>(ctx, a, stream);
-    else if (v && chunk == 64) st = launch_mttkrp<CSF, 32, 1, 2>(ctx, a, stream);
-    else if (v && chunk == 32) st = launch_mttkrp<CSF, 16, 1, 2>(ctx, a, stream);
-    else if (v && chunk == 16) st = launch_mttkrp<CSF, 8, 1, 2>(ctx, a, stream);
-    else if (v && chunk == 8) st = launch_mttkrp<CSF, 4, 1, 2>(ctx, a, stream);
-    else if (v && chunk == 4) st = launch_mttkrp<CSF, 2, 1, 2>(ctx, a, stream);
-    else if (v && chunk == 2) st = launch_mttkrp<CSF, 1, 1, 2>(ctx, a, stream);
-    else if (chunk > 64) st = launch_mttkrp<CSF, 32, 4, 1>(ctx, a, stream);
-    else if (chunk > 32) st = launch_mttkrp<CSF, 32, 2, 1>(ctx, a, stream);
-    else st = launch_mttkrp<CSF, 32, 1, 1>(ctx, a, stream);
+    if (v && pieces == 64) st = launch_mttkrp<CSF, T, 32, 2, PER>(ctx, a, stream);
+    else if (v && pieces == 32) st = launch_mttkrp<CSF, T, 32, 1, PER>(ctx, a, stream);
+    else if (v && pieces == 16) st = launch_mttkrp<CSF, T, 16, 1, PER>(ctx, a, stream);
+    else if (v && pieces == 8) st = launch_mttkrp<CSF, T, 8, 1, PER>(ctx, a, stream);
+    else if (v && pieces == 4) st = launch_mttkrp<CSF, T, 4, 1, PER>(ctx, a, stream);
+    else if (v && pieces == 2) st = launch_mttkrp<CSF, T, 2, 1, PER>(ctx, a, stream);
+    else if (v && pieces == 1) st = launch_mttkrp<CSF, T, 1, 1, PER>(ctx, a, stream);
+    else if (chunk > 64) st = launch_mttkrp<CSF, T, 32, 4, 1>(ctx, a, stream);
+    else if (chunk > 32) st = launch_mttkrp<CSF, T, 32, 2, 1>(ctx, a, stream);
+    else st = launch_mttkrp<CSF, T, 32, 1, 1>(ctx, a, stream);
     if (st != COMET_OK) return st;
     done += chunk;
   }
   return COMET_OK;
 }
 
-comet_status_t mttkrp_coo(Context *ctx, const int32_t *crd0, const int32_t *crd1, const int32_t *crd2,
-                          const double *val, int64_t N, int64_t rows, const double *P, int64_t ldp, const double *Q,
-                          int64_t ldq, int64_t R, double *out, int64_t ldo, cudaStream_t stream) {
+comet_status_t mttkrp_coo(Context *ctx, int dtype, const int32_t *crd0, const int32_t *crd1, const int32_t *crd2,
+                          const void *val, int64_t N, int64_t rows, const void *P, int64_t ldp, const void *Q,
+                          int64_t ldq, int64_t R, void *out, int64_t ldo, cudaStream_t stream) {
   if (ldp >= (1ll << 28) || ldq >= (1ll << 28)) return COMET_ERR_INDEX_OVERFLOW;
-  if (N == 0) return zero_rows(ctx, out, rows, R, ldo, stream);
+  if (N == 0) return zero_rows(ctx, out, dtype, rows, R, ldo, stream);
   MttkrpArgs a{};
   a.crd0 = crd0; a.crd1 = crd1; a.crd2 = crd2; a.val = val; a.N = N; a.rows = rows;
   a.P = P; a.ldp = ldp; a.Q = Q; a.ldq = ldq; a.out = out; a.ldo = ldo;
-  return mttkrp_chunks<false>(ctx, a, R, stream);
+  return dtype == COMET_F32 ? mttkrp_chunks<false, float>(ctx, a, R, stream) : mttkrp_chunks<false, double>(ctx, a, R, stream);
 }
 
-comet_status_t mttkrp_csf(Context *ctx, const int32_t *pos1, const int32_t *crd0, const int32_t *crd1,
-                          const int32_t *pos2, const int32_t *crd2, const double *val, int64_t S, int64_t F,
-                          int64_t N, int64_t rows, const double *P, int64_t ldp, const double *Q, int64_t ldq,
-                          int64_t R, double *out, int64_t ldo, cudaStream_t stream) {
+comet_status_t mttkrp_csf(Context *ctx, int dtype, const int32_t *pos1, const int32_t *crd0, const int32_t *crd1,
+                          const int32_t *pos2, const int32_t *crd2, const void *val, int64_t S, int64_t F,
+                          int64_t N, int64_t rows, const void *P, int64_t ldp, const void *Q, int64_t ldq,
+                          int64_t R, void *out, int64_t ldo, cudaStream_t stream) {
   if (ldp >= (1ll << 28) || ldq >= (1ll << 28)) return COMET_ERR_INDEX_OVERFLOW;
-  if (N == 0 || S == 0) return zero_rows(ctx, out, rows, R, ldo, stream);
+  if (N == 0 || S == 0) return zero_rows(ctx, out, dtype, rows, R, ldo, stream);
   MttkrpArgs a{};
   a.pos1 = pos1; a.crd0 = crd0; a.crd1 = crd1; a.seg_end2 = pos2 + 1; a.crd2 = crd2; a.val = val;
   a.S = S; a.F = F; a.N = N; a.rows = rows;
   a.P = P; a.ldp = ldp; a.Q = Q; a.ldq = ldq; a.out = out; a.ldo = ldo;
-  return mttkrp_chunks<true>(ctx, a, R, stream);
+  return dtype == COMET_F32 ? mttkrp_chunks<true, float>(ctx, a, R, stream) : mttkrp_chunks<true, double>(ctx, a, R, stream);
 }
 
 }  // namespace comet

@@ -314,16 +314,16 @@ __global__ void __launch_bounds__(kLevelThreads) level_count_kernel(const uint64
 struct LevelOut {
   int32_t *pos[COMET_MAX_ORDER];
   int32_t *crd[COMET_MAX_ORDER];
-  double *val;
+  void *val;                   // fp64 or fp32, as the COO values
   int64_t dim0;                // extent of level 0 (for a dense root)
   uint32_t nodes[COMET_MAX_ORDER];   // node count of every counted level (indexed by level)
 };
 
 // Per tile: ranks of the heads (tile-local scan + the tile's scanned offset), then crd / pos / val.
-template <int ORDER>
+template <int ORDER, class V>
 __global__ void __launch_bounds__(kLevelThreads) level_emit_kernel(const uint64_t *__restrict__ keys,
                                                                    const uint32_t *__restrict__ perm,
-                                                                   const double *__restrict__ val_in, int64_t n,
+                                                                   const V *__restrict__ val_in, int64_t n,
                                                                    LevelPlan plan, int64_t tiles,
                                                                    const uint32_t *__restrict__ offsets,
                                                                    LevelOut out) {
@@ -337,9 +337,9 @@ __global__ void __launch_bounds__(kLevelThreads) level_emit_kernel(const uint64_
     k[t + 1] = (base + t < n) ? keys[base + t] : 0;
     src[t] = (base + t < n) ? perm[base + t] : 0;
   }
-  double vals[kLevelItems];
+  V vals[kLevelItems];
 #pragma unroll
-  for (int t = 0; t < kLevelItems; ++t) vals[t] = (base + t < n) ? __ldg(val_in + src[t]) : 0.0;   // the random gather, all in flight
+  for (int t = 0; t < kLevelItems; ++t) vals[t] = (base + t < n) ? __ldg(val_in + src[t]) : (V)0;   // the random gather, all in flight
 
   // rank[l] = nodes of level l opened before this thread's first entry
   uint32_t rank[ORDER];
@@ -397,7 +397,7 @@ __global__ void __launch_bounds__(kLevelThreads) level_emit_kernel(const uint64_
           parent_head = true;
         }
       }
-      out.val[p] = vals[t];
+      static_cast<V *>(out.val)[p] = vals[t];
     }
   }
 }
@@ -503,7 +503,7 @@ extern "C" comet_status_t comet_pack(comet_handle_t handle, int32_t order, const
   if (!handle || !out || !h_dims || !h_coo_crd || !h_mode_order || !h_attr) return COMET_ERR_INVALID_ARG;
   memset(out, 0, sizeof(*out));
   if (order < 1 || order > COMET_MAX_ORDER || nnz < 0) return COMET_ERR_INVALID_ARG;
-  if (dtype != COMET_F64) return COMET_ERR_UNSUPPORTED_FORMAT;
+  if (dtype != COMET_F64 && dtype != COMET_F32) return COMET_ERR_UNSUPPORTED_FORMAT;
   if (nnz > 2147483647ll - 1024) return COMET_ERR_INDEX_OVERFLOW;
   bool seen[COMET_MAX_ORDER] = {false, false, false, false};
   for (int l = 0; l < order; ++l) {
@@ -603,7 +603,7 @@ extern "C" comet_status_t comet_pack(comet_handle_t handle, int32_t order, const
   LevelOut lo{};
   bool alloc_ok = true;
   out->order = order;
-  out->dtype = COMET_F64;
+  out->dtype = dtype;
   out->nnz = n;
   int64_t parents = 1;
   for (int l = 0; l < order; ++l) {
@@ -624,16 +624,25 @@ extern "C" comet_status_t comet_pack(comet_handle_t handle, int32_t order, const
     lo.pos[l] = out->pos[l];
     lo.crd[l] = out->crd[l];
   }
-  if (n > 0) { out->val = owner_alloc(ctx, owner, (size_t)n * 8, s); alloc_ok &= out->val != nullptr; }
-  lo.val = (double *)out->val;
+  const size_t val_size = dtype == COMET_F32 ? 4 : 8;
+  if (n > 0) { out->val = owner_alloc(ctx, owner, (size_t)n * val_size, s); alloc_ok &= out->val != nullptr; }
+  lo.val = out->val;
   lo.dim0 = key.dim[0];
   if (!alloc_ok) { owner_release(ctx, owner, s); memset(out, 0, sizeof(*out)); return COMET_ERR_ALLOC; }
 
-  const double *vin = (const double *)coo_val;
   if (n > 0) {
-    if (order == 2) level_emit_kernel<2><<<(unsigned)level_tiles, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
-    else if (order == 3) level_emit_kernel<3><<<(unsigned)level_tiles, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
-    else level_emit_kernel<4><<<(unsigned)level_tiles, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
+    const unsigned g = (unsigned)level_tiles;
+    if (dtype == COMET_F32) {
+      const float *vin = (const float *)coo_val;
+      if (order == 2) level_emit_kernel<2, float><<<g, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
+      else if (order == 3) level_emit_kernel<3, float><<<g, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
+      else level_emit_kernel<4, float><<<g, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
+    } else {
+      const double *vin = (const double *)coo_val;
+      if (order == 2) level_emit_kernel<2, double><<<g, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
+      else if (order == 3) level_emit_kernel<3, double><<<g, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
+      else level_emit_kernel<4, double><<<g, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
+    }
   }
   if (order == 2) level_finish_kernel<2><<<kSmCount, 256, 0, s>>>(keys_a, n, plan, lo);
   else if (order == 3) level_finish_kernel<3><<<kSmCount, 256, 0, s>>>(keys_a, n, plan, lo);

@@ -68,34 +68,49 @@ __device__ __forceinline__ void sts_s32(uint32_t addr, int32_t v) {
   asm volatile("st.shared.s32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 
-template <int VEC> struct Piece;
-template <> struct Piece<2> {
-  // volatile: the gathers keep their program order relative to the ring reads, so exactly the rolling
-  // window is in flight (the scheduler otherwise hoists loads of far-ahead entries and spills)
+// A lane's piece of a dense row: VEC elements of T. Vector pieces are 16 bytes (2 doubles or 4 floats);
+// VEC == 1 is the scalar path for ragged widths or unaligned operands. Loads are volatile so that the
+// gathers keep their program order relative to the ring reads: exactly the rolling window is in flight
+// (the scheduler otherwise hoists loads of far-ahead entries and spills).
+template <class T, int VEC> struct Piece;
+template <> struct Piece<double, 2> {
   static __device__ __forceinline__ void load(const double *p, double (&d)[2]) {
     asm volatile("ld.global.nc.v2.f64 {%0, %1}, [%2];" : "=d"(d[0]), "=d"(d[1]) : "l"(p));
   }
   static __device__ __forceinline__ void store_stream(double *p, const double (&d)[2]) {
     __stcs(reinterpret_cast<double2 *>(p), make_double2(d[0], d[1]));
   }
-  static __device__ __forceinline__ void store(double *p, const double (&d)[2]) {
-    *reinterpret_cast<double2 *>(p) = make_double2(d[0], d[1]);
-  }
 };
-template <> struct Piece<1> {
+template <> struct Piece<double, 1> {
   static __device__ __forceinline__ void load(const double *p, double (&d)[1]) {
     asm volatile("ld.global.nc.f64 %0, [%1];" : "=d"(d[0]) : "l"(p));
   }
   static __device__ __forceinline__ void store_stream(double *p, const double (&d)[1]) { __stcs(p, d[0]); }
-  static __device__ __forceinline__ void store(double *p, const double (&d)[1]) { *p = d[0]; }
+};
+template <> struct Piece<float, 4> {
+  static __device__ __forceinline__ void load(const float *p, float (&d)[4]) {
+    asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3]) : "l"(p));
+  }
+  static __device__ __forceinline__ void store_stream(float *p, const double (&d)[4]) {
+    __stcs(reinterpret_cast<float4 *>(p), make_float4((float)d[0], (float)d[1], (float)d[2], (float)d[3]));
+  }
+};
+template <> struct Piece<float, 1> {
+  static __device__ __forceinline__ void load(const float *p, float (&d)[1]) {
+    asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(d[0]) : "l"(p));
+  }
+  static __device__ __forceinline__ void store_stream(float *p, const double (&d)[1]) { __stcs(p, (float)d[0]); }
 };
 
-template <int LPN_, int CPL_, int VEC_> struct Lanes {
+// T is the storage type of values and dense operands (double or float); sums are always kept in double.
+template <class T_, int LPN_, int CPL_, int VEC_> struct Lanes {
+  using T = T_;
   static constexpr int LPN = LPN_, CPL = CPL_, VEC = VEC_;
   static constexpr int kChunk = LPN >= 16 ? 32 : (LPN >= 2 ? 16 : 8);   // leaf entries per refill of the ring
   static constexpr int kPer = kChunk / LPN;                // entries each lane loads per refill
   static constexpr int kWorkers = kBlockThreads / LPN;     // workers per CTA
   static constexpr int kStride = LPN * VEC;                // columns between a lane's consecutive pieces
+  static constexpr bool kVector = VEC * sizeof(T) == 16;   // 128-bit pieces: the launch width is never ragged
 
   int g;            // lane within the group
   unsigned mask;    // the group's lanes
@@ -108,7 +123,7 @@ template <int LPN_, int CPL_, int VEC_> struct Lanes {
     mask = LPN == 32 ? 0xffffffffu : (((1u << LPN) - 1u) << (lane & ~(LPN - 1)));
     col0 = g * VEC;
 #pragma unroll
-    for (int t = 0; t < CPL; ++t) ok[t] = VEC == 2 ? true : (col0 + t * kStride) < R;
+    for (int t = 0; t < CPL; ++t) ok[t] = kVector ? true : (col0 + t * kStride) < R;
   }
   __device__ __forceinline__ void sync() const { __syncwarp(mask); }
 
@@ -119,33 +134,35 @@ template <int LPN_, int CPL_, int VEC_> struct Lanes {
       for (int e = 0; e < VEC; ++e) acc[t][e] = 0.0;
   }
   // `row` already points at this lane's piece 0 (row base + col0)
-  __device__ __forceinline__ void gather(const double *row, double (&dst)[CPL][VEC]) const {
+  __device__ __forceinline__ void gather(const T *row, T (&dst)[CPL][VEC]) const {
 #pragma unroll
     for (int t = 0; t < CPL; ++t)
-      if (ok[t]) Piece<VEC>::load(row + t * kStride, dst[t]);
+      if (ok[t]) Piece<T, VEC>::load(row + t * kStride, dst[t]);
   }
-  __device__ __forceinline__ void store_row(double *row, const double (&acc)[CPL][VEC]) const {
+  __device__ __forceinline__ void store_row(T *row, const double (&acc)[CPL][VEC]) const {
 #pragma unroll
     for (int t = 0; t < CPL; ++t)
-      if (ok[t]) Piece<VEC>::store_stream(row + t * kStride, acc[t]);
+      if (ok[t]) Piece<T, VEC>::store_stream(row + t * kStride, acc[t]);
   }
-  __device__ __forceinline__ void store_carry(double *row, const double (&acc)[CPL][VEC]) const {
-#pragma unroll
-    for (int t = 0; t < CPL; ++t)
-      if (ok[t]) Piece<VEC>::store(row + t * kStride, acc[t]);
-  }
-  // rows lo .. hi-1 of a matrix whose lane-piece-0 pointer of row 0 is `base`
-  __device__ __forceinline__ void zero_rows(double *base, int64_t ld, int64_t lo, int64_t hi) const {
-    double z[CPL][VEC];
-    zero(z);
-    for (int64_t r = lo; r < hi; ++r) store_row(base + r * ld, z);
-  }
-  __device__ __forceinline__ void fma_rows(double v, const double (&row)[CPL][VEC], double (&acc)[CPL][VEC]) const {
+  __device__ __forceinline__ void store_carry(double *row, const double (&acc)[CPL][VEC]) const {   // carries stay double
 #pragma unroll
     for (int t = 0; t < CPL; ++t)
       if (ok[t])
 #pragma unroll
-        for (int e = 0; e < VEC; ++e) acc[t][e] = fma(v, row[t][e], acc[t][e]);
+        for (int e = 0; e < VEC; ++e) row[t * kStride + e] = acc[t][e];
+  }
+  // rows lo .. hi-1 of a matrix whose lane-piece-0 pointer of row 0 is `base`
+  __device__ __forceinline__ void zero_rows(T *base, int64_t ld, int64_t lo, int64_t hi) const {
+    double z[CPL][VEC];
+    zero(z);
+    for (int64_t r = lo; r < hi; ++r) store_row(base + r * ld, z);
+  }
+  __device__ __forceinline__ void fma_rows(double v, const T (&row)[CPL][VEC], double (&acc)[CPL][VEC]) const {
+#pragma unroll
+    for (int t = 0; t < CPL; ++t)
+      if (ok[t])
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) acc[t][e] = fma(v, (double)row[t][e], acc[t][e]);
   }
 };
 
