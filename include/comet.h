@@ -167,7 +167,16 @@ comet_status_t comet_ttm(comet_handle_t handle, const comet_sptensor_t *X, int32
 
 /* MTTKRP  out_{i_n r} = sum x_{i1 i2 i3} P_{p r} Q_{q r} over the two other modes p < q (the paper
  * names the operation without defining it; this is the textbook matricised-tensor-times-Khatri-Rao
- * product). `mode` = n must be the mode of X's FIRST level. X: [CN,S,S] (COO) or [CU,CU,CU] (CSF).
+ * product). X: [CN,S,S] (COO) or [CU,CU,CU] (CSF); `mode` = n may be ANY of the three modes, so that
+ * one packed tensor serves the all-modes sequence of CP-ALS:
+ *   - n stored at X's FIRST level: tiled kernels, every output row written by exactly one CTA, results
+ *     bit-identical from run to run;
+ *   - n stored at level 1 or 2: the tensor is used as stored (nothing is re-packed); the terms of an
+ *     output row are then spread over the whole tensor and are added with atomic adds in double, so
+ *     the summation ORDER is not fixed and results agree from run to run only up to rounding (still
+ *     within the stated tolerance). About 2-4x slower than the first-level case; callers that repeat the
+ *     same mode many times may prefer a second comet_pack with that mode first. For fp32 tensors this
+ *     path takes rows x R doubles of handle scratch.
  *   h_factors[3]  HOST array of DEVICE pointers, factor of mode m is dims[m] x R with leading
  *                 dimension h_ld[m]; the entry at `mode` is ignored
  *   out           dims[mode] x R, leading dimension ldo, every row written. */

@@ -324,18 +324,31 @@ extern "C" comet_status_t comet_mttkrp(comet_handle_t handle, const comet_sptens
   comet_status_t st = check_tensor(X, 3);
   if (st != COMET_OK) return st;
   if (mode < 0 || mode > 2) return COMET_ERR_INVALID_ARG;
-  if (X->mode_order[0] != mode) return COMET_ERR_UNSUPPORTED_FORMAT;   // re-pack with the output mode first
-  const int m1 = X->mode_order[1], m2 = X->mode_order[2];
+  const bool coo = is_fmt(X, 3, COMET_CN, COMET_S, COMET_S), csf = is_fmt(X, 3, COMET_CU, COMET_CU, COMET_CU);
+  if (!coo && !csf) return COMET_ERR_UNSUPPORTED_FORMAT;
+  int level = 0;                                     // the level that stores the output mode
+  while (X->mode_order[level] != mode) ++level;
+  const int la = level == 0 ? 1 : 0, lb = level == 2 ? 1 : 2;      // the two other levels, in storage order
+  const int m1 = X->mode_order[la], m2 = X->mode_order[lb];
   if (!h_factors[m1] || !h_factors[m2] || h_ld[m1] < R || h_ld[m2] < R) return COMET_ERR_INVALID_ARG;
   if (misaligned(h_factors[m1], X->dtype) || misaligned(h_factors[m2], X->dtype) || misaligned(out, X->dtype)) return COMET_ERR_MISALIGNED;
   Context *ctx = reinterpret_cast<Context *>(handle);
   cudaStream_t s = (cudaStream_t)stream;
   const int64_t rows = X->dims[mode];
   const void *P = h_factors[m1], *Q = h_factors[m2];
-  if (is_fmt(X, 3, COMET_CN, COMET_S, COMET_S))
+  if (level > 0) {
+    // output mode below the root: atomic accumulation on the tensor as stored
+    if (h_ld[m1] >= (1ll << 28) || h_ld[m2] >= (1ll << 28)) return COMET_ERR_INDEX_OVERFLOW;
+    if (coo)
+      return mttkrp_scatter(ctx, X->dtype, 0, nullptr, X->crd[level], X->crd[la], nullptr, X->crd[lb], X->val, 0, 0,
+                            X->nnz, rows, P, h_ld[m1], Q, h_ld[m2], R, out, ldo, s);
+    return mttkrp_scatter(ctx, X->dtype, level, X->pos[1], X->crd[0], X->crd[1], X->pos[2], X->crd[2], X->val,
+                          X->crd_len[0], X->crd_len[1], X->nnz, rows, P, h_ld[m1], Q, h_ld[m2], R, out, ldo, s);
+  }
+  if (coo)
     return mttkrp_coo(ctx, X->dtype, X->crd[0], X->crd[1], X->crd[2], X->val, X->nnz, rows, P, h_ld[m1], Q, h_ld[m2], R, out,
                       ldo, s);
-  if (is_fmt(X, 3, COMET_CU, COMET_CU, COMET_CU))
+  if (csf)
     return mttkrp_csf(ctx, X->dtype, X->pos[1], X->crd[0], X->crd[1], X->pos[2], X->crd[2], X->val, X->crd_len[0],
                       X->crd_len[1], X->nnz, rows, P, h_ld[m1], Q, h_ld[m2], R, out, ldo, s);
   return COMET_ERR_UNSUPPORTED_FORMAT;

@@ -193,6 +193,40 @@ def test_mttkrp(dims, nnz, seed, mode, attr, tile_items):
         assert_close(out, want, norm, what=f"mttkrp R={R}")
 
 
+@pytest.mark.parametrize("dims,nnz,seed", TENSOR_CASES)
+@pytest.mark.parametrize("mode_order", [(0, 1, 2), (2, 0, 1), (1, 2, 0)])
+@pytest.mark.parametrize("attr", [(CN, S, S), (CU, CU, CU)])
+def test_mttkrp_every_mode_of_a_fixed_tensor(dims, nnz, seed, mode_order, attr):
+    """All three modes on ONE packed tensor (the all-modes sequence of CP-ALS): the mode stored first takes
+    the deterministic kernels, the other two accumulate with atomic adds on the tensor as stored."""
+    coords, val = synth.random_coo(dims, nnz, seed)
+    c, v = _np(coords), val.numpy()
+    X = upload_packed(oracle.pack(c, v, dims, mode_order, attr))
+    for R in (1, 3, 16, 40):
+        F = [synth.random_dense((d, R), seed, 60 + m).numpy() for m, d in enumerate(dims)]
+        for mode in range(3):
+            want, norm = oracle.mttkrp(c, v, dims, mode, F)
+            out = torch.full((dims[mode], R), float("nan"), dtype=torch.float64, device="cuda")
+            comet.mttkrp(X, mode, [None if m == mode else dev(f) for m, f in enumerate(F)], out)
+            assert_close(out, want, norm, what=f"mttkrp mode {mode} of {mode_order} R={R}")
+
+
+def test_mttkrp_non_root_strided_output_and_integers():
+    dims = (25, 20, 15)
+    coords, val = synth.random_coo(dims, 2000, 5, integer_values=True)
+    c, v = _np(coords), val.numpy()
+    R = 6
+    F = [synth.random_dense((d, R), 5, 60 + m, integer_values=True).numpy() for m, d in enumerate(dims)]
+    for attr in [(CN, S, S), (CU, CU, CU)]:
+        X = upload_packed(oracle.pack(c, v, dims, (0, 1, 2), attr))
+        for mode in (1, 2):
+            want, _ = oracle.mttkrp(c, v, dims, mode, F)
+            buf = torch.full((dims[mode], R + 3), 7.0, dtype=torch.float64, device="cuda")
+            comet.mttkrp(X, mode, [None if m == mode else dev(f) for m, f in enumerate(F)], buf[:, :R])
+            assert_equal_arrays(buf[:, :R].contiguous(), want, "integer non-root mttkrp")   # exact sums: any order
+            assert bool((buf[:, R:] == 7.0).all())                                          # padding untouched
+
+
 def test_mttkrp_exact_on_small_integers():
     dims = (25, 20, 15)
     coords, val = synth.random_coo(dims, 2000, 5, integer_values=True)
@@ -255,5 +289,9 @@ def test_argument_errors_are_reported_not_raised_by_cuda():
         comet.ttv(X, 0, torch.ones(2, dtype=torch.float64, device="cuda"))             # mode 0 is not stored last
     assert e.value.status == -2
     with pytest.raises(comet.CometError) as e:
-        comet.mttkrp(X, 2, [B[:, :1], B[:, :1], None])                                 # mode 2 is not stored first
+        comet.mttkrp(X, 3, [B[:, :1], B[:, :1], None])                                 # no such mode
+    assert e.value.status == -1
+    Xd = upload_packed(oracle.pack([[0], [1], [1]], [1.0], (2, 2, 2), (0, 1, 2), (D, CU, CU)))
+    with pytest.raises(comet.CometError) as e:
+        comet.mttkrp(Xd, 0, [None, B[:, :1], B[:, :1]])                                # MTTKRP takes COO or CSF
     assert e.value.status == -2

@@ -181,6 +181,20 @@ def test_mttkrp_fp32(dims, nnz, seed, mode, attr, tile_items):
         check(out, want, norm, f"mttkrp fp32 R={R}")
 
 
+@pytest.mark.parametrize("attr", [(CN, S, S), (CU, CU, CU)])
+def test_mttkrp_fp32_every_mode_of_a_fixed_tensor(attr):
+    dims = (50, 40, 30)
+    c, v = _coo(dims, 6000, 2)
+    X = upload32(oracle.pack(c, v, dims, (0, 1, 2), attr))
+    for R in (1, 5, 16):
+        F = [f32(synth.random_dense((d, R), 2, 60 + m).numpy()) for m, d in enumerate(dims)]
+        for mode in range(3):
+            want, norm = oracle.mttkrp(c, v, dims, mode, F)
+            out = torch.full((dims[mode], R), float("nan"), dtype=torch.float32, device="cuda")
+            comet.mttkrp(X, mode, [None if m == mode else dev32(f) for m, f in enumerate(F)], out)
+            check(out, want, norm, f"mttkrp fp32 mode {mode} R={R}")
+
+
 @pytest.mark.parametrize("attr,order", [((D, CU), 2), ((CU, CU), 2), ((CN, S), 2), ((CU, CU, CU), 3), ((CN, S, S), 3)])
 def test_pack_fp32_bit_exact(attr, order):
     dims = (300, 200) if order == 2 else (50, 40, 30)

@@ -164,3 +164,27 @@ def test_full_c5_mttkrp(attr):
     rel = assert_close(out[torch.from_numpy(rows).cuda()], want, norm, what=f"C5 mttkrp {attr}")
     print(f"C5 {attr} worst normalised error {rel:.2e}")
     assert bool((out[counts == 0] == 0).all())                                     # rows without entries are +0
+
+
+@pytest.mark.parametrize("attr", [(CN, S, S), (CU, CU, CU)])
+@pytest.mark.parametrize("mode", [1, 2])
+def test_full_c5_mttkrp_non_root_modes(attr, mode):
+    """Modes 1 and 2 on the tensor packed with mode 0 first (atomic accumulation), sampled rows."""
+    case = synth.make(5, device="cuda")
+    X = comet.pack(case.coords, case.val, case.dims, (0, 1, 2), attr)
+    R = case.R
+    F = [synth.random_dense((d, R), case.seed, 70 + m, device="cuda") for m, d in enumerate(case.dims)]
+    out = torch.full((case.dims[mode], R), float("nan"), dtype=torch.float64, device="cuda")
+    comet.mttkrp(X, mode, [None if m == mode else f for m, f in enumerate(F)], out)
+    assert not bool(torch.isnan(out).any()), "an output row was not written"
+    counts = torch.bincount(case.coords[mode].long(), minlength=case.dims[mode])
+    heavy = torch.topk(counts, 4).indices.tolist()
+    empty = torch.nonzero(counts == 0)[:4, 0].tolist()
+    rows = sample_rows(case.dims[mode], 5, always=heavy + empty + [0, case.dims[mode] - 1])
+    del X
+    c, v = host(case)
+    want, norm = oracle.mttkrp(c, v, case.dims, mode, [None if m == mode else f.cpu().numpy() for m, f in enumerate(F)],
+                               rows=rows)
+    rel = assert_close(out[torch.from_numpy(rows).cuda()], want, norm, what=f"C5 mttkrp mode {mode} {attr}")
+    print(f"C5 mode {mode} {attr} worst normalised error {rel:.2e}")
+    assert bool((out[counts == 0] == 0).all())
