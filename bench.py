@@ -252,6 +252,22 @@ def per_kernel(comet, handle, steps, warm, peak):
             "pack_us_median": round(pmed * 1e3, 1), "pack_compulsory_bytes": pbytes,
             "pack_GBps": round(pbytes / pmed / 1e6, 1),
         })
+        if op == "mttkrp" and fmt == "csf":
+            # the two other modes of the SAME packed tensor (atomic accumulation, nothing re-packed)
+            for mode in (1, 2):
+                Fm = [synth.random_dense((d, case.R), case.seed, 70 + m, device="cuda") for m, d in enumerate(case.dims)]
+                Fm[mode] = None
+                Am = torch.empty((case.dims[mode], case.R), dtype=torch.float64, device="cuda")
+                med, mn = cuda_time(lambda: comet.mttkrp(T, mode, Fm, Am), steps, warm)
+                out.append({
+                    "workload": case.name, "op": f"mttkrp-mode{mode + 1}-of-root-packed", "format": fmt, "nnz": case.nnz,
+                    "segments": int(T.c.crd_len[1]), "us_median": round(med * 1e3, 2), "us_min": round(mn * 1e3, 2),
+                    "compulsory_bytes": nbytes, "GBps": round(nbytes / med / 1e6, 1),
+                    "frac_of_8000": round(nbytes / med / 1e6 / NOMINAL_GBS, 4),
+                    "frac_of_peak": round(nbytes / med / 1e6 / peak, 4), "GFLOPs": round(flops / med / 1e6, 1),
+                    "l2": "inputs larger than L2", "accumulation": "atomic adds (order not fixed)",
+                })
+                del Fm, Am
         del T
         torch.cuda.empty_cache()
     return out

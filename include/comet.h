@@ -144,12 +144,17 @@ comet_status_t comet_spmm(comet_handle_t handle, const comet_sptensor_t *A, cons
                           void *C, int64_t ldc, void *stream);
 
 /* TTV  Y = X x_n v  (SpTTV definition; `mode` = n, 0-based, must be the mode of X's LAST level).
- * X: 3 levels, [CU,CU,CU] (CSF; a COO tensor is first re-packed with comet_pack). The result is sparse,
- * one order lower:
+ * X: 3 levels, [CU,CU,CU] (CSF) or [CN,S,S] (sorted COO). The result is sparse, one order lower:
  * comet_ttv_symbolic builds its structure over (mode_order[0], mode_order[1]) with level attributes
  * h_out_attr = {D,CU} (CSR) or {CU,CU} (DCSR); values are then (re)computed by comet_ttv, which
  * writes only Y->val. The structure depends on X's structure alone, never on values. Y owns its
- * arrays; X need not outlive it. */
+ * arrays; X need not outlive it.
+ * COO input: the fibers (runs of equal leading coordinate pairs) are not stored, so the symbolic call
+ * derives them from the sorted coordinates (head flags, two scans, one synchronisation to read the
+ * counts) and leaves the fiber boundary array (#fibers + 1 positions into X's entries) in the first
+ * level slot BEYOND Y's own levels: Y->pos[2] / pos_len[2] for TTV, Y->pos[3] / pos_len[3] for TTM.
+ * The numeric call reads it from there, so it must be given the Y that was built from this X
+ * (anything else is COMET_ERR_INVALID_ARG when the sizes disagree). The slot is owned by Y. */
 comet_status_t comet_ttv_symbolic(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode,
                                   const int32_t *h_out_attr, void *stream, comet_sptensor_t *Y);
 comet_status_t comet_ttv(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode, const void *v,
@@ -159,7 +164,7 @@ comet_status_t comet_ttv(comet_handle_t handle, const comet_sptensor_t *X, int32
  * mode n is replaced by r in place. `mode` must be the mode of X's last level. The result is
  * semi-sparse [CU,CU,D]: its two sparse levels equal X's first two levels and every stored fiber is
  * a dense row of R values (val is #fibers x R, row-major). comet_ttm_symbolic builds that structure,
- * comet_ttm writes only Y->val. */
+ * comet_ttm writes only Y->val. Formats of X as for comet_ttv (COO: see the note there). */
 comet_status_t comet_ttm_symbolic(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode, int64_t R,
                                   void *stream, comet_sptensor_t *Y);
 comet_status_t comet_ttm(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode, const void *U, int64_t R,

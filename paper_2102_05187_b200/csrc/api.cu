@@ -179,9 +179,122 @@ static comet_status_t check_last_mode(const comet_sptensor_t *X, int32_t mode) {
   comet_status_t st = check_tensor(X, 3);
   if (st != COMET_OK) return st;
   if (mode < 0 || mode > 2) return COMET_ERR_INVALID_ARG;
-  if (!is_fmt(X, 3, COMET_CU, COMET_CU, COMET_CU)) return COMET_ERR_UNSUPPORTED_FORMAT;
+  if (!is_fmt(X, 3, COMET_CU, COMET_CU, COMET_CU) && !is_fmt(X, 3, COMET_CN, COMET_S, COMET_S))
+    return COMET_ERR_UNSUPPORTED_FORMAT;
   if (X->mode_order[2] != mode) return COMET_ERR_UNSUPPORTED_FORMAT;   // re-pack with the contracted mode last
   return COMET_OK;
+}
+
+// ---- sorted COO [CN,S,S] as input of TTV / TTM -------------------------------------------------------
+// The kernels want the fibers of the two leading modes: where each fiber ends in the entry list, and
+// the (slice, fiber) coordinates of the result's structure. A sorted COO tensor has them implicitly: a
+// fiber starts where (crd0, crd1) changes, a slice where crd0 changes. The symbolic call derives the two
+// upper CSF levels from those head flags (flags -> two exclusive scans -> one read of the counts ->
+// compaction); the leaf level is the COO tensor's own third coordinate array and values, untouched.
+__global__ void coo_heads_kernel(const int32_t *__restrict__ c0, const int32_t *__restrict__ c1, int64_t n,
+                                 uint32_t *__restrict__ fiber_head, uint32_t *__restrict__ slice_head) {
+  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= n) return;
+  const bool s = p == 0 || c0[p] != c0[p - 1];
+  fiber_head[p] = (s || c1[p] != c1[p - 1]) ? 1u : 0u;
+  slice_head[p] = s ? 1u : 0u;
+}
+
+// fiber_rank / slice_rank: exclusive scans of the head flags (rank of the fiber / slice an entry opens)
+__global__ void coo_levels_kernel(const int32_t *__restrict__ c0, const int32_t *__restrict__ c1, int64_t n,
+                                  const uint32_t *__restrict__ fiber_rank, const uint32_t *__restrict__ slice_rank,
+                                  int64_t S, int64_t F, int32_t *__restrict__ pos0, int32_t *__restrict__ crd0,
+                                  int32_t *__restrict__ pos1, int32_t *__restrict__ crd1, int32_t *__restrict__ pos2) {
+  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (p == 0) { pos0[0] = 0; pos0[1] = (int32_t)S; pos1[S] = (int32_t)F; pos2[F] = (int32_t)n; }
+  if (p >= n) return;
+  const bool s = p == 0 || c0[p] != c0[p - 1];
+  if (s || c1[p] != c1[p - 1]) {
+    const uint32_t f = fiber_rank[p];
+    crd1[f] = c1[p];
+    pos2[f] = (int32_t)p;
+    if (s) {
+      const uint32_t sl = slice_rank[p];
+      crd0[sl] = c0[p];
+      pos1[sl] = (int32_t)f;
+    }
+  }
+}
+
+struct CooAsCsf {
+  comet_sptensor_t t;       // CSF-shaped view: derived upper levels + the COO tensor's leaf arrays
+  int32_t *pos2;            // fiber boundaries (F + 1); handed to the result, which the numeric call reads
+  void *temps[4];           // pos0, crd0, pos1, crd1 of the view
+};
+
+static void coo_view_release(Context *ctx, CooAsCsf *v, bool keep_pos2, cudaStream_t s) {
+  for (int i = 0; i < 4; ++i) if (v->temps[i]) ctx_free(ctx, v->temps[i], s);
+  if (!keep_pos2 && v->pos2) ctx_free(ctx, v->pos2, s);
+}
+
+static comet_status_t coo_as_csf(Context *ctx, const comet_sptensor_t *X, cudaStream_t s, CooAsCsf *v) {
+  memset(v, 0, sizeof(*v));
+  const int64_t n = X->nnz;
+  int64_t S = 0, F = 0;
+  uint32_t *fiber_rank = nullptr, *slice_rank = nullptr, *tmp = nullptr;
+  comet_status_t st = COMET_OK;
+  if (n > 0) {
+    fiber_rank = (uint32_t *)ctx_alloc(ctx, (size_t)n * 4, s);
+    slice_rank = (uint32_t *)ctx_alloc(ctx, (size_t)n * 4, s);
+    tmp = (uint32_t *)ctx_alloc(ctx, (size_t)scan_tmp_words(n) * 4, s);
+    if (!fiber_rank || !slice_rank || !tmp) st = COMET_ERR_ALLOC;
+    uint32_t *d_counts = reinterpret_cast<uint32_t *>(ctx->d_status) + 8;
+    if (st == COMET_OK) {
+      coo_heads_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(X->crd[0], X->crd[1], n, fiber_rank, slice_rank);
+      ctx->launches += 1;
+      st = exclusive_scan(ctx, fiber_rank, fiber_rank, n, tmp, d_counts, s);
+    }
+    if (st == COMET_OK) st = exclusive_scan(ctx, slice_rank, slice_rank, n, tmp, d_counts + 1, s);
+    if (st == COMET_OK) {
+      cudaError_t e = cudaMemcpyAsync(ctx->h_pinned, d_counts, 2 * sizeof(uint32_t), cudaMemcpyDeviceToHost, s);
+      if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+      if (e != cudaSuccess) st = cuda_fail(ctx, e);
+      F = reinterpret_cast<uint32_t *>(ctx->h_pinned)[0];
+      S = reinterpret_cast<uint32_t *>(ctx->h_pinned)[1];
+    }
+  }
+  int32_t *pos0 = nullptr, *crd0 = nullptr, *pos1 = nullptr, *crd1 = nullptr;
+  if (st == COMET_OK) {
+    v->temps[0] = pos0 = (int32_t *)ctx_alloc(ctx, 2 * 4, s);
+    v->temps[1] = crd0 = (int32_t *)ctx_alloc(ctx, (size_t)(S > 0 ? S : 1) * 4, s);
+    v->temps[2] = pos1 = (int32_t *)ctx_alloc(ctx, (size_t)(S + 1) * 4, s);
+    v->temps[3] = crd1 = (int32_t *)ctx_alloc(ctx, (size_t)(F > 0 ? F : 1) * 4, s);
+    v->pos2 = (int32_t *)ctx_alloc(ctx, (size_t)(F + 1) * 4, s);
+    if (!pos0 || !crd0 || !pos1 || !crd1 || !v->pos2) st = COMET_ERR_ALLOC;
+  }
+  if (st == COMET_OK) {
+    coo_levels_kernel<<<(unsigned)ceil_div(n > 0 ? n : 1, 256), 256, 0, s>>>(X->crd[0], X->crd[1], n, fiber_rank,
+                                                                           slice_rank, S, F, pos0, crd0, pos1, crd1,
+                                                                           v->pos2);
+    ctx->launches += 1;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) st = cuda_fail(ctx, e);
+  }
+  if (fiber_rank) ctx_free(ctx, fiber_rank, s);
+  if (slice_rank) ctx_free(ctx, slice_rank, s);
+  if (tmp) ctx_free(ctx, tmp, s);
+  if (st != COMET_OK) { coo_view_release(ctx, v, false, s); memset(v, 0, sizeof(*v)); return st; }
+  comet_sptensor_t *t = &v->t;
+  *t = *X;
+  t->owner = nullptr;
+  t->attr[0] = t->attr[1] = t->attr[2] = COMET_CU;
+  t->pos[0] = pos0; t->pos_len[0] = 2; t->crd[0] = crd0; t->crd_len[0] = S;
+  t->pos[1] = pos1; t->pos_len[1] = S + 1; t->crd[1] = crd1; t->crd_len[1] = F;
+  t->pos[2] = v->pos2; t->pos_len[2] = F + 1;          // crd[2], crd_len[2], val, nnz stay the COO tensor's
+  return COMET_OK;
+}
+
+// The fiber boundaries of a COO input travel with the result: level slot `slot` of Y (beyond Y's own
+// levels) holds pos2, owned by Y. The numeric call finds them there.
+static void stash_fiber_pos(comet_sptensor_t *Y, Owner *o, int slot, CooAsCsf *v) {
+  o->blocks[o->count++] = v->pos2;
+  Y->pos[slot] = v->pos2;
+  Y->pos_len[slot] = v->t.pos_len[2];
 }
 
 // Copies X's two upper levels into Y (levels 0 and 1), device to device.
@@ -212,8 +325,15 @@ extern "C" comet_status_t comet_ttv_symbolic(comet_handle_t handle, const comet_
   Context *ctx = reinterpret_cast<Context *>(handle);
   cudaStream_t s = (cudaStream_t)stream;
   memset(Y, 0, sizeof(*Y));
+  CooAsCsf view;
+  const bool from_coo = X->attr[0] == COMET_CN;
+  if (from_coo) {
+    st = coo_as_csf(ctx, X, s, &view);
+    if (st != COMET_OK) return st;
+    X = &view.t;
+  }
   Owner *o = static_cast<Owner *>(owner_new());
-  if (!o) return COMET_ERR_ALLOC;
+  if (!o) { if (from_coo) coo_view_release(ctx, &view, false, s); return COMET_ERR_ALLOC; }
   const int64_t S = X->crd_len[0], F = X->crd_len[1];
   const int64_t rows = X->dims[X->mode_order[0]];
   Y->order = 2;
@@ -248,6 +368,10 @@ extern "C" comet_status_t comet_ttv_symbolic(comet_handle_t handle, const comet_
     Y->val = owned_alloc(ctx, o, (size_t)F * elem_size(X->dtype), s);
     if (!Y->val) st = COMET_ERR_ALLOC;
   }
+  if (from_coo) {
+    if (st == COMET_OK) stash_fiber_pos(Y, o, 2, &view);
+    coo_view_release(ctx, &view, st == COMET_OK, s);
+  }
   if (st != COMET_OK) { release(ctx, o, s); memset(Y, 0, sizeof(*Y)); return st; }
   Y->owner = o;
   return COMET_OK;
@@ -258,12 +382,17 @@ extern "C" comet_status_t comet_ttv(comet_handle_t handle, const comet_sptensor_
   if (!handle || !v || !Y) return COMET_ERR_INVALID_ARG;
   comet_status_t st = check_last_mode(X, mode);
   if (st != COMET_OK) return st;
-  if (Y->order != 2 || Y->nnz != X->crd_len[1] || (Y->nnz > 0 && !Y->val)) return COMET_ERR_INVALID_ARG;
+  // fibers: X's level-2 pos for CSF; for COO the boundaries that the symbolic call left in Y's spare slot
+  const bool from_coo = X->attr[0] == COMET_CN;
+  const int32_t *fiber_pos = from_coo ? Y->pos[2] : X->pos[2];
+  const int64_t F = from_coo ? Y->pos_len[2] - 1 : X->crd_len[1];
+  if (!fiber_pos || F < 0) return COMET_ERR_INVALID_ARG;
+  if (Y->order != 2 || Y->nnz != F || (Y->nnz > 0 && !Y->val)) return COMET_ERR_INVALID_ARG;
   if (Y->dtype != X->dtype) return COMET_ERR_INVALID_ARG;
   if (misaligned(v, X->dtype)) return COMET_ERR_MISALIGNED;
   Context *ctx = reinterpret_cast<Context *>(handle);
-  return seg_dot(ctx, X->dtype, X->pos[2] + 1, X->crd[2], X->val, X->crd_len[1], X->nnz, v, X->dims[mode], Y->val, nullptr,
-                 X->crd_len[1], (cudaStream_t)stream);
+  return seg_dot(ctx, X->dtype, fiber_pos + 1, X->crd[2], X->val, F, X->nnz, v, X->dims[mode], Y->val, nullptr, F,
+                 (cudaStream_t)stream);
 }
 
 extern "C" comet_status_t comet_ttm_symbolic(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode,
@@ -275,8 +404,15 @@ extern "C" comet_status_t comet_ttm_symbolic(comet_handle_t handle, const comet_
   Context *ctx = reinterpret_cast<Context *>(handle);
   cudaStream_t s = (cudaStream_t)stream;
   memset(Y, 0, sizeof(*Y));
+  CooAsCsf view;
+  const bool from_coo = X->attr[0] == COMET_CN;
+  if (from_coo) {
+    st = coo_as_csf(ctx, X, s, &view);
+    if (st != COMET_OK) return st;
+    X = &view.t;
+  }
   Owner *o = static_cast<Owner *>(owner_new());
-  if (!o) return COMET_ERR_ALLOC;
+  if (!o) { if (from_coo) coo_view_release(ctx, &view, false, s); return COMET_ERR_ALLOC; }
   const int64_t F = X->crd_len[1];
   Y->order = 3;
   Y->dtype = X->dtype;
@@ -297,6 +433,10 @@ extern "C" comet_status_t comet_ttm_symbolic(comet_handle_t handle, const comet_
       if (e != cudaSuccess) st = cuda_fail(ctx, e);
     }
   }
+  if (from_coo) {
+    if (st == COMET_OK) stash_fiber_pos(Y, o, 3, &view);
+    coo_view_release(ctx, &view, st == COMET_OK, s);
+  }
   if (st != COMET_OK) { release(ctx, o, s); memset(Y, 0, sizeof(*Y)); return st; }
   Y->owner = o;
   return COMET_OK;
@@ -307,12 +447,15 @@ extern "C" comet_status_t comet_ttm(comet_handle_t handle, const comet_sptensor_
   if (!handle || !U || !Y || R < 1 || ldu < R) return COMET_ERR_INVALID_ARG;
   comet_status_t st = check_last_mode(X, mode);
   if (st != COMET_OK) return st;
-  const int64_t F = X->crd_len[1];
+  const bool from_coo = X->attr[0] == COMET_CN;
+  const int32_t *fiber_pos = from_coo ? Y->pos[3] : X->pos[2];
+  const int64_t F = from_coo ? Y->pos_len[3] - 1 : X->crd_len[1];
+  if (!fiber_pos || F < 0) return COMET_ERR_INVALID_ARG;
   if (Y->order != 3 || Y->nnz != F * R || (Y->nnz > 0 && !Y->val)) return COMET_ERR_INVALID_ARG;
   if (Y->dtype != X->dtype) return COMET_ERR_INVALID_ARG;
   if (misaligned(U, X->dtype)) return COMET_ERR_MISALIGNED;
   Context *ctx = reinterpret_cast<Context *>(handle);
-  return seg_gather(ctx, X->dtype, X->pos[2] + 1, X->crd[2], X->val, F, X->nnz, U, ldu, R, Y->val, R, nullptr, F,
+  return seg_gather(ctx, X->dtype, fiber_pos + 1, X->crd[2], X->val, F, X->nnz, U, ldu, R, Y->val, R, nullptr, F,
                     (cudaStream_t)stream);
 }
 

@@ -37,6 +37,12 @@ comet_status_t mttkrp_scatter(Context *ctx, int dtype, int kind, const int32_t *
                               int64_t R, void *out, int64_t ldo, cudaStream_t stream);
 
 comet_status_t zero_rows(Context *ctx, void *C, int dtype, int64_t rows, int64_t R, int64_t ldc, cudaStream_t stream);
+// Exclusive scan of uint32 words in three launches (tile sums, scan of the sums, apply); defined in pack.cu.
+// `out` may alias `in`; `tmp` holds scan_tmp_words(n) words; `total` (device, optional) receives the sum.
+int64_t scan_tmp_words(int64_t n);
+comet_status_t exclusive_scan(Context *ctx, const uint32_t *in, uint32_t *out, int64_t n, uint32_t *tmp,
+                              uint32_t *total, cudaStream_t s);
+
 int32_t choose_tile_items(int64_t total_items, int workers_per_block);
 
 // Block list of a library-owned tensor (what comet_sptensor_free releases).

@@ -142,9 +142,11 @@ __global__ void scan_apply_kernel(const uint32_t *__restrict__ in, int64_t n, co
   }
 }
 
-// out = exclusive scan of in (may alias); tmp holds ceil(n / kScanTile) words; total (device) optional.
-static comet_status_t exclusive_scan(Context *ctx, const uint32_t *in, uint32_t *out, int64_t n, uint32_t *tmp,
-                                     uint32_t *total, cudaStream_t s) {
+// out = exclusive scan of in (may alias); tmp holds scan_tmp_words(n) words; total (device) optional.
+int64_t scan_tmp_words(int64_t n) { return ceil_div(n > 0 ? n : 1, kScanTile) + 1; }
+
+comet_status_t exclusive_scan(Context *ctx, const uint32_t *in, uint32_t *out, int64_t n, uint32_t *tmp,
+                              uint32_t *total, cudaStream_t s) {
   if (n <= 0) {
     if (total) COMET_CUDA_TRY(ctx, cudaMemsetAsync(total, 0, sizeof(uint32_t), s));
     return COMET_OK;

@@ -178,6 +178,58 @@ def test_ttv_ttm(dims, nnz, seed, mode, tile_items, seg_dot_path):
 
 @pytest.mark.parametrize("dims,nnz,seed", TENSOR_CASES)
 @pytest.mark.parametrize("mode", [0, 1, 2])
+def test_ttv_ttm_from_sorted_coo(dims, nnz, seed, mode, tile_items):
+    """[CN,S,S] input: the fibers are derived from the sorted coordinates in the symbolic call; values and
+    structure must equal those from the CSF tensor of the same entries."""
+    coords, val = synth.random_coo(dims, nnz, seed)
+    c, v = _np(coords), val.numpy()
+    kept = [m for m in range(3) if m != mode]
+    mode_order = (kept[0], kept[1], mode)
+    X = upload_packed(oracle.pack(c, v, dims, mode_order, (CN, S, S)))
+    csf = oracle.pack(c, v, dims, mode_order, (CU, CU, CU))
+    vec = synth.random_dense((dims[mode],), seed).numpy()
+    keys, want, norm = oracle.ttv(c, v, dims, mode, vec)
+    for out_attr in [(D, CU), (CU, CU)]:
+        Y = comet.ttv_symbolic(X, mode, out_attr)
+        comet.validate(Y)
+        Y.val.fill_(float("nan"))
+        comet.ttv(X, mode, dev(vec), Y)
+        assert_close(Y.val, want, norm, what="coo ttv")
+        ka, kb = keys // dims[kept[1]], keys % dims[kept[1]]
+        ref = oracle.pack([ka, kb], np.ones(len(keys)), (dims[kept[0]], dims[kept[1]]), (0, 1), out_attr)
+        for l in range(2):
+            assert_equal_arrays(Y.pos(l), ref.pos[l], f"coo ttv pos{l}")
+            assert_equal_arrays(Y.crd(l), ref.crd[l], f"coo ttv crd{l}")
+        comet.ttv(X, mode, dev(vec), Y)                                  # the numeric phase can be repeated
+        assert_close(Y.val, want, norm, what="coo ttv again")
+    for R in (1, 16, 5):
+        U = synth.random_dense((dims[mode], R), seed + 1).numpy()
+        _, wantm, normm = oracle.ttm(c, v, dims, mode, U)
+        Z = comet.ttm_symbolic(X, mode, R)
+        Z.val.fill_(float("nan"))
+        comet.ttm(X, mode, dev(U), Z)
+        assert_close(Z.val.reshape(-1, R), wantm, normm, what=f"coo ttm R={R}")
+        assert Z.attr == (CU, CU, D)
+        for l in range(2):
+            assert_equal_arrays(Z.pos(l), csf.pos[l], f"coo ttm pos{l}")
+            assert_equal_arrays(Z.crd(l), csf.crd[l], f"coo ttm crd{l}")
+        assert Z.pos(2).tolist() == [R]
+
+
+def test_ttv_numeric_phase_rejects_a_result_built_for_another_tensor():
+    dims = (12, 11, 10)
+    coords, val = synth.random_coo(dims, 400, 3)
+    c, v = _np(coords), val.numpy()
+    Xcoo = upload_packed(oracle.pack(c, v, dims, (0, 1, 2), (CN, S, S)))
+    Xcsf = upload_packed(oracle.pack(c, v, dims, (0, 1, 2), (CU, CU, CU)))
+    Y = comet.ttv_symbolic(Xcsf, 2)            # carries no fiber boundaries: a COO numeric call cannot use it
+    with pytest.raises(comet.CometError) as e:
+        comet.ttv(Xcoo, 2, dev(np.ones(10)), Y)
+    assert e.value.status == -1
+
+
+@pytest.mark.parametrize("dims,nnz,seed", TENSOR_CASES)
+@pytest.mark.parametrize("mode", [0, 1, 2])
 @pytest.mark.parametrize("attr", [(CN, S, S), (CU, CU, CU)])
 def test_mttkrp(dims, nnz, seed, mode, attr, tile_items):
     coords, val = synth.random_coo(dims, nnz, seed)

@@ -188,3 +188,23 @@ def test_full_c5_mttkrp_non_root_modes(attr, mode):
     rel = assert_close(out[torch.from_numpy(rows).cuda()], want, norm, what=f"C5 mttkrp mode {mode} {attr}")
     print(f"C5 mode {mode} {attr} worst normalised error {rel:.2e}")
     assert bool((out[counts == 0] == 0).all())
+
+
+def test_full_c3_c4_from_sorted_coo_equal_the_csf_results():
+    """[CN,S,S] inputs at full size: the derived fibers must reproduce the CSF tensor's structure, and the
+    values (same kernels, same boundaries) must be bit-identical to the CSF results, which the tests above
+    check against the oracle."""
+    for cfg in (3, 4):
+        case = synth.make(cfg, device="cuda")
+        Xs = comet.pack(case.coords, case.val, case.dims, (0, 1, 2), (CU, CU, CU))
+        Xc = comet.pack(case.coords, case.val, case.dims, (0, 1, 2), (CN, S, S))
+        if cfg == 3:
+            Ys, Yc = comet.ttv(Xs, 2, case.dense["v"]), comet.ttv(Xc, 2, case.dense["v"])
+        else:
+            Ys, Yc = comet.ttm(Xs, 2, case.dense["U"]), comet.ttm(Xc, 2, case.dense["U"])
+        assert Yc.c.nnz == Ys.c.nnz and Yc.attr == Ys.attr and Yc.dims == Ys.dims
+        for l in range(2):
+            assert torch.equal(Yc.pos(l), Ys.pos(l)) and torch.equal(Yc.crd(l), Ys.crd(l))
+        assert torch.equal(Yc.val, Ys.val)
+        del Xs, Xc, Ys, Yc, case
+        torch.cuda.empty_cache()
