@@ -393,17 +393,29 @@ def mttkrp(X: SpTensor, mode: int, factors, out: torch.Tensor | None = None) -> 
     return out
 
 
+_copy_stream = None
+
+
 def spmm_from_host(h_coords, h_val, dims, h_B, h_out, handle: Handle | None = None):
     """The whole SpMM path from HOST buffers: copies the COO entries and B to the device (pinned host
     tensors make the copies asynchronous), packs to CSR, multiplies, and copies C back into `h_out`.
-    Returns after the result has landed in `h_out`."""
+    B travels on a second stream, so the packing kernels run while B is still crossing the bus; the
+    multiplication waits for it. Returns after the result has landed in `h_out`."""
+    global _copy_stream
     handle = handle or default_handle()
+    cur = torch.cuda.current_stream()
+    if _copy_stream is None or _copy_stream.device != cur.device:
+        _copy_stream = torch.cuda.Stream(device=cur.device)
     coords = [c.to("cuda", non_blocking=True) for c in h_coords]
     val = h_val.to("cuda", non_blocking=True)
-    B = h_B.to("cuda", non_blocking=True)
+    _copy_stream.wait_stream(cur)                     # the bus serves the COO entries first
+    with torch.cuda.stream(_copy_stream):
+        B = h_B.to("cuda", non_blocking=True)
     A = pack(coords, val, dims, (0, 1), (D, CU), handle)
+    cur.wait_stream(_copy_stream)
+    B.record_stream(cur)
     C_dev = spmm(A, B)
     h_out.copy_(C_dev, non_blocking=True)
-    torch.cuda.current_stream().synchronize()
+    cur.synchronize()
     A.free()
     return h_out
