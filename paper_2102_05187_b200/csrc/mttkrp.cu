@@ -25,6 +25,7 @@
 #define COMET_MINB_CSF 4
 #endif
 
+
 namespace comet {
 
 struct MttkrpArgs {
@@ -150,7 +151,10 @@ struct CsfPolicy {
   T *ocol;
   const T *val;
   double tac[CPL][VEC], aac[CPL][VEC];   // open fiber sum, open slice sum
-  T prow[CPL][VEC];                      // P row of the open fiber, fetched when the fiber opened
+  T prow[CPL][VEC];                      // P row of the open fiber
+  T pnext[CPL][VEC];                     // P row of the fiber after it: fetched one fiber ahead, so that a fold
+                                         // never waits for its gather (fibers are a few entries long)
+  int32_t end1;                          // leaf position where the fiber after the open one ends
   // cursors instead of indices: the per-fiber path is executed once per fiber and per worker (divergently),
   // so it is kept to pointer bumps and 32-bit compares
   const int32_t *endp;                   // seg_end2 + open fiber
@@ -170,7 +174,7 @@ struct CsfPolicy {
 #pragma unroll
     for (int t = 0; t < CPL; ++t)
 #pragma unroll
-      for (int k = 0; k < VEC; ++k) prow[t][k] = (T)0;
+      for (int k = 0; k < VEC; ++k) { prow[t][k] = (T)0; pnext[t][k] = (T)0; }
     pcol = reinterpret_cast<const char *>(static_cast<const T *>(a.P) + ln.col0);
     qcol = reinterpret_cast<const char *>(static_cast<const T *>(a.Q) + ln.col0);
     ldp_bytes = (int32_t)(a.ldp * sizeof(T));
@@ -181,13 +185,15 @@ struct CsfPolicy {
     c1p = a.crd1 + f0;
     fibers_left = (int32_t)(a.F - f0);
     next_end = fibers_left > 0 ? __ldg(endp) : -1;
+    end1 = fibers_left > 1 ? __ldg(endp + 1) : -1;
     rel_end = next_end - base;
     to_slice_end = s < a.S ? (int32_t)(__ldg(a.pos1 + s + 1) - f0) : -1;
-    open_fiber();
+    if (fibers_left > 0) ln.gather(reinterpret_cast<const T *>(pcol + (int64_t)__ldg(c1p) * ldp_bytes), prow);
+    fetch_ahead();
   }
   __device__ __forceinline__ int64_t fiber() const { return a.F - fibers_left; }
-  __device__ __forceinline__ void open_fiber() {         // start fetching the P row the fiber will be folded with
-    if (fibers_left > 0) ln.gather(reinterpret_cast<const T *>(pcol + (int64_t)__ldg(c1p) * ldp_bytes), prow);
+  __device__ __forceinline__ void fetch_ahead() {        // start fetching the P row of the fiber after the open one
+    if (fibers_left > 1) ln.gather(reinterpret_cast<const T *>(pcol + (int64_t)__ldg(c1p + 1) * ldp_bytes), pnext);
   }
   __device__ __forceinline__ void fetch(int32_t j, Entry16 &e, int32_t &) const {
     e.v = (double)ld_stream(val + j);
@@ -223,9 +229,14 @@ struct CsfPolicy {
     ++endp;
     ++c1p;
     --fibers_left;
-    next_end = fibers_left > 0 ? __ldg(endp) : -1;
+    next_end = end1;                                     // loaded one fiber ago
+    end1 = fibers_left > 1 ? __ldg(endp + 1) : -1;
     rel_end = next_end - base;
-    open_fiber();
+#pragma unroll
+    for (int t = 0; t < CPL; ++t)
+#pragma unroll
+      for (int k = 0; k < VEC; ++k) prow[t][k] = pnext[t][k];
+    fetch_ahead();
     if (--to_slice_end == 0) close_slice();
   }
   __device__ __forceinline__ void consume(int q, double v, int32_t, Slot &sl) {
