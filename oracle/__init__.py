@@ -34,6 +34,7 @@ def lib():
     if _lib is None:
         _lib = C.CDLL(_build())
         _lib.oracle_fiber_keys.restype = C.c_int64
+        _lib.oracle_fiber_keys_n.restype = C.c_int64
     return _lib
 
 
@@ -101,6 +102,40 @@ def fiber_keys(coords, dims, mode):
     if n < 0:
         raise OracleError(n, "fiber_keys")
     return keys[:n].copy()
+
+
+def _coord_ptrs(c):
+    return (C.c_void_p * len(c))(*[x.ctypes.data for x in c])
+
+
+def fiber_keys_n(coords, dims, mode):
+    """Sorted distinct keys of the kept modes (linearised in increasing mode order) for tensors of order 2..4."""
+    c = [_i32(x) for x in coords]
+    keys = np.zeros(max(1, len(c[0])), dtype=np.int64)
+    n = lib().oracle_fiber_keys_n(C.c_int(len(dims)), C.c_int64(len(c[0])), _coord_ptrs(c), _p(_i64(dims)),
+                                  C.c_int(mode), _p(keys))
+    if n < 0:
+        raise OracleError(n, "fiber_keys_n")
+    return keys[:n].copy()
+
+
+def ttm_n(coords, val, dims, mode, U, keys=None):
+    """Y = X x_mode U for tensors of order 2..4 (U is I_mode x R; one column = tensor times vector).
+    Returns (keys, Y[nkeys, R], normaliser)."""
+    c = [_i32(x) for x in coords]
+    val, U = _f64(val), _f64(U)
+    if U.ndim == 1:
+        U = U.reshape(-1, 1)
+    R = U.shape[1]
+    keys = fiber_keys_n(coords, dims, mode) if keys is None else _i64(keys)
+    Y = np.zeros((len(keys), R))
+    Yn = np.zeros((len(keys), R))
+    rc = lib().oracle_ttm_n(C.c_int(len(dims)), C.c_int64(len(val)), _coord_ptrs(c), _p(val), _p(_i64(dims)),
+                            C.c_int(mode), _p(U), C.c_int64(R), C.c_int64(R), _p(keys), C.c_int64(len(keys)), _p(Y),
+                            _p(Yn))
+    if rc:
+        raise OracleError(rc, "ttm_n")
+    return keys, Y, Yn
 
 
 def ttv(coords, val, dims, mode, v, keys=None):

@@ -182,6 +182,56 @@ int oracle_ttm(int64_t nnz, const int32_t *c0, const int32_t *c1, const int32_t 
   return ORACLE_OK;
 }
 
+/* ------------------------------------------------------------------------------- TTV / TTM, any order
+ * The same two definitions for a tensor of `order` modes (2 <= order <= 4): the mode-n product
+ * contracts mode n and keeps the others. An output fiber is identified by the kept coordinates,
+ * linearised in increasing mode order (the last kept mode varies fastest): key = sum c_m * stride_m.
+ * `coords` holds one pointer per mode. Plain loops over the raw COO entries, long-double sums. */
+static int64_t kept_key(int order, const int32_t *const *c, const int64_t *dims, int mode, int64_t e) {
+  int64_t key = 0;
+  for (int m = 0; m < order; ++m)
+    if (m != mode) key = key * dims[m] + (int64_t)c[m][e];
+  return key;
+}
+
+int64_t oracle_fiber_keys_n(int order, int64_t nnz, const int32_t *const *coords, const int64_t *dims, int mode,
+                            int64_t *keys) {
+  if (order < 2 || order > 4 || mode < 0 || mode >= order) return ORACLE_ERR_ARG;
+  for (int64_t e = 0; e < nnz; ++e) keys[e] = kept_key(order, coords, dims, mode, e);
+  qsort(keys, (size_t)nnz, sizeof(int64_t), cmp_i64);
+  int64_t n = 0;
+  for (int64_t e = 0; e < nnz; ++e)
+    if (e == 0 || keys[e] != keys[e - 1]) keys[n++] = keys[e];
+  return n;
+}
+
+/* U is I_mode x R (ldu >= R); R = 1 with ldu = 1 is the tensor-times-vector product. */
+int oracle_ttm_n(int order, int64_t nnz, const int32_t *const *coords, const double *val, const int64_t *dims,
+                 int mode, const double *U, int64_t R, int64_t ldu, const int64_t *keys, int64_t nkeys, double *Y,
+                 double *Ynorm) {
+  if (order < 2 || order > 4 || mode < 0 || mode >= order || nnz < 0 || nkeys < 0 || R < 0 || ldu < R)
+    return ORACLE_ERR_ARG;
+  size_t cells = (size_t)nkeys * (size_t)R;
+  long double *acc = (long double *)calloc(cells ? cells : 1, sizeof(long double));
+  if (!acc) return ORACLE_ERR_ALLOC;
+  for (size_t q = 0; q < cells; ++q) Ynorm[q] = 0.0;
+  for (int64_t e = 0; e < nnz; ++e) {
+    for (int m = 0; m < order; ++m)
+      if (coords[m][e] < 0 || coords[m][e] >= dims[m]) { free(acc); return ORACLE_ERR_RANGE; }
+    int64_t f = find_key(keys, nkeys, kept_key(order, coords, dims, mode, e));
+    if (f < 0) continue;
+    int64_t k = coords[mode][e];
+    for (int64_t r = 0; r < R; ++r) {
+      double u = U[k * ldu + r];
+      acc[f * R + r] += (long double)val[e] * (long double)u;
+      Ynorm[f * R + r] += abs_d(val[e]) * abs_d(u);
+    }
+  }
+  for (size_t q = 0; q < cells; ++q) Y[q] = (double)acc[q];
+  free(acc);
+  return ORACLE_OK;
+}
+
 /* ---------------------------------------------------------------------------------------- MTTKRP
  * Mode-n matricised-tensor-times-Khatri-Rao product (the paper only names it; this is the textbook
  * definition): out_{i_n r} = sum over the other two modes of x * P_{p r} * Q_{q r}, where P and Q are

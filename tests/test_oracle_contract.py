@@ -235,3 +235,61 @@ def test_out_of_range_rejected():
         oracle.spmv([[0], [9]], [1.0], (2, 2), [1.0, 1.0])
     with pytest.raises(oracle.OracleError):
         oracle.mttkrp([[0], [0], [5]], [1.0], (2, 2, 2), 0, [None, np.ones((2, 1)), np.ones((2, 1))])
+
+
+# ----------------------------------------------------------------------------- order-N TTV / TTM
+@pytest.mark.parametrize("dims,nnz,seed", [((5, 4, 3, 6), 120, 1), ((2, 7, 1, 5), 40, 2), ((3, 3, 3, 3), 81, 3),
+                                           ((6, 5, 4), 70, 4), ((9, 7), 30, 5)])
+@pytest.mark.parametrize("integer", [False, True])
+def test_order_n_products_vs_einsum(dims, nnz, seed, integer):
+    """The order-N oracle against numpy.einsum on the densified tensor, every mode, matrix and vector factor."""
+    coords, val = synth.random_coo(dims, nnz, seed, integer_values=integer)
+    c, v = _np(coords), val.numpy()
+    X = _dense(c, v, dims)
+    letters = "abcd"[:len(dims)]
+    for mode in range(len(dims)):
+        kept = [m for m in range(len(dims)) if m != mode]
+        U = synth.random_dense((dims[mode], 3), seed, 40 + mode, integer_values=integer).numpy()
+        keys, Y, norm = oracle.ttm_n(c, v, dims, mode, U)
+        out = letters.replace(letters[mode], "") + "r"
+        dense = np.einsum(f"{letters},{letters[mode]}r->{out}", X, U)
+        dnorm = np.einsum(f"{letters},{letters[mode]}r->{out}", np.abs(X), np.abs(U))
+        flat = dense.reshape(-1, 3)
+        # the keys are exactly the kept-coordinate tuples that hold an entry, ascending
+        occupied = np.unique(np.ravel_multi_index([c[m] for m in kept], [dims[m] for m in kept]))
+        assert keys.tolist() == occupied.tolist()
+        if integer:
+            assert np.array_equal(Y, flat[keys])
+        else:
+            _close(Y, flat[keys], dnorm.reshape(-1, 3)[keys])
+        _close(norm, dnorm.reshape(-1, 3)[keys], dnorm.reshape(-1, 3)[keys], tol=1e-14)
+        mask = np.ones(flat.shape[0], dtype=bool)
+        mask[keys] = False
+        assert not flat[mask].any()                      # nothing outside the listed fibers
+        # one column = the tensor-times-vector product
+        _, y1, _ = oracle.ttm_n(c, v, dims, mode, U[:, 0].copy())
+        assert np.array_equal(y1[:, 0], Y[:, 0])
+
+
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_order_n_functions_agree_with_the_three_order_ones(mode):
+    dims = (9, 8, 7)
+    coords, val = synth.random_coo(dims, 200, 12)
+    c, v = _np(coords), val.numpy()
+    U = synth.random_dense((dims[mode], 4), 12).numpy()
+    k3, Y3, n3 = oracle.ttm(c, v, dims, mode, U)
+    kn, Yn, nn = oracle.ttm_n(c, v, dims, mode, U)
+    assert k3.tolist() == kn.tolist() and np.array_equal(Y3, Yn) and np.array_equal(n3, nn)
+    _, y3, _ = oracle.ttv(c, v, dims, mode, U[:, 1].copy())
+    _, yn, _ = oracle.ttm_n(c, v, dims, mode, U[:, 1].copy())
+    assert np.array_equal(y3, yn[:, 0])
+
+
+def test_order_n_matrix_case_is_spmm():
+    dims = (11, 13)
+    coords, val = synth.random_coo(dims, 60, 8)
+    c, v = _np(coords), val.numpy()
+    B = synth.random_dense((13, 5), 8).numpy()
+    Y, _ = oracle.spmm(c, v, dims, B)
+    keys, Yn, _ = oracle.ttm_n(c, v, dims, 1, B)           # contracting the column mode of a matrix
+    assert np.array_equal(Y[keys], Yn) and not np.delete(Y, keys, axis=0).any()
