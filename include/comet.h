@@ -144,10 +144,11 @@ comet_status_t comet_spmm(comet_handle_t handle, const comet_sptensor_t *A, cons
                           void *C, int64_t ldc, void *stream);
 
 /* TTV  Y = X x_n v  (SpTTV definition; `mode` = n, 0-based, must be the mode of X's LAST level).
- * X: 3 levels, [CU,CU,CU] (CSF) or [CN,S,S] (sorted COO). The result is sparse, one order lower:
- * comet_ttv_symbolic builds its structure over (mode_order[0], mode_order[1]) with level attributes
- * h_out_attr = {D,CU} (CSR) or {CU,CU} (DCSR); values are then (re)computed by comet_ttv, which
- * writes only Y->val. The structure depends on X's structure alone, never on values. Y owns its
+ * X: 3 levels, [CU,CU,CU] (CSF) or [CN,S,S] (sorted COO), or 4 levels, [CU,CU,CU,CU] (CSF). The result
+ * is sparse, one order lower: comet_ttv_symbolic builds its structure over the kept modes in storage
+ * order (Y's modes are renumbered 0..order-2) with h_out_attr[order-1] level attributes: {D,CU} (CSR) or
+ * {CU,CU} (DCSR) for a 3-order X, {CU,CU,CU} (CSF) for a 4-order X; values are then (re)computed by
+ * comet_ttv, which writes only Y->val. The structure depends on X's structure alone, never on values. Y owns its
  * arrays; X need not outlive it.
  * COO input: the fibers (runs of equal leading coordinate pairs) are not stored, so the symbolic call
  * derives them from the sorted coordinates (head flags, two scans, one synchronisation to read the
@@ -162,8 +163,8 @@ comet_status_t comet_ttv(comet_handle_t handle, const comet_sptensor_t *X, int32
 
 /* TTM  Y = X x_n U, U in R^{I_n x R} with rows indexed by the contracted mode (SpTTM definition);
  * mode n is replaced by r in place. `mode` must be the mode of X's last level. The result is
- * semi-sparse [CU,CU,D]: its two sparse levels equal X's first two levels and every stored fiber is
- * a dense row of R values (val is #fibers x R, row-major). comet_ttm_symbolic builds that structure,
+ * semi-sparse, [CU,CU,D] for a 3-order X and [CU,CU,CU,D] for a 4-order X: its sparse levels equal X's
+ * upper levels and every stored fiber is a dense row of R values (val is #fibers x R, row-major). comet_ttm_symbolic builds that structure,
  * comet_ttm writes only Y->val. Formats of X as for comet_ttv (COO: see the note there). */
 comet_status_t comet_ttm_symbolic(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode, int64_t R,
                                   void *stream, comet_sptensor_t *Y);

@@ -336,9 +336,15 @@ def spmm(A: SpTensor, B: torch.Tensor, out: torch.Tensor | None = None) -> torch
     return out
 
 
-def ttv_symbolic(X: SpTensor, mode: int, out_attr=(D, CU)) -> SpTensor:
+def ttv_symbolic(X: SpTensor, mode: int, out_attr=None) -> SpTensor:
+    """Structure of X x_mode v: one level fewer than X. Default format: CSR [D,CU] for a 3-order X,
+    CSF [CU,CU,CU] for a 4-order X."""
     out = SpTensorStruct()
-    h_at = (C.c_int32 * 2)(*out_attr)
+    n = X.c.order - 1
+    if out_attr is None:
+        out_attr = (D, CU) if n == 2 else (CU,) * n
+    assert len(out_attr) == n
+    h_at = (C.c_int32 * n)(*out_attr)
     st = X.handle.lib.comet_ttv_symbolic(X.handle._h, C.byref(X.c), C.c_int32(mode), h_at, _stream_ptr(), C.byref(out))
     X.handle.check(st, "comet_ttv_symbolic")
     return SpTensor(X.handle, out)

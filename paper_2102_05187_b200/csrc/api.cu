@@ -175,13 +175,19 @@ extern "C" comet_status_t comet_spmm(comet_handle_t handle, const comet_sptensor
 }
 
 // ------------------------------------------------------------------------------------------ TTV / TTM
+// TTV / TTM take 3-order tensors in CSF or sorted COO and 4-order tensors in CSF ([CU,CU,CU,CU]); the
+// contracted mode must be stored last. The kernels only see the last level (where each fiber of the level
+// above ends, the leaf coordinates, the values), so the order only matters for the result's structure.
 static comet_status_t check_last_mode(const comet_sptensor_t *X, int32_t mode) {
-  comet_status_t st = check_tensor(X, 3);
+  if (!X) return COMET_ERR_INVALID_ARG;
+  if (X->order != 3 && X->order != 4) return COMET_ERR_UNSUPPORTED_FORMAT;
+  comet_status_t st = check_tensor(X, X->order);
   if (st != COMET_OK) return st;
-  if (mode < 0 || mode > 2) return COMET_ERR_INVALID_ARG;
-  if (!is_fmt(X, 3, COMET_CU, COMET_CU, COMET_CU) && !is_fmt(X, 3, COMET_CN, COMET_S, COMET_S))
-    return COMET_ERR_UNSUPPORTED_FORMAT;
-  if (X->mode_order[2] != mode) return COMET_ERR_UNSUPPORTED_FORMAT;   // re-pack with the contracted mode last
+  if (mode < 0 || mode >= X->order) return COMET_ERR_INVALID_ARG;
+  bool csf = true;
+  for (int l = 0; l < X->order; ++l) csf = csf && X->attr[l] == COMET_CU;
+  if (!csf && !is_fmt(X, 3, COMET_CN, COMET_S, COMET_S)) return COMET_ERR_UNSUPPORTED_FORMAT;
+  if (X->mode_order[X->order - 1] != mode) return COMET_ERR_UNSUPPORTED_FORMAT;   // re-pack with the contracted mode last
   return COMET_OK;
 }
 
@@ -297,10 +303,10 @@ static void stash_fiber_pos(comet_sptensor_t *Y, Owner *o, int slot, CooAsCsf *v
   Y->pos_len[slot] = v->t.pos_len[2];
 }
 
-// Copies X's two upper levels into Y (levels 0 and 1), device to device.
+// Copies X's upper levels (all but the last) into the same levels of Y, device to device.
 static comet_status_t copy_upper_levels(Context *ctx, const comet_sptensor_t *X, comet_sptensor_t *Y, Owner *o,
                                         cudaStream_t s) {
-  for (int l = 0; l < 2; ++l) {
+  for (int l = 0; l < X->order - 1; ++l) {
     Y->pos_len[l] = X->pos_len[l];
     Y->crd_len[l] = X->crd_len[l];
     Y->pos[l] = (int32_t *)owned_alloc(ctx, o, (size_t)X->pos_len[l] * 4, s);
@@ -319,8 +325,10 @@ extern "C" comet_status_t comet_ttv_symbolic(comet_handle_t handle, const comet_
   if (!handle || !Y || !h_out_attr) return COMET_ERR_INVALID_ARG;
   comet_status_t st = check_last_mode(X, mode);
   if (st != COMET_OK) return st;
-  const bool csr = h_out_attr[0] == COMET_D && h_out_attr[1] == COMET_CU;
-  const bool dcsr = h_out_attr[0] == COMET_CU && h_out_attr[1] == COMET_CU;
+  const int out_order = X->order - 1;
+  const bool csr = out_order == 2 && h_out_attr[0] == COMET_D && h_out_attr[1] == COMET_CU;
+  bool dcsr = true;                       // every level compressed: DCSR (3-order input) or CSF (4-order input)
+  for (int l = 0; l < out_order; ++l) dcsr = dcsr && h_out_attr[l] == COMET_CU;
   if (!csr && !dcsr) return COMET_ERR_UNSUPPORTED_FORMAT;
   Context *ctx = reinterpret_cast<Context *>(handle);
   cudaStream_t s = (cudaStream_t)stream;
@@ -334,16 +342,15 @@ extern "C" comet_status_t comet_ttv_symbolic(comet_handle_t handle, const comet_
   }
   Owner *o = static_cast<Owner *>(owner_new());
   if (!o) { if (from_coo) coo_view_release(ctx, &view, false, s); return COMET_ERR_ALLOC; }
-  const int64_t S = X->crd_len[0], F = X->crd_len[1];
+  const int64_t S = X->crd_len[0], F = X->crd_len[out_order - 1];
   const int64_t rows = X->dims[X->mode_order[0]];
-  Y->order = 2;
+  Y->order = out_order;
   Y->dtype = X->dtype;
-  Y->dims[0] = rows;
-  Y->dims[1] = X->dims[X->mode_order[1]];
-  Y->mode_order[0] = 0;
-  Y->mode_order[1] = 1;
-  Y->attr[0] = h_out_attr[0];
-  Y->attr[1] = h_out_attr[1];
+  for (int l = 0; l < out_order; ++l) {       // the kept modes, renumbered in storage order
+    Y->dims[l] = X->dims[X->mode_order[l]];
+    Y->mode_order[l] = l;
+    Y->attr[l] = h_out_attr[l];
+  }
   Y->nnz = F;
   st = COMET_OK;
   if (dcsr) {
@@ -384,14 +391,15 @@ extern "C" comet_status_t comet_ttv(comet_handle_t handle, const comet_sptensor_
   if (st != COMET_OK) return st;
   // fibers: X's level-2 pos for CSF; for COO the boundaries that the symbolic call left in Y's spare slot
   const bool from_coo = X->attr[0] == COMET_CN;
-  const int32_t *fiber_pos = from_coo ? Y->pos[2] : X->pos[2];
-  const int64_t F = from_coo ? Y->pos_len[2] - 1 : X->crd_len[1];
+  const int last = X->order - 1;
+  const int32_t *fiber_pos = from_coo ? Y->pos[2] : X->pos[last];
+  const int64_t F = from_coo ? Y->pos_len[2] - 1 : X->crd_len[last - 1];
   if (!fiber_pos || F < 0) return COMET_ERR_INVALID_ARG;
-  if (Y->order != 2 || Y->nnz != F || (Y->nnz > 0 && !Y->val)) return COMET_ERR_INVALID_ARG;
+  if (Y->order != last || Y->nnz != F || (Y->nnz > 0 && !Y->val)) return COMET_ERR_INVALID_ARG;
   if (Y->dtype != X->dtype) return COMET_ERR_INVALID_ARG;
   if (misaligned(v, X->dtype)) return COMET_ERR_MISALIGNED;
   Context *ctx = reinterpret_cast<Context *>(handle);
-  return seg_dot(ctx, X->dtype, fiber_pos + 1, X->crd[2], X->val, F, X->nnz, v, X->dims[mode], Y->val, nullptr, F,
+  return seg_dot(ctx, X->dtype, fiber_pos + 1, X->crd[last], X->val, F, X->nnz, v, X->dims[mode], Y->val, nullptr, F,
                  (cudaStream_t)stream);
 }
 
@@ -413,21 +421,23 @@ extern "C" comet_status_t comet_ttm_symbolic(comet_handle_t handle, const comet_
   }
   Owner *o = static_cast<Owner *>(owner_new());
   if (!o) { if (from_coo) coo_view_release(ctx, &view, false, s); return COMET_ERR_ALLOC; }
-  const int64_t F = X->crd_len[1];
-  Y->order = 3;
+  const int last = X->order - 1;
+  const int64_t F = X->crd_len[last - 1];
+  Y->order = X->order;
   Y->dtype = X->dtype;
-  for (int m = 0; m < 3; ++m) { Y->dims[m] = X->dims[m]; Y->mode_order[m] = X->mode_order[m]; }
+  for (int m = 0; m < X->order; ++m) { Y->dims[m] = X->dims[m]; Y->mode_order[m] = X->mode_order[m]; }
   Y->dims[mode] = R;                      // mode n is replaced by r in place
-  Y->attr[0] = COMET_CU; Y->attr[1] = COMET_CU; Y->attr[2] = COMET_D;
+  for (int l = 0; l < last; ++l) Y->attr[l] = COMET_CU;
+  Y->attr[last] = COMET_D;
   Y->nnz = F * R;
   st = copy_upper_levels(ctx, X, Y, o, s);
   if (st == COMET_OK) {
-    Y->pos_len[2] = 1;
-    Y->pos[2] = (int32_t *)owned_alloc(ctx, o, 4, s);
+    Y->pos_len[last] = 1;
+    Y->pos[last] = (int32_t *)owned_alloc(ctx, o, 4, s);
     Y->val = owned_alloc(ctx, o, (size_t)F * R * elem_size(X->dtype), s);
-    if (!Y->pos[2] || !Y->val) st = COMET_ERR_ALLOC;
+    if (!Y->pos[last] || !Y->val) st = COMET_ERR_ALLOC;
     else {
-      set_word_kernel<<<1, 1, 0, s>>>(Y->pos[2], (int32_t)R);
+      set_word_kernel<<<1, 1, 0, s>>>(Y->pos[last], (int32_t)R);
       ctx->launches += 1;
       cudaError_t e = cudaGetLastError();
       if (e != cudaSuccess) st = cuda_fail(ctx, e);
@@ -448,14 +458,15 @@ extern "C" comet_status_t comet_ttm(comet_handle_t handle, const comet_sptensor_
   comet_status_t st = check_last_mode(X, mode);
   if (st != COMET_OK) return st;
   const bool from_coo = X->attr[0] == COMET_CN;
-  const int32_t *fiber_pos = from_coo ? Y->pos[3] : X->pos[2];
-  const int64_t F = from_coo ? Y->pos_len[3] - 1 : X->crd_len[1];
+  const int last = X->order - 1;
+  const int32_t *fiber_pos = from_coo ? Y->pos[3] : X->pos[last];
+  const int64_t F = from_coo ? Y->pos_len[3] - 1 : X->crd_len[last - 1];
   if (!fiber_pos || F < 0) return COMET_ERR_INVALID_ARG;
-  if (Y->order != 3 || Y->nnz != F * R || (Y->nnz > 0 && !Y->val)) return COMET_ERR_INVALID_ARG;
+  if (Y->order != X->order || Y->nnz != F * R || (Y->nnz > 0 && !Y->val)) return COMET_ERR_INVALID_ARG;
   if (Y->dtype != X->dtype) return COMET_ERR_INVALID_ARG;
   if (misaligned(U, X->dtype)) return COMET_ERR_MISALIGNED;
   Context *ctx = reinterpret_cast<Context *>(handle);
-  return seg_gather(ctx, X->dtype, fiber_pos + 1, X->crd[2], X->val, F, X->nnz, U, ldu, R, Y->val, R, nullptr, F,
+  return seg_gather(ctx, X->dtype, fiber_pos + 1, X->crd[last], X->val, F, X->nnz, U, ldu, R, Y->val, R, nullptr, F,
                     (cudaStream_t)stream);
 }
 

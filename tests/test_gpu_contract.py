@@ -216,6 +216,61 @@ def test_ttv_ttm_from_sorted_coo(dims, nnz, seed, mode, tile_items):
         assert Z.pos(2).tolist() == [R]
 
 
+ORDER4_CASES = [((9, 8, 7, 6), 900, 1), ((20, 15, 12, 10), 6000, 2), ((1, 12, 12, 12), 300, 3),
+                ((12, 12, 12, 1), 300, 4), ((6, 5, 4, 3), 360, 5), ((10, 10, 10, 10), 0, 6), ((400, 3, 5, 4), 500, 7)]
+
+
+@pytest.mark.parametrize("dims,nnz,seed", ORDER4_CASES)
+@pytest.mark.parametrize("mode", [0, 1, 2, 3])
+def test_ttv_ttm_order4_csf(dims, nnz, seed, mode, tile_items):
+    """4-order tensors in CSF [CU,CU,CU,CU], contracted mode stored last: the result's structure is X's three
+    upper levels, values against the order-N oracle."""
+    coords, val = synth.random_coo(dims, nnz, seed)
+    c, v = _np(coords), val.numpy()
+    kept = [m for m in range(4) if m != mode]
+    mode_order = (kept[0], kept[1], kept[2], mode)
+    pk = oracle.pack(c, v, dims, mode_order, (CU, CU, CU, CU))
+    X = upload_packed(pk)
+    vec = synth.random_dense((dims[mode],), seed).numpy()
+    keys, want, norm = oracle.ttm_n(c, v, dims, mode, vec)
+    Y = comet.ttv_symbolic(X, mode)
+    comet.validate(Y)
+    assert Y.attr == (CU, CU, CU) and Y.dims == tuple(dims[m] for m in kept) and Y.c.nnz == len(keys)
+    Y.val.fill_(float("nan"))
+    comet.ttv(X, mode, dev(vec), Y)
+    assert_close(Y.val, want[:, 0], norm[:, 0], what="ttv order 4")
+    for l in range(3):
+        assert_equal_arrays(Y.pos(l), pk.pos[l], f"ttv4 pos{l}")
+        assert_equal_arrays(Y.crd(l), pk.crd[l], f"ttv4 crd{l}")
+    # the leaf coordinates of Y enumerate the kept-coordinate keys in ascending order
+    for R in (1, 16, 5):
+        U = synth.random_dense((dims[mode], R), seed + 1).numpy()
+        _, wantm, normm = oracle.ttm_n(c, v, dims, mode, U)
+        Z = comet.ttm_symbolic(X, mode, R)
+        assert Z.attr == (CU, CU, CU, D) and Z.pos(3).tolist() == [R]
+        assert Z.dims == tuple(R if m == mode else d for m, d in enumerate(dims))
+        Z.val.fill_(float("nan"))
+        comet.ttm(X, mode, dev(U), Z)
+        assert_close(Z.val.reshape(-1, R), wantm, normm, what=f"ttm order 4 R={R}")
+        for l in range(3):
+            assert_equal_arrays(Z.pos(l), pk.pos[l], f"ttm4 pos{l}")
+            assert_equal_arrays(Z.crd(l), pk.crd[l], f"ttm4 crd{l}")
+
+
+def test_order4_packed_on_the_device_then_contracted():
+    dims = (30, 25, 20, 15)
+    coords, val = synth.random_coo(dims, 20000, 9)
+    c, v = _np(coords), val.numpy()
+    X = comet.pack([t.cuda() for t in coords], val.cuda(), dims, (3, 1, 0, 2), (CU, CU, CU, CU))
+    vec = synth.random_dense((dims[2],), 9).numpy()
+    _, want, norm = oracle.ttm_n(c, v, dims, 2, vec)
+    # oracle keys are in increasing MODE order (0,1,3); the stored order is (3,1,0): compare as sets of fibers
+    Y = comet.ttv(X, 2, dev(vec))
+    assert Y.c.nnz == len(want)
+    got = Y.val.cpu().numpy()
+    assert abs(np.sort(got) - np.sort(want[:, 0])).max() <= 1e-12 * norm.max()
+
+
 def test_ttv_numeric_phase_rejects_a_result_built_for_another_tensor():
     dims = (12, 11, 10)
     coords, val = synth.random_coo(dims, 400, 3)
