@@ -179,9 +179,8 @@ __global__ void __launch_bounds__(kSortThreads) radix_histogram_kernel(const uin
 __global__ void __launch_bounds__(kSortThreads, 4) radix_scatter_kernel(
     const uint64_t *__restrict__ kin, const uint32_t *__restrict__ pin, uint64_t *__restrict__ kout,
     uint32_t *__restrict__ pout, const uint32_t *__restrict__ table, int64_t n, int shift, int64_t tiles) {
-  __shared__ uint32_t s_cnt[kSortWarps][256];     // per-warp digit counts, then per-warp local offsets
-  __shared__ uint32_t s_start[256];               // where digit d starts inside the tile's sorted order
-  __shared__ uint32_t s_delta[256];               // global position of digit d's run minus s_start[d]
+  __shared__ uint32_t s_cnt[kSortWarps][256];     // per-warp digit counts, then where each warp's keys of a digit go
+  __shared__ uint32_t s_delta[256];               // global position of digit d's run minus its start inside the tile
   __shared__ uint64_t s_key[kSortTile];           // the tile in sorted order
   __shared__ uint32_t s_pay[kSortTile];
   __shared__ uint32_t s_warp[32];
@@ -208,33 +207,33 @@ __global__ void __launch_bounds__(kSortThreads, 4) radix_scatter_kernel(
     const unsigned peers = __match_any_sync(0xffffffffu, d);
     const int leader = __ffs(peers) - 1;
     uint32_t old = 0;
-    if (lane == leader) {
-      old = s_cnt[warp][d];
-      s_cnt[warp][d] = old + __popc(peers);
-    }
+    if (lane == leader) old = atomicAdd(&s_cnt[warp][d], (uint32_t)__popc(peers));   // one shared-memory operation
     old = __shfl_sync(0xffffffffu, old, leader);
     rank[r] = old + __popc(peers & lt);
     __syncwarp();
   }
   __syncthreads();
   {
-    // digit `tid`: tile total, per-warp offsets inside the digit's run, start of the run inside the tile
+    // digit `tid`: tile total -> start of the digit's run inside the tile -> where each warp's keys of the
+    // digit start (run start + the counts of the warps before it), so that placing a key costs one lookup
     uint32_t run = 0;
+#pragma unroll
+    for (int w = 0; w < kSortWarps; ++w) run += s_cnt[w][tid];
+    const uint32_t start = block_exclusive_scan(run, s_warp, nullptr);
+    uint32_t off = start;
 #pragma unroll
     for (int w = 0; w < kSortWarps; ++w) {
       const uint32_t c = s_cnt[w][tid];
-      s_cnt[w][tid] = run;
-      run += c;
+      s_cnt[w][tid] = off;
+      off += c;
     }
-    const uint32_t start = block_exclusive_scan(run, s_warp, nullptr);
-    s_start[tid] = start;
     s_delta[tid] = table[(int64_t)tid * tiles + blockIdx.x] - start;
   }
   __syncthreads();
 #pragma unroll
   for (int r = 0; r < kSortItems; ++r) {          // local sort: every item to its place in the tile's order
     const uint32_t d = (uint32_t)(key[r] >> shift) & 255u;
-    const uint32_t at = s_start[d] + s_cnt[warp][d] + rank[r];
+    const uint32_t at = s_cnt[warp][d] + rank[r];
     s_key[at] = key[r];
     s_pay[at] = pay[r];
   }
