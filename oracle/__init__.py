@@ -190,6 +190,26 @@ def mttkrp(coords, val, dims, mode, factors, rows=None):
     return A, An
 
 
+def mttkrp_n(coords, val, dims, mode, factors, rows=None):
+    """MTTKRP for tensors of order 3 or 4: out_{i_mode, r} = sum x * prod of the other modes' factor entries.
+    `factors`: one (dim_m x R) array per mode; the one at `mode` is ignored (may be None)."""
+    order = len(dims)
+    c = [_i32(x) for x in coords]
+    val = _f64(val)
+    F = [None if (m == mode or f is None) else _f64(f) for m, f in enumerate(factors)]
+    R = next(f.shape[1] for f in F if f is not None)
+    fp = (C.c_void_p * order)(*[None if f is None else f.ctypes.data for f in F])
+    slot, n_out = _slots(rows, dims[mode])
+    A = np.zeros((n_out, R))
+    An = np.zeros((n_out, R))
+    rc = lib().oracle_mttkrp_n(C.c_int(order), C.c_int64(len(val)), _coord_ptrs(c), _p(val), _p(_i64(dims)),
+                               C.c_int(mode), fp, _p(_i64([R] * order)), C.c_int64(R), _p(slot), C.c_int64(n_out),
+                               _p(A), _p(An))
+    if rc:
+        raise OracleError(rc, "mttkrp_n")
+    return A, An
+
+
 class _Packed(C.Structure):
     _fields_ = [("order", C.c_int32), ("nnz", C.c_int64),
                 ("pos", C.c_void_p * MAX_ORDER), ("pos_len", C.c_int64 * MAX_ORDER),

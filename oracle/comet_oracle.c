@@ -267,6 +267,42 @@ int oracle_mttkrp(int64_t nnz, const int32_t *c0, const int32_t *c1, const int32
   return ORACLE_OK;
 }
 
+/* MTTKRP for tensors of order 3 or 4: out_{i_n r} = sum over the entries of x * prod_{m != n} F_m[i_m, r]
+ * (the textbook definition for any order). The product is formed left to right in increasing mode
+ * order, ((x * F_a) * F_b) * F_c, so that the 3-order case is the function above, operation for
+ * operation. `factors` / `ld` hold one entry per mode (the one at `mode` is ignored). */
+int oracle_mttkrp_n(int order, int64_t nnz, const int32_t *const *coords, const double *val, const int64_t *dims,
+                    int mode, const double *const *factors, const int64_t *ld, int64_t R, const int64_t *row_slot,
+                    int64_t n_out, double *A, double *Anorm) {
+  if (order < 3 || order > 4 || mode < 0 || mode >= order || nnz < 0 || n_out < 0 || R < 0) return ORACLE_ERR_ARG;
+  size_t cells = (size_t)n_out * (size_t)R;
+  long double *acc = (long double *)calloc(cells ? cells : 1, sizeof(long double));
+  if (!acc) return ORACLE_ERR_ALLOC;
+  for (size_t q = 0; q < cells; ++q) Anorm[q] = 0.0;
+  for (int64_t e = 0; e < nnz; ++e) {
+    for (int m = 0; m < order; ++m)
+      if (coords[m][e] < 0 || coords[m][e] >= dims[m]) { free(acc); return ORACLE_ERR_RANGE; }
+    int64_t i = coords[mode][e];
+    int64_t o = row_slot ? row_slot[i] : i;
+    if (o < 0) continue;
+    for (int64_t r = 0; r < R; ++r) {
+      long double term = (long double)val[e];
+      double mag = abs_d(val[e]);
+      for (int m = 0; m < order; ++m) {
+        if (m == mode) continue;
+        double f = factors[m][(int64_t)coords[m][e] * ld[m] + r];
+        term *= (long double)f;
+        mag *= abs_d(f);
+      }
+      acc[o * R + r] += term;
+      Anorm[o * R + r] += mag;
+    }
+  }
+  for (size_t q = 0; q < cells; ++q) A[q] = (double)acc[q];
+  free(acc);
+  return ORACLE_OK;
+}
+
 /* ------------------------------------------------------------------------------------------ Pack
  * COO -> per-level pos/crd arrays from the level attributes.
  *

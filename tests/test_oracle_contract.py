@@ -293,3 +293,40 @@ def test_order_n_matrix_case_is_spmm():
     Y, _ = oracle.spmm(c, v, dims, B)
     keys, Yn, _ = oracle.ttm_n(c, v, dims, 1, B)           # contracting the column mode of a matrix
     assert np.array_equal(Y[keys], Yn) and not np.delete(Y, keys, axis=0).any()
+
+
+@pytest.mark.parametrize("dims,nnz,seed", [((5, 4, 3, 6), 120, 1), ((2, 7, 1, 5), 40, 2), ((3, 3, 3, 3), 81, 3),
+                                           ((6, 5, 4), 70, 4)])
+@pytest.mark.parametrize("integer", [False, True])
+def test_order_n_mttkrp_vs_einsum(dims, nnz, seed, integer):
+    coords, val = synth.random_coo(dims, nnz, seed, integer_values=integer)
+    c, v = _np(coords), val.numpy()
+    X = _dense(c, v, dims)
+    R = 3
+    F = [synth.random_dense((d, R), seed, 60 + m, integer_values=integer).numpy() for m, d in enumerate(dims)]
+    letters = "abcd"[:len(dims)]
+    for mode in range(len(dims)):
+        others = [m for m in range(len(dims)) if m != mode]
+        expr = letters + "," + ",".join(letters[m] + "r" for m in others) + "->" + letters[mode] + "r"
+        want = np.einsum(expr, X, *[F[m] for m in others])
+        norm = np.einsum(expr, np.abs(X), *[np.abs(F[m]) for m in others])
+        got, gnorm = oracle.mttkrp_n(c, v, dims, mode, F)
+        if integer:
+            assert np.array_equal(got, want)
+        else:
+            _close(got, want, norm)
+        _close(gnorm, norm, norm, tol=1e-14)
+        rows = np.array(sorted({0, dims[mode] - 1, dims[mode] // 2}))
+        sub, _ = oracle.mttkrp_n(c, v, dims, mode, F, rows=rows)
+        assert np.array_equal(sub, got[rows])
+
+
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_order_n_mttkrp_is_the_three_order_function_on_three_order_input(mode):
+    dims = (9, 8, 7)
+    coords, val = synth.random_coo(dims, 200, 12)
+    c, v = _np(coords), val.numpy()
+    F = [synth.random_dense((d, 5), 12, 60 + m).numpy() for m, d in enumerate(dims)]
+    a3, n3 = oracle.mttkrp(c, v, dims, mode, F)
+    an, nn = oracle.mttkrp_n(c, v, dims, mode, F)
+    assert np.array_equal(a3, an) and np.array_equal(n3, nn)
