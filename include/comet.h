@@ -183,8 +183,10 @@ comet_status_t comet_ttm(comet_handle_t handle, const comet_sptensor_t *X, int32
  *     within the stated tolerance). About 2-4x slower than the first-level case; callers that repeat the
  *     same mode many times may prefer a second comet_pack with that mode first. For fp32 tensors this
  *     path takes rows x R doubles of handle scratch.
- *   h_factors[3]  HOST array of DEVICE pointers, factor of mode m is dims[m] x R with leading
- *                 dimension h_ld[m]; the entry at `mode` is ignored
+ * 4-order tensors ([CN,S,S,S] or [CU,CU,CU,CU]; out_{i_n r} = sum x * the three other factors' entries): every
+ * mode, all by atomic accumulation (the note on the summation order applies to all four modes).
+ *   h_factors[order]  HOST array of DEVICE pointers, factor of mode m is dims[m] x R with leading
+ *                 dimension h_ld[m] (h_ld has `order` entries too); the entry at `mode` is ignored
  *   out           dims[mode] x R, leading dimension ldo, every row written. */
 comet_status_t comet_mttkrp(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode,
                             const void *const *h_factors, const int64_t *h_ld, int64_t R, void *out, int64_t ldo,

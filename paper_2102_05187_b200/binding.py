@@ -391,8 +391,10 @@ def mttkrp(X: SpTensor, mode: int, factors, out: torch.Tensor | None = None) -> 
     dt = _same_dtype(X, out, *live)
     if out is None:
         out = torch.empty((rows, R), dtype=dt, device=live[0].device)
-    h_f = (C.c_void_p * 3)(*[0 if (m == mode or f is None) else f.data_ptr() for m, f in enumerate(factors)])
-    h_ld = (C.c_int64 * 3)(*[0 if (m == mode or f is None) else f.stride(0) for m, f in enumerate(factors)])
+    order = X.c.order
+    assert len(factors) == order
+    h_f = (C.c_void_p * order)(*[0 if (m == mode or f is None) else f.data_ptr() for m, f in enumerate(factors)])
+    h_ld = (C.c_int64 * order)(*[0 if (m == mode or f is None) else f.stride(0) for m, f in enumerate(factors)])
     st = X.handle.lib.comet_mttkrp(X.handle._h, C.byref(X.c), C.c_int32(mode), h_f, h_ld, C.c_int64(R), _ptr(out),
                                    C.c_int64(out.stride(0)), _stream_ptr())
     X.handle.check(st, "comet_mttkrp")

@@ -471,10 +471,49 @@ extern "C" comet_status_t comet_ttm(comet_handle_t handle, const comet_sptensor_
 }
 
 // ------------------------------------------------------------------------------------------ MTTKRP
+// 4-order tensors: COO [CN,S,S,S] or CSF [CU,CU,CU,CU], any output mode, atomic accumulation throughout.
+static comet_status_t mttkrp_order4(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode,
+                                    const void *const *h_factors, const int64_t *h_ld, int64_t R, void *out,
+                                    int64_t ldo, void *stream) {
+  comet_status_t st = check_tensor(X, 4);
+  if (st != COMET_OK) return st;
+  if (mode < 0 || mode > 3) return COMET_ERR_INVALID_ARG;
+  bool coo = X->attr[0] == COMET_CN, csf = X->attr[0] == COMET_CU;
+  for (int l = 1; l < 4; ++l) { coo = coo && X->attr[l] == COMET_S; csf = csf && X->attr[l] == COMET_CU; }
+  if (!coo && !csf) return COMET_ERR_UNSUPPORTED_FORMAT;
+  int level = 0;
+  while (X->mode_order[level] != mode) ++level;
+  int other[3], n = 0;                                 // the three other levels, in storage order
+  for (int l = 0; l < 4; ++l) if (l != level) other[n++] = l;
+  const void *F[3];
+  int64_t ld[3];
+  for (int q = 0; q < 3; ++q) {
+    const int m = X->mode_order[other[q]];
+    if (!h_factors[m] || h_ld[m] < R) return COMET_ERR_INVALID_ARG;
+    if (misaligned(h_factors[m], X->dtype)) return COMET_ERR_MISALIGNED;
+    if (h_ld[m] >= (1ll << 28)) return COMET_ERR_INDEX_OVERFLOW;
+    F[q] = h_factors[m];
+    ld[q] = h_ld[m];
+  }
+  if (misaligned(out, X->dtype)) return COMET_ERR_MISALIGNED;
+  Context *ctx = reinterpret_cast<Context *>(handle);
+  const int64_t rows = X->dims[mode];
+  if (coo) {
+    const int32_t *crd[4] = {X->crd[level], X->crd[other[0]], X->crd[other[1]], X->crd[other[2]]};
+    return mttkrp_scatter4(ctx, X->dtype, -1, nullptr, nullptr, nullptr, crd, X->val, 0, 0, 0, X->nnz, rows, F[0], ld[0],
+                           F[1], ld[1], F[2], ld[2], R, out, ldo, (cudaStream_t)stream);
+  }
+  const int32_t *crd[4] = {X->crd[0], X->crd[1], X->crd[2], X->crd[3]};
+  return mttkrp_scatter4(ctx, X->dtype, level, X->pos[1], X->pos[2], X->pos[3], crd, X->val, X->crd_len[0], X->crd_len[1],
+                         X->crd_len[2], X->nnz, rows, F[0], ld[0], F[1], ld[1], F[2], ld[2], R, out, ldo,
+                         (cudaStream_t)stream);
+}
+
 extern "C" comet_status_t comet_mttkrp(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode,
                                        const void *const *h_factors, const int64_t *h_ld, int64_t R, void *out,
                                        int64_t ldo, void *stream) {
   if (!handle || !h_factors || !h_ld || !out || R < 1 || ldo < R) return COMET_ERR_INVALID_ARG;
+  if (X && X->order == 4) return mttkrp_order4(handle, X, mode, h_factors, h_ld, R, out, ldo, stream);
   comet_status_t st = check_tensor(X, 3);
   if (st != COMET_OK) return st;
   if (mode < 0 || mode > 2) return COMET_ERR_INVALID_ARG;

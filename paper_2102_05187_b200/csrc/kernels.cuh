@@ -36,6 +36,15 @@ comet_status_t mttkrp_scatter(Context *ctx, int dtype, int kind, const int32_t *
                               int64_t F, int64_t N, int64_t rows, const void *A, int64_t lda, const void *B, int64_t ldb,
                               int64_t R, void *out, int64_t ldo, cudaStream_t stream);
 
+// The same for 4-order tensors, every output mode. kind -1: COO (crd[0] = output-mode coordinates, crd[1..3] =
+// those of A's, B's, C's modes); kind 0..3: CSF, output mode at that level, A / B / C = the factors of the three
+// other levels in storage order.
+comet_status_t mttkrp_scatter4(Context *ctx, int dtype, int kind, const int32_t *pos1, const int32_t *pos2,
+                               const int32_t *pos3, const int32_t *const *crd, const void *val, int64_t S, int64_t F1,
+                               int64_t F2, int64_t N, int64_t rows, const void *A, int64_t lda, const void *B,
+                               int64_t ldb, const void *C, int64_t ldc, int64_t R, void *out, int64_t ldo,
+                               cudaStream_t stream);
+
 comet_status_t zero_rows(Context *ctx, void *C, int dtype, int64_t rows, int64_t R, int64_t ldc, cudaStream_t stream);
 // Exclusive scan of uint32 words in three launches (tile sums, scan of the sums, apply); defined in pack.cu.
 // `out` may alias `in`; `tmp` holds scan_tmp_words(n) words; `total` (device, optional) receives the sum.

@@ -257,6 +257,41 @@ def test_ttv_ttm_order4_csf(dims, nnz, seed, mode, tile_items):
             assert_equal_arrays(Z.crd(l), pk.crd[l], f"ttm4 crd{l}")
 
 
+@pytest.mark.parametrize("dims,nnz,seed", ORDER4_CASES)
+@pytest.mark.parametrize("mode_order", [(0, 1, 2, 3), (3, 1, 0, 2)])
+@pytest.mark.parametrize("attr", [(CN, S, S, S), (CU, CU, CU, CU)])
+def test_mttkrp_order4_every_mode(dims, nnz, seed, mode_order, attr):
+    coords, val = synth.random_coo(dims, nnz, seed)
+    c, v = _np(coords), val.numpy()
+    X = upload_packed(oracle.pack(c, v, dims, mode_order, attr))
+    for R in (1, 5, 16, 40):
+        F = [synth.random_dense((d, R), seed, 60 + m).numpy() for m, d in enumerate(dims)]
+        for mode in range(4):
+            want, norm = oracle.mttkrp_n(c, v, dims, mode, F)
+            out = torch.full((dims[mode], R), float("nan"), dtype=torch.float64, device="cuda")
+            comet.mttkrp(X, mode, [None if m == mode else dev(f) for m, f in enumerate(F)], out)
+            assert_close(out, want, norm, what=f"mttkrp4 mode {mode} of {mode_order} {attr} R={R}")
+
+
+def test_mttkrp_order4_integers_exact_and_fp32():
+    dims = (12, 10, 9, 8)
+    coords, val = synth.random_coo(dims, 3000, 4, integer_values=True)
+    c, v = _np(coords), val.numpy()
+    F = [synth.random_dense((d, 6), 4, 60 + m, integer_values=True).numpy() for m, d in enumerate(dims)]
+    for attr in [(CN, S, S, S), (CU, CU, CU, CU)]:
+        pk = oracle.pack(c, v, dims, (1, 0, 3, 2), attr)
+        X = upload_packed(pk)
+        pos = [dev(p, torch.int32) if p.size else None for p in pk.pos]
+        crd = [dev(x, torch.int32) if x.size else None for x in pk.crd]
+        X32 = comet.SpTensor.from_arrays(pk.dims, pk.mode_order, pk.attr, pos, crd, dev(pk.val.astype(np.float32)))
+        for mode in range(4):
+            want, _ = oracle.mttkrp_n(c, v, dims, mode, F)
+            got = comet.mttkrp(X, mode, [None if m == mode else dev(f) for m, f in enumerate(F)])
+            assert_equal_arrays(got, want, "integer mttkrp4")
+            got32 = comet.mttkrp(X32, mode, [None if m == mode else dev(f.astype(np.float32)) for m, f in enumerate(F)])
+            assert got32.dtype == torch.float32 and np.array_equal(got32.cpu().numpy().astype(np.float64), want)
+
+
 def test_order4_packed_on_the_device_then_contracted():
     dims = (30, 25, 20, 15)
     coords, val = synth.random_coo(dims, 20000, 9)
