@@ -236,9 +236,32 @@ def _copy(ptr, n, dtype):
     return np.ctypeslib.as_array(C.cast(ptr, C.POINTER(np.ctypeslib.as_ctypes_type(dtype))), shape=(n,)).copy()
 
 
-def pack(coords, val, dims, mode_order, attr) -> Packed:
-    """COO -> level arrays for the given storage order and per-level attributes (D, CU, CN, S)."""
+def sum_duplicates(coords, val, dims, mode_order):
+    """Merge entries with equal coordinates (values added one by one in double, in input order).
+    Returns (coords, val, first): the merged entries sorted in storage order and, for each, the input
+    index of its first contributor."""
     order = len(dims)
+    c = [_i32(x) for x in coords]
+    val = _f64(val)
+    n = len(val)
+    oc = [np.zeros(max(n, 1), dtype=np.int32) for _ in range(order)]
+    ov = np.zeros(max(n, 1))
+    first = np.zeros(max(n, 1), dtype=np.int64)
+    lib().oracle_sum_duplicates.restype = C.c_int64
+    m = lib().oracle_sum_duplicates(C.c_int32(order), C.c_int64(n), _coord_ptrs(c), _p(val), _p(_i32(mode_order)),
+                                    _coord_ptrs(oc), _p(ov), _p(first))
+    if m < 0:
+        raise OracleError(m, "sum_duplicates")
+    return [x[:m].copy() for x in oc], ov[:m].copy(), first[:m].copy()
+
+
+def pack(coords, val, dims, mode_order, attr, sum_duplicates_first: bool = False) -> Packed:
+    """COO -> level arrays for the given storage order and per-level attributes (D, CU, CN, S).
+    Entries with equal coordinates are an error unless `sum_duplicates_first`, in which case they are
+    merged (see sum_duplicates) before packing; `perm` then refers to the merged entry list."""
+    order = len(dims)
+    if sum_duplicates_first:
+        coords, val, _ = sum_duplicates(coords, val, dims, mode_order)
     c = [_i32(x) for x in coords]
     val = _f64(val)
     ptrs = (C.c_void_p * order)(*[a.ctypes.data for a in c])

@@ -369,6 +369,38 @@ void oracle_packed_free(oracle_packed_t *t) {
   t->perm = NULL;
 }
 
+/* Entries that share all coordinates are merged into one whose value is their sum, added one by one in
+ * double in the order the entries were given (a stable sort keeps that order inside a run of equal
+ * coordinates). Writes the merged entries (in sorted storage order, which the packing does not need
+ * but which makes the result unique) and returns how many there are; out_coo[m] / out_val hold nnz
+ * slots. `first[k]` receives the input index of the first entry of merged entry k. */
+int64_t oracle_sum_duplicates(int32_t order, int64_t nnz, const int32_t *const *coo, const double *val,
+                              const int32_t *mode_order, int32_t *const *out_coo, double *out_val, int64_t *first) {
+  if (order < 1 || order > ORACLE_MAX_ORDER || nnz < 0) return ORACLE_ERR_ARG;
+  size_t n1 = (size_t)(nnz ? nnz : 1);
+  rec_t *rec = (rec_t *)malloc(n1 * sizeof(rec_t));
+  rec_t *tmp = (rec_t *)malloc(n1 * sizeof(rec_t));
+  if (!rec || !tmp) { free(rec); free(tmp); return ORACLE_ERR_ALLOC; }
+  for (int64_t e = 0; e < nnz; ++e) {
+    for (int l = 0; l < order; ++l) rec[e].c[l] = coo[mode_order[l]][e];
+    rec[e].src = e;
+  }
+  merge_sort(rec, tmp, 0, nnz, order);
+  int64_t m = 0;
+  for (int64_t e = 0; e < nnz; ++e) {
+    if (e > 0 && !rec_less(&rec[e - 1], &rec[e], order)) {
+      out_val[m - 1] = out_val[m - 1] + val[rec[e].src];      /* same coordinates: add to the open entry */
+    } else {
+      for (int l = 0; l < order; ++l) out_coo[mode_order[l]][m] = rec[e].c[l];
+      out_val[m] = val[rec[e].src];
+      first[m] = rec[e].src;
+      m += 1;
+    }
+  }
+  free(rec); free(tmp);
+  return m;
+}
+
 int oracle_pack(int32_t order, const int64_t *dims, int64_t nnz, const int32_t *const *coo, const double *val,
                 const int32_t *mode_order, const int32_t *attr, oracle_packed_t *out) {
   if (order < 1 || order > ORACLE_MAX_ORDER || nnz < 0 || !out) return ORACLE_ERR_ARG;

@@ -195,3 +195,46 @@ def test_rejects_bad_input():
         assert e.value.code == -2
     with pytest.raises(oracle.OracleError):
         oracle.pack([[0], [1]], [1.0], (2, 2), (0, 0), (D, CU))
+
+
+# ----------------------------------------------------------------------------- merging duplicates
+def test_sum_duplicates_against_a_dictionary_and_scipy():
+    import scipy.sparse as sp
+    rng = np.random.default_rng(5)
+    dims = (7, 9)
+    n = 300                                            # 63 cells: many duplicates
+    ci, cj = rng.integers(0, 7, n).astype(np.int32), rng.integers(0, 9, n).astype(np.int32)
+    v = rng.integers(-4, 5, n).astype(np.float64)      # small integers: every order of summation is exact
+    (oi, oj), ov, first = oracle.sum_duplicates([ci, cj], v, dims, (0, 1))
+    acc, seen_first = {}, {}
+    for e in range(n):
+        acc[(ci[e], cj[e])] = acc.get((ci[e], cj[e]), 0.0) + v[e]
+        seen_first.setdefault((ci[e], cj[e]), e)
+    cells = sorted(acc)
+    assert list(zip(oi.tolist(), oj.tolist())) == cells
+    assert ov.tolist() == [acc[k] for k in cells] and first.tolist() == [seen_first[k] for k in cells]
+    csr = sp.coo_matrix((v, (ci, cj)), shape=dims).tocsr()      # scipy sums duplicates on conversion
+    csr.sort_indices()
+    pk = oracle.pack([ci, cj], v, dims, (0, 1), (oracle.D, oracle.CU), sum_duplicates_first=True)
+    assert pk.pos[1].tolist() == csr.indptr.tolist() and pk.crd[1].tolist() == csr.indices.tolist()
+    assert pk.val.tolist() == csr.data.tolist()
+    # column-major storage order merges the same cells
+    (pi, pj), pv, _ = oracle.sum_duplicates([ci, cj], v, dims, (1, 0))
+    assert sorted(zip(pi.tolist(), pj.tolist())) == cells
+    assert sorted(zip(pi.tolist(), pj.tolist(), pv.tolist())) == sorted((a, b, acc[(a, b)]) for a, b in cells)
+
+
+def test_sum_duplicates_adds_in_input_order():
+    # 1e16 + 1 + 1 differs from 1 + 1 + 1e16 in double: the sum must follow the order the entries were given
+    c = [np.array([2, 2, 2, 0], dtype=np.int32), np.array([1, 1, 1, 0], dtype=np.int32), np.array([3, 3, 3, 0], dtype=np.int32)]
+    _, v1, _ = oracle.sum_duplicates(c, np.array([1e16, 1.0, 1.0, 5.0]), (3, 2, 4), (0, 1, 2))
+    _, v2, _ = oracle.sum_duplicates(c, np.array([1.0, 1.0, 1e16, 5.0]), (3, 2, 4), (0, 1, 2))
+    assert v1.tolist() == [5.0, (1e16 + 1.0) + 1.0] and v2.tolist() == [5.0, (1.0 + 1.0) + 1e16] and v1[1] != v2[1]
+
+
+def test_without_the_flag_duplicates_are_still_rejected():
+    c = [np.array([1, 1], dtype=np.int32), np.array([2, 2], dtype=np.int32)]
+    with pytest.raises(oracle.OracleError):
+        oracle.pack(c, np.array([1.0, 2.0]), (3, 3), (0, 1), (oracle.D, oracle.CU))
+    pk = oracle.pack(c, np.array([1.0, 2.0]), (3, 3), (0, 1), (oracle.D, oracle.CU), sum_duplicates_first=True)
+    assert pk.val.tolist() == [3.0] and pk.crd[1].tolist() == [2] and pk.pos[1].tolist() == [0, 0, 1, 1]
