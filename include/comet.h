@@ -121,6 +121,20 @@ comet_status_t comet_pack(comet_handle_t handle, int32_t order, const int64_t *h
                           const int32_t *h_mode_order, const int32_t *h_attr, void *stream,
                           comet_sptensor_t *out);
 
+/* comet_pack with options. flags: a bitwise OR of
+ *   COMET_PACK_SUM_DUPLICATES  entries that share all coordinates are merged into one entry whose value is
+ *                              their sum, added one by one in double in the order the entries were given
+ *                              (fp32 values: summed in double, rounded once), instead of being reported as
+ *                              COMET_ERR_DUPLICATE_COORD. out->nnz is then the number of distinct cells. The
+ *                              paper does not say what a duplicate means; this is the common reading of a COO
+ *                              file and costs one more stream synchronisation and one more pass.
+ * Any other bit: COMET_ERR_INVALID_ARG. flags = 0 is comet_pack. */
+#define COMET_PACK_SUM_DUPLICATES 1u
+comet_status_t comet_pack_ex(comet_handle_t handle, int32_t order, const int64_t *h_dims, int64_t nnz,
+                             const int32_t *const *h_coo_crd, const void *coo_val, comet_dtype_t dtype,
+                             const int32_t *h_mode_order, const int32_t *h_attr, uint32_t flags, void *stream,
+                             comet_sptensor_t *out);
+
 /* Releases the arrays of a library-owned tensor (no-op for caller-built descriptors) and zeroes it. */
 comet_status_t comet_sptensor_free(comet_handle_t handle, comet_sptensor_t *tensor, void *stream);
 

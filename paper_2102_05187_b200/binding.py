@@ -50,7 +50,7 @@ EXPORTS = [
     "comet_create", "comet_destroy", "comet_status_string", "comet_last_cuda_error", "comet_kernel_launches",
     "comet_pack",
     "comet_sptensor_free", "comet_validate", "comet_spmv", "comet_spmm", "comet_ttv_symbolic", "comet_ttv",
-    "comet_ttm_symbolic", "comet_ttm", "comet_mttkrp", "comet_spmv_static",
+    "comet_ttm_symbolic", "comet_ttm", "comet_mttkrp", "comet_spmv_static", "comet_pack_ex",
 ]
 
 
@@ -288,8 +288,12 @@ def _from_ptr(ptr, n, dtype, owner):
 
 # ------------------------------------------------------------------------------------------- entry points
 
-def pack(coords, val, dims, mode_order, attr, handle: Handle | None = None) -> SpTensor:
-    """comet_pack: COO (one int32 CUDA tensor per mode, any order, distinct cells) -> packed levels."""
+PACK_SUM_DUPLICATES = 1
+
+
+def pack(coords, val, dims, mode_order, attr, handle: Handle | None = None, sum_duplicates: bool = False) -> SpTensor:
+    """comet_pack / comet_pack_ex: COO (one int32 CUDA tensor per mode, any order) -> packed levels. Cells must be
+    distinct unless `sum_duplicates`, which merges equal cells (values added in input order)."""
     handle = handle or default_handle()
     order = len(dims)
     _require_cuda(val, *coords)
@@ -301,8 +305,10 @@ def pack(coords, val, dims, mode_order, attr, handle: Handle | None = None) -> S
     h_mo = (C.c_int32 * order)(*[int(m) for m in mode_order])
     h_at = (C.c_int32 * order)(*[int(a) for a in attr])
     out = SpTensorStruct()
-    st = handle.lib.comet_pack(handle._h, C.c_int32(order), h_dims, C.c_int64(val.numel()), h_crd, _ptr(val),
-                               C.c_int(_dtype_code(val)), h_mo, h_at, _stream_ptr(), C.byref(out))
+    st = handle.lib.comet_pack_ex(handle._h, C.c_int32(order), h_dims, C.c_int64(val.numel()), h_crd, _ptr(val),
+                                  C.c_int(_dtype_code(val)), h_mo, h_at,
+                                  C.c_uint32(PACK_SUM_DUPLICATES if sum_duplicates else 0), _stream_ptr(),
+                                  C.byref(out))
     handle.check(st, "comet_pack")
     return SpTensor(handle, out)
 

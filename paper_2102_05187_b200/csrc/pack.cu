@@ -252,6 +252,33 @@ __global__ void __launch_bounds__(kSortThreads, 4) radix_scatter_kernel(
   }
 }
 
+// ------------------------------------------------------------------------------------------------ duplicates
+// COMET_PACK_SUM_DUPLICATES: after the sort, entries with equal keys are adjacent and, the sort being stable,
+// in the order they were given. The first entry of each run keeps the key; its value becomes the sum of the
+// run, added one by one in double in that order (one thread per run: runs are short unless the input is
+// degenerate). The level pass then sees distinct keys, an identity permutation and the merged values.
+__global__ void dup_heads_kernel(const uint64_t *__restrict__ keys, int64_t n, uint32_t *__restrict__ head) {
+  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (p < n) head[p] = (p == 0 || keys[p] != keys[p - 1]) ? 1u : 0u;
+}
+
+template <class V>
+__global__ void dup_merge_kernel(const uint64_t *__restrict__ keys, const uint32_t *__restrict__ perm,
+                                 const V *__restrict__ val_in, int64_t n, const uint32_t *__restrict__ rank,
+                                 uint64_t *__restrict__ keys_out, uint32_t *__restrict__ perm_out,
+                                 V *__restrict__ val_out) {
+  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= n) return;
+  const uint64_t k = keys[p];
+  if (p > 0 && keys[p - 1] == k) return;
+  double sum = (double)val_in[perm[p]];
+  for (int64_t q = p + 1; q < n && keys[q] == k; ++q) sum = sum + (double)val_in[perm[q]];
+  const uint32_t r = rank[p];
+  keys_out[r] = k;
+  perm_out[r] = r;
+  val_out[r] = (V)sum;
+}
+
 // ------------------------------------------------------------------------------------------------ levels
 struct LevelPlan {
   int order;
@@ -484,7 +511,7 @@ bool supported_attrs(int order, const int32_t *attr) {
 struct TempBlocks {
   Context *ctx;
   cudaStream_t s;
-  void *p[8];
+  void *p[12];
   int n = 0;
   TempBlocks(Context *c, cudaStream_t st) : ctx(c), s(st) {}
   void *get(size_t bytes) {
@@ -501,6 +528,14 @@ extern "C" comet_status_t comet_pack(comet_handle_t handle, int32_t order, const
                                      const int32_t *const *h_coo_crd, const void *coo_val, comet_dtype_t dtype,
                                      const int32_t *h_mode_order, const int32_t *h_attr, void *stream,
                                      comet_sptensor_t *out) {
+  return comet_pack_ex(handle, order, h_dims, nnz, h_coo_crd, coo_val, dtype, h_mode_order, h_attr, 0u, stream, out);
+}
+
+extern "C" comet_status_t comet_pack_ex(comet_handle_t handle, int32_t order, const int64_t *h_dims, int64_t nnz,
+                                        const int32_t *const *h_coo_crd, const void *coo_val, comet_dtype_t dtype,
+                                        const int32_t *h_mode_order, const int32_t *h_attr, uint32_t flags,
+                                        void *stream, comet_sptensor_t *out) {
+  if (flags & ~(uint32_t)COMET_PACK_SUM_DUPLICATES) return COMET_ERR_INVALID_ARG;
   if (!handle || !out || !h_dims || !h_coo_crd || !h_mode_order || !h_attr) return COMET_ERR_INVALID_ARG;
   memset(out, 0, sizeof(*out));
   if (order < 1 || order > COMET_MAX_ORDER || nnz < 0) return COMET_ERR_INVALID_ARG;
@@ -545,9 +580,9 @@ extern "C" comet_status_t comet_pack(comet_handle_t handle, int32_t order, const
   }
   if (h_attr[0] == COMET_D && h_dims[h_mode_order[0]] == 0 && nnz > 0) return COMET_ERR_COORD_OUT_OF_RANGE;
 
-  const int64_t n = nnz;
+  int64_t n = nnz;                     // entries the level pass sees (fewer after duplicates are merged)
   const int64_t sort_tiles = ceil_div(n > 0 ? n : 1, kSortTile);
-  const int64_t level_tiles = ceil_div(n > 0 ? n : 1, kLevelTile);
+  int64_t level_tiles = ceil_div(n > 0 ? n : 1, kLevelTile);
   const int64_t table_len = 256 * sort_tiles;
   const int64_t counts_len = (int64_t)COMET_MAX_ORDER * level_tiles;
 
@@ -579,6 +614,35 @@ extern "C" comet_status_t comet_pack(comet_handle_t handle, int32_t order, const
       COMET_LAUNCH_CHECK(ctx);
       uint64_t *tk = keys_a; keys_a = keys_b; keys_b = tk;
       uint32_t *tp = perm_a; perm_a = perm_b; perm_b = tp;
+    }
+    if (flags & COMET_PACK_SUM_DUPLICATES) {
+      // merge runs of equal keys; costs one more synchronisation (the number of distinct cells sizes the rest)
+      uint32_t *rank = (uint32_t *)tmp.get((size_t)n * 4);
+      void *merged = tmp.get((size_t)n * (dtype == COMET_F32 ? 4 : 8));
+      if (!rank || !merged) return COMET_ERR_ALLOC;
+      uint32_t *d_distinct = reinterpret_cast<uint32_t *>(ctx->d_status) + 12;
+      dup_heads_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(keys_a, n, rank);
+      COMET_LAUNCH_CHECK(ctx);
+      uint32_t *rank_tmp = (uint32_t *)keys_b;                 // free until the merge writes it
+      comet_status_t st = exclusive_scan(ctx, rank, rank, n, rank_tmp, d_distinct, s);
+      if (st != COMET_OK) return st;
+      COMET_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->h_pinned, ctx->d_status, 16 * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+      COMET_CUDA_TRY(ctx, cudaStreamSynchronize(s));
+      if (ctx->h_pinned[kStatusRange]) return COMET_ERR_COORD_OUT_OF_RANGE;
+      const int64_t distinct = reinterpret_cast<uint32_t *>(ctx->h_pinned)[12];
+      // keys_b is both the scan's scratch and the merge's output: the scan has finished (synchronised above)
+      if (dtype == COMET_F32)
+        dup_merge_kernel<float><<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(keys_a, perm_a, (const float *)coo_val, n, rank,
+                                                                          keys_b, perm_b, (float *)merged);
+      else
+        dup_merge_kernel<double><<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(keys_a, perm_a, (const double *)coo_val, n,
+                                                                           rank, keys_b, perm_b, (double *)merged);
+      COMET_LAUNCH_CHECK(ctx);
+      keys_a = keys_b;
+      perm_a = perm_b;
+      coo_val = merged;
+      n = distinct;
+      level_tiles = ceil_div(n > 0 ? n : 1, kLevelTile);
     }
     // node counts of the counted levels: per-tile counts -> scanned offsets (kept in `table`) + totals
     if (order == 2) level_count_kernel<2><<<(unsigned)level_tiles, kLevelThreads, 0, s>>>(keys_a, n, plan, level_tiles, table, ctx->d_status);

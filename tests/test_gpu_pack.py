@@ -145,3 +145,65 @@ def test_pack_then_contract_end_to_end():
     Y = comet.ttm(X, 2, case.dense["U"].cuda())
     _, want, norm = oracle.ttm(_np(case.coords), case.val.numpy(), case.dims, 2, case.dense["U"].numpy())
     assert_close(Y.val.reshape(-1, case.R), want, norm, what="pack+ttm")
+
+
+# ----------------------------------------------------------------------------- COMET_PACK_SUM_DUPLICATES
+def _with_duplicates(dims, n, seed):
+    """n entries over few cells (many repeats), values of very different magnitudes so that the order of the
+    additions shows in the last bits."""
+    g = np.random.default_rng(seed)
+    coords = [torch.from_numpy(g.integers(0, d, n).astype(np.int32)) for d in dims]
+    val = torch.from_numpy(g.standard_normal(n) * 10.0 ** g.integers(-8, 9, n))
+    return coords, val
+
+
+@pytest.mark.parametrize("dims,n,attr,mode_order", [
+    ((7, 9), 400, (D, CU), (0, 1)), ((7, 9), 400, (CU, CU), (1, 0)), ((7, 9), 400, (CN, S), (0, 1)),
+    ((40, 30), 20000, (D, CU), (0, 1)), ((6, 5, 4), 3000, (CU, CU, CU), (2, 0, 1)), ((6, 5, 4), 3000, (CN, S, S), (0, 1, 2)),
+    ((30, 20, 10), 50000, (D, CU, CU), (1, 2, 0)), ((5, 4, 3, 2), 4000, (CU, CU, CU, CU), (3, 2, 1, 0)),
+    ((1, 1), 1000, (D, CU), (0, 1)), ((300, 200), 500, (D, CU), (0, 1))])
+def test_pack_sum_duplicates_bit_exact(dims, n, attr, mode_order):
+    coords, val = _with_duplicates(dims, n, 17)
+    want = oracle.pack(_np(coords), val.numpy(), dims, mode_order, attr, sum_duplicates_first=True)
+    got = comet.pack([c.cuda() for c in coords], val.cuda(), dims, mode_order, attr, sum_duplicates=True)
+    assert got.nnz == len(want.val) and got.nnz <= n
+    for l in range(len(dims)):
+        assert_equal_arrays(got.pos(l), want.pos[l], f"pos[{l}]")
+        assert_equal_arrays(got.crd(l), want.crd[l], f"crd[{l}]")
+    assert_equal_arrays(got.val, want.val, "merged values")        # same additions in the same order: same bits
+    comet.validate(got)
+    with pytest.raises(comet.CometError) as e:                     # without the flag the same input is refused
+        comet.pack([c.cuda() for c in coords], val.cuda(), dims, mode_order, attr)
+    assert comet.binding.STATUS_NAMES[e.value.status] == "COMET_ERR_DUPLICATE_COORD"
+
+
+def test_pack_sum_duplicates_is_a_no_op_on_distinct_cells_and_handles_empty_and_fp32():
+    dims = (60, 50, 40)
+    coords, val = synth.random_coo(dims, 20000, 6)
+    a = comet.pack([c.cuda() for c in coords], val.cuda(), dims, (0, 1, 2), (CU, CU, CU))
+    b = comet.pack([c.cuda() for c in coords], val.cuda(), dims, (0, 1, 2), (CU, CU, CU), sum_duplicates=True)
+    assert a.nnz == b.nnz and torch.equal(a.val, b.val)
+    for l in range(3):
+        assert torch.equal(a.pos(l), b.pos(l)) and torch.equal(a.crd(l), b.crd(l))
+    e = comet.pack([torch.zeros(0, dtype=torch.int32, device="cuda")] * 2, torch.zeros(0, dtype=torch.float64, device="cuda"),
+                   (4, 4), (0, 1), (D, CU), sum_duplicates=True)
+    assert e.nnz == 0 and e.pos(1).tolist() == [0, 0, 0, 0, 0]
+    dc, dv = _with_duplicates((7, 9), 400, 3)
+    v32 = dv.float()
+    want = oracle.pack(_np(dc), v32.double().numpy(), (7, 9), (0, 1), (D, CU), sum_duplicates_first=True)
+    got = comet.pack([c.cuda() for c in dc], v32.cuda(), (7, 9), (0, 1), (D, CU), sum_duplicates=True)
+    assert got.val.dtype == torch.float32
+    assert np.array_equal(got.val.cpu().numpy(), want.val.astype(np.float32))   # summed in double, rounded once
+
+
+def test_pack_ex_rejects_unknown_flags():
+    import ctypes as C
+    h = comet.default_handle()
+    out = comet.binding.SpTensorStruct()
+    dims = (C.c_int64 * 2)(2, 2)
+    crd = (C.c_void_p * 2)(0, 0)
+    mo = (C.c_int32 * 2)(0, 1)
+    at = (C.c_int32 * 2)(D, CU)
+    st = h.lib.comet_pack_ex(h._h, C.c_int32(2), dims, C.c_int64(0), crd, None, C.c_int(0), mo, at, C.c_uint32(6), None,
+                             C.byref(out))
+    assert st == -1
