@@ -182,6 +182,12 @@ comet_status_t comet_ttv(comet_handle_t handle, const comet_sptensor_t *X, int32
  * comet_ttm writes only Y->val. Formats of X as for comet_ttv (COO: see the note there). */
 comet_status_t comet_ttm_symbolic(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode, int64_t R,
                                   void *stream, comet_sptensor_t *Y);
+/* comet_ttm_symbolic with a choice of result format. h_out_attr (one attribute per level of Y): the default
+ * {CU,..,CU,D}, or, for a 3-order X, the mode-generic form {CN,S,D} that the paper names for semi-sparse
+ * tensors: pos[0] = [0, #fibers], crd[0] / crd[1] hold one coordinate pair per stored fiber (sorted), and val is
+ * the same #fibers x R matrix. NULL selects the default. comet_ttm takes either kind of Y. */
+comet_status_t comet_ttm_symbolic_ex(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode, int64_t R,
+                                     const int32_t *h_out_attr, void *stream, comet_sptensor_t *Y);
 comet_status_t comet_ttm(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode, const void *U, int64_t R,
                          int64_t ldu, comet_sptensor_t *Y, void *stream);
 

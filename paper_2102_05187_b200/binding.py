@@ -50,7 +50,7 @@ EXPORTS = [
     "comet_create", "comet_destroy", "comet_status_string", "comet_last_cuda_error", "comet_kernel_launches",
     "comet_pack",
     "comet_sptensor_free", "comet_validate", "comet_spmv", "comet_spmm", "comet_ttv_symbolic", "comet_ttv",
-    "comet_ttm_symbolic", "comet_ttm", "comet_mttkrp", "comet_spmv_static", "comet_pack_ex",
+    "comet_ttm_symbolic", "comet_ttm", "comet_mttkrp", "comet_spmv_static", "comet_pack_ex", "comet_ttm_symbolic_ex",
 ]
 
 
@@ -366,10 +366,13 @@ def ttv(X: SpTensor, mode: int, v: torch.Tensor, Y: SpTensor | None = None) -> S
     return Y
 
 
-def ttm_symbolic(X: SpTensor, mode: int, R: int) -> SpTensor:
+def ttm_symbolic(X: SpTensor, mode: int, R: int, out_attr=None) -> SpTensor:
+    """Structure of X x_mode U. out_attr: None (compressed levels + dense last level) or, for a 3-order X,
+    (CN, S, D): the mode-generic form with one coordinate pair per stored fiber."""
     out = SpTensorStruct()
-    st = X.handle.lib.comet_ttm_symbolic(X.handle._h, C.byref(X.c), C.c_int32(mode), C.c_int64(R), _stream_ptr(),
-                                         C.byref(out))
+    h_at = None if out_attr is None else (C.c_int32 * X.c.order)(*out_attr)
+    st = X.handle.lib.comet_ttm_symbolic_ex(X.handle._h, C.byref(X.c), C.c_int32(mode), C.c_int64(R), h_at,
+                                            _stream_ptr(), C.byref(out))
     X.handle.check(st, "comet_ttm_symbolic")
     return SpTensor(X.handle, out)
 

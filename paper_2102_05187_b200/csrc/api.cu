@@ -76,6 +76,23 @@ __global__ void expand_root_pos_kernel(const int32_t *__restrict__ crd0, const i
 }
 
 __global__ void set_word_kernel(int32_t *p, int32_t v) { *p = v; }
+__global__ void set_two_words_kernel(int32_t *p, int32_t v0, int32_t v1) { p[0] = v0; p[1] = v1; }
+
+// Coordinates of every fiber of a 3-level CSF structure: out0[f] = crd0[slice that holds f], out1[f] = crd1[f]
+// (the slice is the last one whose first fiber is at or before f).
+__global__ void fiber_coords_kernel(const int32_t *__restrict__ pos1, const int32_t *__restrict__ crd0,
+                                    const int32_t *__restrict__ crd1, int64_t S, int64_t F, int32_t *__restrict__ out0,
+                                    int32_t *__restrict__ out1) {
+  const int64_t f = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (f >= F) return;
+  int64_t lo = 0, hi = S;
+  while (hi - lo > 1) {
+    const int64_t mid = (lo + hi) >> 1;
+    if ((int64_t)__ldg(pos1 + mid) <= f) lo = mid; else hi = mid;
+  }
+  out0[f] = __ldg(crd0 + lo);
+  out1[f] = __ldg(crd1 + f);
+}
 
 // CSR pos of a sorted COO matrix: pos[i] = number of entries whose root coordinate is below i
 __global__ void coo_row_pos_kernel(const int32_t *__restrict__ crd0, int64_t n, int64_t rows, int32_t *__restrict__ pos) {
@@ -405,10 +422,25 @@ extern "C" comet_status_t comet_ttv(comet_handle_t handle, const comet_sptensor_
 
 extern "C" comet_status_t comet_ttm_symbolic(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode,
                                              int64_t R, void *stream, comet_sptensor_t *Y) {
+  return comet_ttm_symbolic_ex(handle, X, mode, R, nullptr, stream, Y);
+}
+
+extern "C" comet_status_t comet_ttm_symbolic_ex(comet_handle_t handle, const comet_sptensor_t *X, int32_t mode,
+                                                int64_t R, const int32_t *h_out_attr, void *stream,
+                                                comet_sptensor_t *Y) {
   if (!handle || !Y || R < 1) return COMET_ERR_INVALID_ARG;
   if (R > kIndexLimit) return COMET_ERR_INDEX_OVERFLOW;
   comet_status_t st = check_last_mode(X, mode);
   if (st != COMET_OK) return st;
+  // result format: compressed upper levels + dense last level (default), or, for 3-order inputs, the
+  // mode-generic form [CN,S,D]: one coordinate pair per stored fiber + dense last level
+  bool generic = false;
+  if (h_out_attr) {
+    bool semi = h_out_attr[X->order - 1] == COMET_D;
+    for (int l = 0; l + 1 < X->order; ++l) semi = semi && h_out_attr[l] == COMET_CU;
+    generic = X->order == 3 && h_out_attr[0] == COMET_CN && h_out_attr[1] == COMET_S && h_out_attr[2] == COMET_D;
+    if (!semi && !generic) return COMET_ERR_UNSUPPORTED_FORMAT;
+  }
   Context *ctx = reinterpret_cast<Context *>(handle);
   cudaStream_t s = (cudaStream_t)stream;
   memset(Y, 0, sizeof(*Y));
@@ -430,7 +462,25 @@ extern "C" comet_status_t comet_ttm_symbolic(comet_handle_t handle, const comet_
   for (int l = 0; l < last; ++l) Y->attr[l] = COMET_CU;
   Y->attr[last] = COMET_D;
   Y->nnz = F * R;
-  st = copy_upper_levels(ctx, X, Y, o, s);
+  if (generic) {
+    Y->attr[0] = COMET_CN; Y->attr[1] = COMET_S;
+    Y->pos_len[0] = 2; Y->crd_len[0] = F; Y->crd_len[1] = F;
+    Y->pos[0] = (int32_t *)owned_alloc(ctx, o, 8, s);
+    Y->crd[0] = (int32_t *)owned_alloc(ctx, o, (size_t)(F > 0 ? F : 1) * 4, s);
+    Y->crd[1] = (int32_t *)owned_alloc(ctx, o, (size_t)(F > 0 ? F : 1) * 4, s);
+    if (!Y->pos[0] || !Y->crd[0] || !Y->crd[1]) st = COMET_ERR_ALLOC;
+    else {
+      set_two_words_kernel<<<1, 1, 0, s>>>(Y->pos[0], 0, (int32_t)F);
+      if (F > 0)
+        fiber_coords_kernel<<<(unsigned)ceil_div(F, 256), 256, 0, s>>>(X->pos[1], X->crd[0], X->crd[1], X->crd_len[0], F,
+                                                                      Y->crd[0], Y->crd[1]);
+      ctx->launches += F > 0 ? 2 : 1;
+      cudaError_t e = cudaGetLastError();
+      if (e != cudaSuccess) st = cuda_fail(ctx, e);
+    }
+  } else {
+    st = copy_upper_levels(ctx, X, Y, o, s);
+  }
   if (st == COMET_OK) {
     Y->pos_len[last] = 1;
     Y->pos[last] = (int32_t *)owned_alloc(ctx, o, 4, s);

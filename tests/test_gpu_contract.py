@@ -306,6 +306,29 @@ def test_order4_packed_on_the_device_then_contracted():
     assert abs(np.sort(got) - np.sort(want[:, 0])).max() <= 1e-12 * norm.max()
 
 
+@pytest.mark.parametrize("dims,nnz,seed", TENSOR_CASES)
+@pytest.mark.parametrize("attr", [(CU, CU, CU), (CN, S, S)])
+def test_ttm_mode_generic_output(dims, nnz, seed, attr):
+    """[CN,S,D] result: one coordinate pair per stored fiber, the same values as the default [CU,CU,D] result."""
+    coords, val = synth.random_coo(dims, nnz, seed)
+    c, v = _np(coords), val.numpy()
+    mode, R = 2, 6
+    X = upload_packed(oracle.pack(c, v, dims, (0, 1, 2), attr))
+    U = synth.random_dense((dims[mode], R), seed + 1).numpy()
+    keys, want, norm = oracle.ttm(c, v, dims, mode, U)
+    Z = comet.ttm_symbolic(X, mode, R, (CN, S, D))
+    assert Z.attr == (CN, S, D) and Z.dims == (dims[0], dims[1], R) and Z.c.nnz == len(keys) * R
+    assert Z.pos(0).tolist() == [0, len(keys)] and Z.pos(2).tolist() == [R]
+    assert_equal_arrays(Z.crd(0), (keys // dims[1]).astype(np.int32), "fiber coordinates of mode 0")
+    assert_equal_arrays(Z.crd(1), (keys % dims[1]).astype(np.int32), "fiber coordinates of mode 1")
+    Z.val.fill_(float("nan"))
+    comet.ttm(X, mode, dev(U), Z)
+    assert_close(Z.val.reshape(-1, R), want, norm, what="mode-generic ttm")
+    with pytest.raises(comet.CometError) as e:
+        comet.ttm_symbolic(X, mode, R, (D, CU, D))
+    assert e.value.status == -2
+
+
 def test_ttv_numeric_phase_rejects_a_result_built_for_another_tensor():
     dims = (12, 11, 10)
     coords, val = synth.random_coo(dims, 400, 3)
