@@ -212,6 +212,25 @@ comet_status_t comet_mttkrp(comet_handle_t handle, const comet_sptensor_t *X, in
                             const void *const *h_factors, const int64_t *h_ld, int64_t R, void *out, int64_t ldo,
                             void *stream);
 
+/* Reordering pre-pass (Data Reordering section: sort one dimension at a time lexicographically by the
+ * coordinates of its entries in the other dimensions, all dimensions in turn, to gather the entries around the
+ * diagonal). The paper gives no further detail; this call keeps the first element of each index's sorted entry
+ * list: in a step for mode m, key(x) = the smallest tuple (current numbers of the other modes' coordinates, in
+ * increasing mode order) over the entries with mode-m index x, +infinity for an index without entries, and the
+ * indices are re-numbered in ascending key order, ties in the order of their current numbers. One iteration is
+ * a step for every mode in turn.
+ *   h_coo_crd[order]    HOST array of DEVICE pointers: int32[nnz] coordinates per mode (COO, any order;
+ *                       duplicates allowed); orders 2 and 3
+ *   h_new_label[order]  HOST array of DEVICE pointers: int32[dims[m]] OUT, new_label[m][x] = the new number of
+ *                       original index x (a permutation of 0..dims[m]-1; the identity for iterations = 0)
+ * The caller applies it: coordinates become new_label[m][c], row j of a dense operand indexed by mode m moves to
+ * row new_label[m][j], and row i of a result indexed by mode m is found at row new_label[m][i]. The result of
+ * a contraction is unchanged up to that relabelling. Synchronises `stream` once (coordinate range check);
+ * COMET_ERR_COORD_OUT_OF_RANGE leaves the labels at the identity. */
+comet_status_t comet_reorder(comet_handle_t handle, int32_t order, const int64_t *h_dims, int64_t nnz,
+                             const int32_t *const *h_coo_crd, int32_t iterations, int32_t *const *h_new_label,
+                             void *stream);
+
 /* CSR SpMV without any allocation (the paper has no counterpart; this exists for deployment only).
  *
  * Who needs it: callers that cannot obtain device memory at call time. Examples are a service whose

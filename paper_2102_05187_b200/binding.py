@@ -50,7 +50,7 @@ EXPORTS = [
     "comet_create", "comet_destroy", "comet_status_string", "comet_last_cuda_error", "comet_kernel_launches",
     "comet_pack",
     "comet_sptensor_free", "comet_validate", "comet_spmv", "comet_spmm", "comet_ttv_symbolic", "comet_ttv",
-    "comet_ttm_symbolic", "comet_ttm", "comet_mttkrp", "comet_spmv_static", "comet_pack_ex", "comet_ttm_symbolic_ex",
+    "comet_ttm_symbolic", "comet_ttm", "comet_mttkrp", "comet_spmv_static", "comet_pack_ex", "comet_ttm_symbolic_ex", "comet_reorder",
 ]
 
 
@@ -408,6 +408,25 @@ def mttkrp(X: SpTensor, mode: int, factors, out: torch.Tensor | None = None) -> 
                                    C.c_int64(out.stride(0)), _stream_ptr())
     X.handle.check(st, "comet_mttkrp")
     return out
+
+
+def reorder(coords, dims, iterations: int = 5, handle: Handle | None = None):
+    """comet_reorder: new numbers for the indices of every mode (one int32 CUDA tensor per mode) that gather
+    the entries around the diagonal. Apply with `label[m][coords[m].long()]`; dense operands and results
+    indexed by mode m move their rows accordingly."""
+    handle = handle or default_handle()
+    order = len(dims)
+    _require_cuda(*coords)
+    coords = [c.contiguous() for c in coords]
+    assert all(c.dtype == torch.int32 for c in coords)
+    labels = [torch.empty(int(d), dtype=torch.int32, device=coords[0].device) for d in dims]
+    h_dims = (C.c_int64 * order)(*[int(d) for d in dims])
+    h_crd = (C.c_void_p * order)(*[c.data_ptr() for c in coords])
+    h_lab = (C.c_void_p * order)(*[l.data_ptr() for l in labels])
+    st = handle.lib.comet_reorder(handle._h, C.c_int32(order), h_dims, C.c_int64(coords[0].numel()), h_crd,
+                                  C.c_int32(iterations), h_lab, _stream_ptr())
+    handle.check(st, "comet_reorder")
+    return labels
 
 
 _copy_stream = None

@@ -52,6 +52,13 @@ int64_t scan_tmp_words(int64_t n);
 comet_status_t exclusive_scan(Context *ctx, const uint32_t *in, uint32_t *out, int64_t n, uint32_t *tmp,
                               uint32_t *total, cudaStream_t s);
 
+// Stable LSD radix sort of (64-bit key, 32-bit payload) pairs over the low `bits` key bits (pack.cu). The sorted
+// pairs end up behind `ka` / `pa` (the pointers are swapped with `kb` / `pb` after every pass); every buffer holds
+// n + 1 elements, `table` radix_sort_table_words(n) words and `scan_tmp` scan_tmp_words(that) words.
+int64_t radix_sort_table_words(int64_t n);
+comet_status_t radix_sort_pairs(Context *ctx, uint64_t *&ka, uint64_t *&kb, uint32_t *&pa, uint32_t *&pb, int64_t n,
+                                int bits, uint32_t *table, uint32_t *scan_tmp, cudaStream_t s);
+
 int32_t choose_tile_items(int64_t total_items, int workers_per_block);
 
 // Block list of a library-owned tensor (what comet_sptensor_free releases).

@@ -252,6 +252,28 @@ __global__ void __launch_bounds__(kSortThreads, 4) radix_scatter_kernel(
   }
 }
 
+// Stable LSD radix sort of (key, payload) pairs over the low `bits` key bits, 8 bits per pass. `ka`/`pa` hold
+// the input and, on return, the sorted pairs (the pointers are swapped with `kb`/`pb` after every pass); all four
+// buffers hold n + 1 elements. `table` holds radix_sort_table_words(n) words, `scan_tmp` scan_tmp_words of that.
+int64_t radix_sort_table_words(int64_t n) { return 256 * ceil_div(n > 0 ? n : 1, kSortTile); }
+
+comet_status_t radix_sort_pairs(Context *ctx, uint64_t *&ka, uint64_t *&kb, uint32_t *&pa, uint32_t *&pb, int64_t n,
+                                int bits, uint32_t *table, uint32_t *scan_tmp, cudaStream_t s) {
+  if (n <= 0) return COMET_OK;
+  const int64_t tiles = ceil_div(n, kSortTile);
+  for (int shift = 0; shift < bits; shift += 8) {
+    radix_histogram_kernel<<<(unsigned)tiles, kSortThreads, 0, s>>>(ka, n, shift, tiles, table);
+    COMET_LAUNCH_CHECK(ctx);
+    comet_status_t st = exclusive_scan(ctx, table, table, 256 * tiles, scan_tmp, nullptr, s);
+    if (st != COMET_OK) return st;
+    radix_scatter_kernel<<<(unsigned)tiles, kSortThreads, 0, s>>>(ka, pa, kb, pb, table, n, shift, tiles);
+    COMET_LAUNCH_CHECK(ctx);
+    uint64_t *tk = ka; ka = kb; kb = tk;
+    uint32_t *tp = pa; pa = pb; pb = tp;
+  }
+  return COMET_OK;
+}
+
 // ------------------------------------------------------------------------------------------------ duplicates
 // COMET_PACK_SUM_DUPLICATES: after the sort, entries with equal keys are adjacent and, the sort being stable,
 // in the order they were given. The first entry of each run keeps the key; its value becomes the sum of the
@@ -604,16 +626,9 @@ extern "C" comet_status_t comet_pack_ex(comet_handle_t handle, int32_t order, co
     else if (order == 3) make_keys_kernel<3><<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(coords, key, n, keys_a, perm_a, ctx->d_status);
     else make_keys_kernel<4><<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(coords, key, n, keys_a, perm_a, ctx->d_status);
     COMET_LAUNCH_CHECK(ctx);
-    for (int shift = 0; shift < total_bits; shift += 8) {
-      radix_histogram_kernel<<<(unsigned)sort_tiles, kSortThreads, 0, s>>>(keys_a, n, shift, sort_tiles, table);
-      COMET_LAUNCH_CHECK(ctx);
-      comet_status_t st = exclusive_scan(ctx, table, table, table_len, scan_tmp, nullptr, s);
+    {
+      comet_status_t st = radix_sort_pairs(ctx, keys_a, keys_b, perm_a, perm_b, n, total_bits, table, scan_tmp, s);
       if (st != COMET_OK) return st;
-      radix_scatter_kernel<<<(unsigned)sort_tiles, kSortThreads, 0, s>>>(keys_a, perm_a, keys_b, perm_b, table, n,
-                                                                         shift, sort_tiles);
-      COMET_LAUNCH_CHECK(ctx);
-      uint64_t *tk = keys_a; keys_a = keys_b; keys_b = tk;
-      uint32_t *tp = perm_a; perm_a = perm_b; perm_b = tp;
     }
     if (flags & COMET_PACK_SUM_DUPLICATES) {
       // merge runs of equal keys; costs one more synchronisation (the number of distinct cells sizes the rest)
