@@ -412,6 +412,184 @@ seg_dot_stream_kernel(const SegDotArgs a, int64_t x_len, int32_t span, unsigned 
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// The same walk with 64 entries per step: lane l owns entries 2l and 2l+1 of the step (one 8-byte and one
+// 16-byte load per step and lane), so a step that contains a segment end -- the expensive kind: segmented
+// scan, warp sum of the private partials, stores -- pays for 64 entries instead of 32. Inside a lane the
+// pair is summed before the scan unless a segment ends between its two entries; a lane then contributes a
+// "tail" (the sub-sum still open at its second entry, which the lane-level scan extends) and, if a segment
+// ends at its first entry, a "head" sum (its first product plus the tail of the lane before it).
+#ifndef COMET_STREAM2_STEPS
+#define COMET_STREAM2_STEPS 3      // 64-entry steps whose loads are issued together (4 spills registers)
+#endif
+template <class T> struct Pair2;
+template <> struct Pair2<double> {
+  static __device__ __forceinline__ void load(const double *p, double &a, double &b) {
+    const double2 t = __ldcs(reinterpret_cast<const double2 *>(p));
+    a = t.x; b = t.y;
+  }
+};
+template <> struct Pair2<float> {
+  static __device__ __forceinline__ void load(const float *p, double &a, double &b) {
+    const float2 t = __ldcs(reinterpret_cast<const float2 *>(p));
+    a = (double)t.x; b = (double)t.y;
+  }
+};
+
+template <class T, bool XSMEM>
+__global__ void __launch_bounds__(1024, 1)
+seg_dot_stream2_kernel(const SegDotArgs a, int64_t x_len, int32_t span, unsigned long long *next_tile) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const T *s_x = reinterpret_cast<const T *>(smem_raw);
+  const T *const val = static_cast<const T *>(a.val), *const x = static_cast<const T *>(a.x);
+  T *const y = static_cast<T *>(a.y);
+  if (XSMEM) {
+    T *w = reinterpret_cast<T *>(smem_raw);
+    for (int64_t i = threadIdx.x; i < x_len; i += blockDim.x) w[i] = __ldg(x + i);
+    __syncthreads();
+  }
+  const unsigned full = 0xffffffffu;
+  const int lane = threadIdx.x & 31;
+  auto xval = [&](int32_t c) -> double { return XSMEM ? (double)s_x[c] : (double)__ldg(x + c); };
+  auto warp_sum = [&](double v) -> double {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(full, v, off);
+    return v;
+  };
+
+  while (true) {
+    int64_t tile = 0;
+    if (lane == 0) tile = atomicAdd(next_tile, 1ull);
+    tile = __shfl_sync(full, tile, 0);
+    if (tile >= a.num_tiles) break;
+    const int32_t w0 = (int32_t)(tile * span);
+    const int32_t w1 = (int64_t)w0 + span < a.N ? w0 + span : (int32_t)a.N;
+    const bool whole = w1 - w0 == span && span % (64 * COMET_STREAM2_STEPS) == 0;   // full rounds only: no bounds checks inside
+
+    int64_t lo = 0, hi = a.M;                            // open segment: the first one whose end lies beyond w0
+    while (lo < hi) {
+      const int64_t stride = (hi - lo + 31) / 32;
+      const int64_t q = lo + (int64_t)lane * stride + stride - 1;
+      const bool inside = q < hi && __ldg(a.seg_end + q) <= w0;
+      const int fullr = __popc(__ballot_sync(full, inside));
+      lo += (int64_t)fullr * stride;
+      const int64_t cap = lo + stride - 1;
+      if (cap < hi) hi = cap;
+    }
+    int64_t s = lo;
+    if (tile == 0)
+      for (int64_t q = lane; q < s; q += 32) y[a.out_row ? (int64_t)__ldg(a.out_row + q) : q] = (T)0;
+
+    // ends of the next 32 segments, and of the 32 after them: closing k segments shifts the window by k with
+    // shuffles, and the load that refills the far half is not waited for until the shift after
+    int32_t ew = (s + lane < a.M) ? __ldg(a.seg_end + s + lane) : 0x7fffffff;
+    int32_t ew2 = (s + 32 + lane < a.M) ? __ldg(a.seg_end + s + 32 + lane) : 0x7fffffff;
+    int32_t last_end = w0;
+    double run = 0.0;
+
+    for (int32_t j0 = w0; j0 < w1; j0 += 64 * COMET_STREAM2_STEPS) {   // the loads of a round's steps are issued together
+      int32_t c[COMET_STREAM2_STEPS][2];
+      double v[COMET_STREAM2_STEPS][2];
+#pragma unroll
+      for (int u = 0; u < COMET_STREAM2_STEPS; ++u) {
+        const int32_t jj = j0 + u * 64 + 2 * lane;
+        if (whole) {
+          const int2 cc = __ldcs(reinterpret_cast<const int2 *>(a.crd + jj));
+          c[u][0] = cc.x; c[u][1] = cc.y;
+          Pair2<T>::load(val + jj, v[u][0], v[u][1]);
+        } else {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            c[u][h] = 0; v[u][h] = 0.0;
+            if (jj + h < w1) { c[u][h] = ld_stream(a.crd + jj + h); v[u][h] = (double)ld_stream(val + jj + h); }
+          }
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < COMET_STREAM2_STEPS; ++u) {
+        const int32_t j = j0 + u * 64;
+        if (!whole && j >= w1) break;
+        const int32_t q0 = j + 2 * lane;
+        const double p0 = (whole || q0 < w1) ? v[u][0] * xval(c[u][0]) : 0.0;
+        const double p1 = (whole || q0 + 1 < w1) ? v[u][1] * xval(c[u][1]) : 0.0;
+        const int32_t top = (whole || j + 64 < w1) ? j + 64 : w1;   // segments with an end in (j, top] close in this step
+        if (!__any_sync(full, ew <= top)) { run += p0 + p1; continue; }
+
+        // every end that falls into this step, as one bit per entry position (64 of them)
+        unsigned elo, ehi;
+        {
+          const bool closing = ew <= top;
+          const int b = ew - j - 1;
+          elo = __reduce_or_sync(full, (closing && b < 32) ? 1u << b : 0u);
+          ehi = __reduce_or_sync(full, (closing && b >= 32) ? 1u << (b - 32) : 0u);
+          if (__all_sync(full, closing)) {
+            for (int64_t more = s + 32;; more += 32) {
+              const int32_t e2 = (more + lane < a.M) ? __ldg(a.seg_end + more + lane) : 0x7fffffff;
+              const bool c2 = e2 <= top;
+              const int b2 = e2 - j - 1;
+              elo |= __reduce_or_sync(full, (c2 && b2 < 32) ? 1u << b2 : 0u);
+              ehi |= __reduce_or_sync(full, (c2 && b2 >= 32) ? 1u << (b2 - 32) : 0u);
+              if (!__all_sync(full, c2)) break;
+            }
+          }
+        }
+        const unsigned long long endbits = (unsigned long long)elo | ((unsigned long long)ehi << 32);
+        const bool e0 = (endbits >> (2 * lane)) & 1ull, e1 = (endbits >> (2 * lane + 1)) & 1ull;
+        const unsigned E0 = __ballot_sync(full, e0), E1 = __ballot_sync(full, e1);
+        // lane-level scan of the tails: a lane starts a fresh sub-sum when a segment ends at its first entry
+        // or at the second entry of the lane before it
+        const unsigned heads = E0 | (E1 << 1) | 1u;
+        const int dist = lane - (31 - __clz(heads & (0xffffffffu >> (31 - lane))));
+        double sc = e0 ? p1 : p0 + p1;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const double t = __shfl_up_sync(full, sc, off);
+          if (off <= dist) sc += t;
+        }
+        // sum of the segment that ends at this lane's FIRST entry: that product plus what the lane before left open
+        const double before = __shfl_up_sync(full, sc, 1);
+        const double hd = p0 + ((lane > 0 && !((E1 >> (lane - 1)) & 1u)) ? before : 0.0);
+        const int firstb = elo ? __ffs(elo) - 1 : 32 + __ffs(ehi) - 1;
+        const int lastb = ehi ? 63 - __clz(ehi) : 31 - __clz(elo);
+        const double tot = warp_sum(run);                // what earlier steps hold for the segment closed first
+        run = (2 * lane > lastb ? p0 : 0.0) + (2 * lane + 1 > lastb ? p1 : 0.0);   // entries behind the last end
+
+        while (true) {                                   // emit: each lane owns the segment whose end it caches
+          const bool closing = ew <= top;
+          const unsigned cm = __ballot_sync(full, closing);
+          const int b = closing ? ew - j - 1 : 0;
+          const double tail = __shfl_sync(full, sc, b >> 1), head = __shfl_sync(full, hd, b >> 1);
+          double segsum = (b & 1) ? tail : head;
+          int32_t prev = __shfl_up_sync(full, ew, 1);
+          if (lane == 0) prev = last_end;
+          if (closing) {
+            if (ew == prev) segsum = 0.0;                // an empty segment: its end repeats its predecessor's
+            else if (b == firstb) segsum += tot;
+            const int64_t seg = s + lane;
+            y[a.out_row ? (int64_t)__ldg(a.out_row + seg) : seg] = (T)segsum;
+          }
+          const int k = __popc(cm);                      // closing lanes are a prefix: ends are sorted; k >= 1
+          last_end = __shfl_sync(full, ew, k - 1);
+          s += k;
+          // shift the window by k: lanes take the end k places up, from this window or from the next one
+          const int from = lane + k;
+          const int32_t near = __shfl_sync(full, ew, from & 31), far = __shfl_sync(full, ew2, from & 31);
+          ew = from < 32 ? near : far;
+          const int32_t fresh = (s + 32 + lane < a.M) ? __ldg(a.seg_end + s + 32 + lane) : 0x7fffffff;
+          ew2 = fresh;
+          if (k < 32) break;                             // lane k's end lies beyond this step: nothing more closes
+          if (!__any_sync(full, ew <= top)) break;
+        }
+      }
+    }
+    const double open = warp_sum(run);
+    if (lane == 0) {
+      a.carry_seg[tile] = s < a.M ? (int32_t)s : -1;
+      a.carry_val[tile] = open;
+    }
+  }
+}
+
 template <class T, int THREADS, int IPT>
 static comet_status_t launch_dot(Context *ctx, SegDotArgs a, cudaStream_t stream) {
   const int64_t total = a.M + a.N;
@@ -470,14 +648,18 @@ static comet_status_t launch_resident(Context *ctx, SegDotArgs a, int64_t x_len,
 }
 
 template <class T>
-static comet_status_t launch_stream(Context *ctx, SegDotArgs a, int64_t x_len, cudaStream_t stream) {
+static comet_status_t launch_stream(Context *ctx, SegDotArgs a, int64_t x_len, bool pairs, cudaStream_t stream) {
   const size_t x_bytes = align_up((size_t)x_len * sizeof(T), 16);
   const bool xsmem = x_bytes <= kMaxDynamicSmem - 1024;
-  // spans: a multiple of 128 entries, several per warp of the 148 persistent CTAs so that the tail is short
+  // the two-entries-per-lane kernel loads pairs with one instruction: the arrays must be aligned for that
+  pairs = pairs && (reinterpret_cast<uintptr_t>(a.crd) % 8 == 0) && (reinterpret_cast<uintptr_t>(a.val) % (2 * sizeof(T)) == 0);
+  // spans: whole rounds of the kernel (128 entries, or 64 per step of the pair kernel), several per warp of the
+  // 148 persistent CTAs so that the tail is short
+  const int64_t round = pairs ? 64 * COMET_STREAM2_STEPS : 128;
   const int64_t warps = (int64_t)kSmCount * 32;
-  int64_t span = ceil_div(ceil_div(a.N, warps * 10), 128) * 128;
-  if (span < 512) span = 512;
-  if (span > 2048) span = 2048;
+  int64_t span = ceil_div(ceil_div(a.N, warps * 10), round) * round;
+  if (span < 4 * round) span = 4 * round;
+  if (span > 2048 / round * round) span = 2048 / round * round;
   if (const char *e = getenv("COMET_STREAM_SPAN")) { const int v = atoi(e); if (v >= 128 && v % 128 == 0) span = v; }
   a.num_tiles = ceil_div(a.N, span);
   const size_t val_bytes = align_up((size_t)a.num_tiles * sizeof(double), 256);
@@ -490,9 +672,11 @@ static comet_status_t launch_stream(Context *ctx, SegDotArgs a, int64_t x_len, c
   COMET_CUDA_TRY(ctx, cudaMemsetAsync(next_tile, 0, sizeof(unsigned long long), stream));
   const int64_t ctas = ceil_div(a.num_tiles, 32) < kSmCount ? ceil_div(a.num_tiles, 32) : kSmCount;
   if (xsmem) {
-    auto kernel = seg_dot_stream_kernel<T, true>;
+    auto kernel = pairs ? seg_dot_stream2_kernel<T, true> : seg_dot_stream_kernel<T, true>;
     COMET_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)x_bytes));
     kernel<<<(unsigned)ctas, 1024, x_bytes, stream>>>(a, x_len, (int32_t)span, next_tile);
+  } else if (pairs) {
+    seg_dot_stream2_kernel<T, false><<<(unsigned)ctas, 1024, 0, stream>>>(a, x_len, (int32_t)span, next_tile);
   } else {
     seg_dot_stream_kernel<T, false><<<(unsigned)ctas, 1024, 0, stream>>>(a, x_len, (int32_t)span, next_tile);
   }
@@ -517,8 +701,10 @@ static comet_status_t seg_dot_typed(Context *ctx, int dtype, const int32_t *seg_
   // Large problems: the warp-stream kernel (x in shared memory when it fits).
   {
     const char *force = getenv("COMET_SEG_DOT_KERNEL");   // tests: "stream", "resident" or "tile" on any input
-    const bool want_stream = force ? !strcmp(force, "stream") : (N >= (int64_t)kSmCount * 32 * 512 && N > 0);
-    if (want_stream && N > 0) return launch_stream<T>(ctx, a, x_len, stream);
+    // tests force a kernel on any input: "stream" (32 entries per step), "stream2" (64), "resident" or "tile"
+    const bool want_stream = force ? !strncmp(force, "stream", 6) : (N >= (int64_t)kSmCount * 32 * 512 && N > 0);
+    const bool pairs = force ? !strcmp(force, "stream2") : true;
+    if (want_stream && N > 0) return launch_stream<T>(ctx, a, x_len, pairs, stream);
   }
   // Mid-size problems whose vector fits in shared memory beside the staging: persistent CTAs, x resident.
   {

@@ -35,14 +35,14 @@ def tile_items(request, monkeypatch):
     return request.param
 
 
-@pytest.fixture(params=["default", "resident", "stream", "stream-short-spans"])
+@pytest.fixture(params=["default", "resident", "stream", "stream-short-spans", "stream2", "stream2-short-spans"])
 def seg_dot_path(request, monkeypatch):
     monkeypatch.delenv("COMET_SEG_DOT_KERNEL", raising=False)
     monkeypatch.delenv("COMET_STREAM_SPAN", raising=False)
     if request.param == "resident":
         monkeypatch.setenv("COMET_SEG_DOT_KERNEL", "resident")
     elif request.param.startswith("stream"):
-        monkeypatch.setenv("COMET_SEG_DOT_KERNEL", "stream")
+        monkeypatch.setenv("COMET_SEG_DOT_KERNEL", "stream2" if request.param.startswith("stream2") else "stream")
         if request.param.endswith("short-spans"):
             monkeypatch.setenv("COMET_STREAM_SPAN", "128")
     return request.param
