@@ -70,6 +70,14 @@ extern "C" comet_status_t comet_create(comet_handle_t *handle, const comet_alloc
     delete ctx;
     return COMET_ERR_CUDA;
   }
+  // words 32.. hold counters that kernels leave at zero when they finish (see contract_scalar.cu)
+  if (cudaMemset(ctx->d_status, 0, 64 * sizeof(int32_t)) != cudaSuccess) {
+    cudaGetLastError();
+    cudaFreeHost(ctx->h_pinned);
+    cudaFree(ctx->d_status);
+    delete ctx;
+    return COMET_ERR_CUDA;
+  }
   *handle = reinterpret_cast<comet_handle_t>(ctx);
   return COMET_OK;
 }

@@ -438,7 +438,8 @@ template <> struct Pair2<float> {
 
 template <class T, bool XSMEM>
 __global__ void __launch_bounds__(1024, 1)
-seg_dot_stream2_kernel(const SegDotArgs a, int64_t x_len, int32_t span, unsigned long long *next_tile) {
+seg_dot_stream2_kernel(const SegDotArgs a, int64_t x_len, int32_t span, unsigned long long *next_tile,
+                       unsigned int *ctas_done) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const T *s_x = reinterpret_cast<const T *>(smem_raw);
   const T *const val = static_cast<const T *>(a.val), *const x = static_cast<const T *>(a.x);
@@ -588,6 +589,11 @@ seg_dot_stream2_kernel(const SegDotArgs a, int64_t x_len, int32_t span, unsigned
       a.carry_val[tile] = open;
     }
   }
+
+  // The CTA that finishes last puts the two counters back to zero, the state the next call on this handle
+  // expects (no CTA waits for another: each one counts itself done and leaves). This spares a memset per call.
+  __syncthreads();
+  if (threadIdx.x == 0 && atomicAdd(ctas_done, 1u) == gridDim.x - 1) { *next_tile = 0ull; *ctas_done = 0u; }
 }
 
 template <class T, int THREADS, int IPT>
@@ -668,15 +674,31 @@ static comet_status_t launch_stream(Context *ctx, SegDotArgs a, int64_t x_len, b
   if (!scratch) return COMET_ERR_ALLOC;
   a.carry_val = (double *)scratch;
   a.carry_seg = (int32_t *)(scratch + val_bytes);
+  const int64_t ctas = ceil_div(a.num_tiles, 32) < kSmCount ? ceil_div(a.num_tiles, 32) : kSmCount;
+  if (pairs) {
+    // span counter and finished-CTA counter live in the handle and are zero between calls (the kernel's last
+    // CTA resets them): no memset
+    unsigned long long *next_tile = reinterpret_cast<unsigned long long *>(ctx->d_status + 32);
+    unsigned int *ctas_done = reinterpret_cast<unsigned int *>(ctx->d_status + 34);
+    if (xsmem) {
+      auto kernel = seg_dot_stream2_kernel<T, true>;
+      COMET_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)x_bytes));
+      kernel<<<(unsigned)ctas, 1024, x_bytes, stream>>>(a, x_len, (int32_t)span, next_tile, ctas_done);
+    } else {
+      seg_dot_stream2_kernel<T, false><<<(unsigned)ctas, 1024, 0, stream>>>(a, x_len, (int32_t)span, next_tile, ctas_done);
+    }
+    COMET_LAUNCH_CHECK(ctx);
+    carry_fixup_launch(sizeof(T) == 4 ? COMET_F32 : COMET_F64, a.carry_val, a.carry_seg, a.num_tiles, 1, 1, a.y, 1,
+                       a.out_row, stream);
+    COMET_LAUNCH_CHECK(ctx);
+    return COMET_OK;
+  }
   unsigned long long *next_tile = (unsigned long long *)(scratch + val_bytes + seg_bytes);
   COMET_CUDA_TRY(ctx, cudaMemsetAsync(next_tile, 0, sizeof(unsigned long long), stream));
-  const int64_t ctas = ceil_div(a.num_tiles, 32) < kSmCount ? ceil_div(a.num_tiles, 32) : kSmCount;
   if (xsmem) {
-    auto kernel = pairs ? seg_dot_stream2_kernel<T, true> : seg_dot_stream_kernel<T, true>;
+    auto kernel = seg_dot_stream_kernel<T, true>;
     COMET_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)x_bytes));
     kernel<<<(unsigned)ctas, 1024, x_bytes, stream>>>(a, x_len, (int32_t)span, next_tile);
-  } else if (pairs) {
-    seg_dot_stream2_kernel<T, false><<<(unsigned)ctas, 1024, 0, stream>>>(a, x_len, (int32_t)span, next_tile);
   } else {
     seg_dot_stream_kernel<T, false><<<(unsigned)ctas, 1024, 0, stream>>>(a, x_len, (int32_t)span, next_tile);
   }
