@@ -33,6 +33,8 @@ struct SegDotArgs {
   int64_t num_tiles;
   double *carry_val;
   int32_t *carry_seg;
+  unsigned int *ctas_done;  // tile kernel only, may be NULL: counter (zero between calls) that lets the CTA which
+                            // finishes last add the carries itself, so that a small problem is ONE launch
 };
 
 struct BlockBarrier {
@@ -184,6 +186,28 @@ __global__ void __launch_bounds__(THREADS) seg_dot_kernel(const SegDotArgs a) {
   __syncthreads();
 
   walk_staged_tile<T, THREADS, IPT>(a, s_end, s_prod, s_wkey, s_wval, tid, rows, nnz, i0, i1, tile, BlockBarrier());
+
+  if (a.ctas_done == nullptr) return;
+  // Single-launch mode (few tiles): no CTA waits for another; each counts itself done, and the one that finds
+  // all others already counted adds the carries (their writers fenced before counting) and zeroes the counter.
+  __shared__ bool s_last;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = atomicAdd(a.ctas_done, 1u) == gridDim.x - 1;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  T *const y = static_cast<T *>(a.y);
+  for (int64_t t0 = tid; t0 < a.num_tiles; t0 += THREADS) {
+    const int32_t seg = __ldcg(a.carry_seg + t0);                      // written by other SMs: read past this SM's L1
+    if (seg < 0) continue;
+    if (t0 > 0 && __ldcg(a.carry_seg + t0 - 1) == seg) continue;        // the first tile of a run adds the whole run
+    double sum = 0.0;
+    for (int64_t t = t0; t < a.num_tiles && __ldcg(a.carry_seg + t) == seg; ++t) sum += __ldcg(a.carry_val + t);
+    const int64_t row = a.out_row ? (int64_t)a.out_row[seg] : (int64_t)seg;
+    y[row] = (T)((double)__ldcg(y + row) + sum);
+  }
+  if (tid == 0) *a.ctas_done = 0u;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -606,9 +630,12 @@ static comet_status_t launch_dot(Context *ctx, SegDotArgs a, cudaStream_t stream
   if (!scratch) return COMET_ERR_ALLOC;
   a.carry_val = (double *)scratch;
   a.carry_seg = (int32_t *)(scratch + val_bytes);
+  // up to a few thousand tiles the last CTA adds the carries itself: one launch instead of two
+  const bool fused = a.num_tiles > 1 && a.num_tiles <= 4096;
+  a.ctas_done = fused ? reinterpret_cast<unsigned int *>(ctx->d_status + 35) : nullptr;
   seg_dot_kernel<T, THREADS, IPT><<<(unsigned)a.num_tiles, THREADS, 0, stream>>>(a);
   COMET_LAUNCH_CHECK(ctx);
-  if (a.num_tiles > 1) {
+  if (a.num_tiles > 1 && !fused) {
     carry_fixup_launch(sizeof(T) == 4 ? COMET_F32 : COMET_F64, a.carry_val, a.carry_seg, a.num_tiles, 1, 1, a.y, 1,
                        a.out_row, stream);
     COMET_LAUNCH_CHECK(ctx);
