@@ -102,3 +102,34 @@ def test_contractions_report_scratch_allocation_failure():
         with pytest.raises(comet.CometError) as e:
             comet.ttm_symbolic(X, 2, 16)
         assert e.value.status == -6 and len(h._live) == live_before
+
+
+def test_sizes_beyond_the_index_types_are_refused_before_any_launch():
+    """int32 indices: extents and entry counts of 2^31 - 1 or more, key widths beyond 63 bits and leading
+    dimensions of 2^28 or more are reported as such; nothing is launched (the launch counter does not move)."""
+    import ctypes as C
+    h = comet.default_handle()
+    before = h.kernel_launches()
+    one = torch.zeros(1, dtype=torch.int32, device="cuda")
+    v = torch.ones(1, dtype=torch.float64, device="cuda")
+    for dims, status in [((1 << 31, 4), "COMET_ERR_INDEX_OVERFLOW"), ((4, (1 << 31) - 1), "COMET_ERR_INDEX_OVERFLOW"),
+                         ((1 << 30, 1 << 30, 1 << 30), "COMET_ERR_UNSUPPORTED_FORMAT")]:
+        with pytest.raises(comet.CometError) as e:
+            comet.pack([one] * len(dims), v, dims, tuple(range(len(dims))), (comet.CU,) * len(dims))
+        assert comet.binding.STATUS_NAMES[e.value.status] == status
+    # a descriptor that claims more entries than int32 positions can address
+    A = comet.SpTensor.from_arrays((2, 2), (0, 1), (comet.D, comet.CU),
+                                   [torch.tensor([2], dtype=torch.int32, device="cuda"),
+                                    torch.tensor([0, 1, 1], dtype=torch.int32, device="cuda")],
+                                   [None, torch.zeros(1, dtype=torch.int32, device="cuda")], v)
+    A.c.nnz = (1 << 31) + 5
+    with pytest.raises(comet.CometError) as e:
+        comet.spmv(A, torch.ones(2, dtype=torch.float64, device="cuda"))
+    assert comet.binding.STATUS_NAMES[e.value.status] == "COMET_ERR_INDEX_OVERFLOW"
+    A.c.nnz = 1
+    # leading dimension of a gathered operand beyond what 32-bit byte offsets can form
+    out = torch.empty((2, 1), dtype=torch.float64, device="cuda")
+    st = h.lib.comet_spmm(h._h, C.byref(A.c), C.c_void_p(v.data_ptr()), C.c_int64(1), C.c_int64(1 << 28),
+                          C.c_void_p(out.data_ptr()), C.c_int64(1), None)
+    assert comet.binding.STATUS_NAMES[st] == "COMET_ERR_INDEX_OVERFLOW"
+    assert h.kernel_launches() == before

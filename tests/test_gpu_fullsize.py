@@ -242,3 +242,28 @@ def test_hypersparse_matrix_csr_dcsr_coo():
         del C, A
         torch.cuda.empty_cache()
     assert index_bytes["dcsr"] < index_bytes["csr"] / 5
+
+
+def test_large_matrix_268m_entries():
+    """Sizes well beyond the benchmark's: 268,435,456 entries in a 1,048,576^2 matrix (positions and merge-list
+    indices in the 2^28..2^29 range). Packing is checked against the sorted input, SpMV on sampled rows."""
+    dims, nnz = (1 << 20, 1 << 20), 1 << 28
+    coords, val = synth.random_coo(dims, nnz, 91, device="cuda")
+
+    class _Case:
+        pass
+    case = _Case()
+    case.nnz, case.dims, case.coords, case.val = nnz, dims, coords, val
+    A = comet.pack(coords, val, dims, (0, 1), (D, CU))
+    check_packed_against_sorted_input(case, A, (0, 1), (D, CU))
+    x = synth.random_dense((dims[1],), 91, device="cuda")
+    y = torch.full((dims[0],), float("nan"), dtype=torch.float64, device="cuda")
+    comet.spmv(A, x, y)
+    assert not bool(torch.isnan(y).any())
+    rows = sample_rows(dims[0], 13, always=[0, dims[0] - 1])
+    c, v = [t.cpu().numpy() for t in coords], val.cpu().numpy()
+    del A, coords, val
+    torch.cuda.empty_cache()
+    want, norm = oracle.spmv(c, v, dims, x.cpu().numpy(), rows=rows)
+    rel = assert_close(y[torch.from_numpy(rows).cuda()], want, norm, what="268M-entry spmv")
+    print(f"268M entries: worst normalised error {rel:.2e}")
