@@ -289,11 +289,14 @@ def _from_ptr(ptr, n, dtype, owner):
 # ------------------------------------------------------------------------------------------- entry points
 
 PACK_SUM_DUPLICATES = 1
+PACK_CSR_HISTOGRAM = 2
 
 
-def pack(coords, val, dims, mode_order, attr, handle: Handle | None = None, sum_duplicates: bool = False) -> SpTensor:
+def pack(coords, val, dims, mode_order, attr, handle: Handle | None = None, sum_duplicates: bool = False,
+         csr_histogram: bool = False) -> SpTensor:
     """comet_pack / comet_pack_ex: COO (one int32 CUDA tensor per mode, any order) -> packed levels. Cells must be
-    distinct unless `sum_duplicates`, which merges equal cells (values added in input order)."""
+    distinct unless `sum_duplicates`, which merges equal cells (values added in input order). `csr_histogram`:
+    for [D,CU] matrices with rows of similar length, build the rows as a histogram instead of a full sort."""
     handle = handle or default_handle()
     order = len(dims)
     _require_cuda(val, *coords)
@@ -307,7 +310,8 @@ def pack(coords, val, dims, mode_order, attr, handle: Handle | None = None, sum_
     out = SpTensorStruct()
     st = handle.lib.comet_pack_ex(handle._h, C.c_int32(order), h_dims, C.c_int64(val.numel()), h_crd, _ptr(val),
                                   C.c_int(_dtype_code(val)), h_mo, h_at,
-                                  C.c_uint32(PACK_SUM_DUPLICATES if sum_duplicates else 0), _stream_ptr(),
+                                  C.c_uint32((PACK_SUM_DUPLICATES if sum_duplicates else 0) | (PACK_CSR_HISTOGRAM if csr_histogram else 0)),
+                                  _stream_ptr(),
                                   C.byref(out))
     handle.check(st, "comet_pack")
     return SpTensor(handle, out)

@@ -752,7 +752,8 @@ static comet_status_t seg_dot_typed(Context *ctx, int dtype, const int32_t *seg_
     const char *force = getenv("COMET_SEG_DOT_KERNEL");   // tests: "stream", "resident" or "tile" on any input
     // tests force a kernel on any input: "stream" (32 entries per step), "stream2" (64), "resident" or "tile"
     const bool want_stream = force ? !strncmp(force, "stream", 6) : (N >= (int64_t)kSmCount * 32 * 512 && N > 0);
-    const bool pairs = force ? !strcmp(force, "stream2") : true;
+    // many more segments than entries (hypersparse CSR): segment ends dominate, and the 32-entry kernel closes them cheaper
+    const bool pairs = force ? !strcmp(force, "stream2") : M <= N;
     if (want_stream && N > 0) return launch_stream<T>(ctx, a, x_len, pairs, stream);
   }
   // Mid-size problems whose vector fits in shared memory beside the staging: persistent CTAs, x resident.

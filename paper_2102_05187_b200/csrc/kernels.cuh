@@ -59,6 +59,12 @@ int64_t radix_sort_table_words(int64_t n);
 comet_status_t radix_sort_pairs(Context *ctx, uint64_t *&ka, uint64_t *&kb, uint32_t *&pa, uint32_t *&pb, int64_t n,
                                 int bits, uint32_t *table, uint32_t *scan_tmp, cudaStream_t s);
 
+// COO -> CSR without the full sort (pack_csr.cu): fills pos_out (rows + 1), crd_out (n), val_out (n); synchronises
+// the stream once. *fallback = 1 with COMET_OK when a row is too long for it: run the generic path instead.
+comet_status_t pack_csr_fast(Context *ctx, int dtype, const int32_t *row, const int32_t *col, const void *val, int64_t n,
+                             int64_t rows, int64_t cols, int32_t *pos_out, int32_t *crd_out, void *val_out,
+                             int *fallback, cudaStream_t s);
+
 int32_t choose_tile_items(int64_t total_items, int workers_per_block);
 
 // Block list of a library-owned tensor (what comet_sptensor_free releases).

@@ -17,6 +17,7 @@
 #include "common.cuh"
 #include "kernels.cuh"
 
+#include <stdlib.h>
 #include <string.h>
 
 namespace comet {
@@ -557,7 +558,7 @@ extern "C" comet_status_t comet_pack_ex(comet_handle_t handle, int32_t order, co
                                         const int32_t *const *h_coo_crd, const void *coo_val, comet_dtype_t dtype,
                                         const int32_t *h_mode_order, const int32_t *h_attr, uint32_t flags,
                                         void *stream, comet_sptensor_t *out) {
-  if (flags & ~(uint32_t)COMET_PACK_SUM_DUPLICATES) return COMET_ERR_INVALID_ARG;
+  if (flags & ~(uint32_t)(COMET_PACK_SUM_DUPLICATES | COMET_PACK_CSR_HISTOGRAM)) return COMET_ERR_INVALID_ARG;
   if (!handle || !out || !h_dims || !h_coo_crd || !h_mode_order || !h_attr) return COMET_ERR_INVALID_ARG;
   memset(out, 0, sizeof(*out));
   if (order < 1 || order > COMET_MAX_ORDER || nnz < 0) return COMET_ERR_INVALID_ARG;
@@ -578,6 +579,48 @@ extern "C" comet_status_t comet_pack_ex(comet_handle_t handle, int32_t order, co
 
   Context *ctx = reinterpret_cast<Context *>(handle);
   cudaStream_t s = (cudaStream_t)stream;
+
+  // CSR of a matrix with a dense row level: the row structure is a histogram, so the full sort is not needed
+  // (pack_csr.cu). On request only (COMET_PACK_CSR_HISTOGRAM): it wins on matrices whose rows are of similar
+  // length and loses on skewed ones, where the atomic counters of the heavy rows serialise. The environment
+  // variable COMET_PACK_CSR=1 / 0 overrides the flag (tests).
+  {
+    const char *force = getenv("COMET_PACK_CSR");
+    const int64_t rows = h_dims[h_mode_order[0]], cols = h_dims[h_mode_order[1 % order]];
+    const bool shape = order == 2 && h_attr[0] == COMET_D && h_attr[1] == COMET_CU &&
+                       !(flags & COMET_PACK_SUM_DUPLICATES) && rows <= (1ll << 27) &&
+                       rows <= 4 * nnz + 1024;            // a warp visits every row: not for hypersparse matrices
+    const bool want = force ? force[0] == '1' : (flags & COMET_PACK_CSR_HISTOGRAM) != 0;
+    if (shape && want) {
+      void *owner = owner_new();
+      if (!owner) return COMET_ERR_ALLOC;
+      const size_t val_size = dtype == COMET_F32 ? 4 : 8;
+      out->order = 2; out->dtype = dtype; out->nnz = nnz;
+      for (int l = 0; l < 2; ++l) { out->dims[l] = h_dims[l]; out->mode_order[l] = h_mode_order[l]; out->attr[l] = h_attr[l]; }
+      out->pos_len[0] = 1; out->crd_len[0] = 0; out->pos_len[1] = rows + 1; out->crd_len[1] = nnz;
+      out->pos[0] = (int32_t *)owner_alloc(ctx, owner, 4, s);
+      out->pos[1] = (int32_t *)owner_alloc(ctx, owner, (size_t)(rows + 1) * 4, s);
+      if (nnz > 0) {
+        out->crd[1] = (int32_t *)owner_alloc(ctx, owner, (size_t)nnz * 4, s);
+        out->val = owner_alloc(ctx, owner, (size_t)nnz * val_size, s);
+      }
+      comet_status_t st = COMET_OK;
+      if (!out->pos[0] || !out->pos[1] || (nnz > 0 && (!out->crd[1] || !out->val))) st = COMET_ERR_ALLOC;
+      int fallback = 0;
+      if (st == COMET_OK) {
+        const int32_t dim0 = (int32_t)rows;
+        cudaError_t e = cudaMemcpyAsync(out->pos[0], &dim0, 4, cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) st = cuda_fail(ctx, e);
+      }
+      if (st == COMET_OK)
+        st = pack_csr_fast(ctx, dtype, h_coo_crd[h_mode_order[0]], h_coo_crd[h_mode_order[1]], coo_val, nnz, rows, cols,
+                           out->pos[1], out->crd[1], out->val, &fallback, s);
+      if (st == COMET_OK && !fallback) { out->owner = owner; return COMET_OK; }
+      owner_release(ctx, owner, s);
+      memset(out, 0, sizeof(*out));
+      if (st != COMET_OK) return st;
+    }
+  }
 
   KeyLayout key{};
   LevelPlan plan{};

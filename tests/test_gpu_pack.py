@@ -31,9 +31,24 @@ def check_pack(coords, val, dims, mode_order, attr):
     for l in range(len(dims)):
         assert_equal_arrays(got.pos(l), want.pos[l], f"pos[{l}] {attr} {mode_order}")
         assert_equal_arrays(got.crd(l), want.crd[l], f"crd[{l}] {attr} {mode_order}")
-    assert_equal_arrays(got.val, want.val, "val")
+    if val.dtype == torch.float32:
+        assert got.val.dtype == torch.float32
+        assert np.array_equal(got.val.cpu().numpy().view(np.int32), want.val.astype(np.float32).view(np.int32)), "val"
+    else:
+        assert_equal_arrays(got.val, want.val, "val")
     comet.validate(got)
     return got
+
+
+@pytest.fixture(params=["default", "csr-histogram", "generic"])
+def csr_path(request, monkeypatch):
+    """[D,CU] matrices: the size-based choice, then the histogram path and the generic radix path forced."""
+    monkeypatch.delenv("COMET_PACK_CSR", raising=False)
+    if request.param == "csr-histogram":
+        monkeypatch.setenv("COMET_PACK_CSR", "1")
+    elif request.param == "generic":
+        monkeypatch.setenv("COMET_PACK_CSR", "0")
+    return request.param
 
 
 FORMATS_2D = [(CN, S), (D, CU), (CU, CU)]
@@ -45,9 +60,54 @@ FORMATS_3D = [(CN, S, S), (CU, CU, CU), (D, CU, CU)]
 @pytest.mark.parametrize("dims,nnz,seed", [((7, 5), 12, 1), ((1, 9), 4, 2), ((9, 1), 4, 3), ((6, 6), 36, 4),
                                            ((8, 8), 1, 5), ((8, 8), 0, 6), ((300, 200), 5000, 7),
                                            ((5000, 3), 9000, 8), ((3, 70000), 20000, 9), ((1, 1), 1, 10)])
-def test_pack_matrices(attr, mode_order, dims, nnz, seed):
+def test_pack_matrices(attr, mode_order, dims, nnz, seed, csr_path):
+    if attr != (D, CU) and csr_path != "default":
+        pytest.skip("the path choice only exists for [D,CU]")
     coords, val = synth.random_coo(dims, nnz, seed)
     check_pack(coords, val, dims, mode_order, attr)
+
+
+@pytest.mark.parametrize("mode_order", [(0, 1), (1, 0)])
+@pytest.mark.parametrize("dims,nnz,seed", [((40, 3000), 30000, 1),      # rows of ~750: the shared-memory network
+                                           ((6, 9000), 30000, 2),       # rows of ~5000: the shared-memory radix sort
+                                           ((3, 12288), 36864, 3),      # full rows of exactly the longest length handled
+                                           ((2, 40000), 50000, 4),      # rows of 25000: handed to the generic path
+                                           ((2000, 2100), 60000, 5),    # every class of short row
+                                           ((70, 33), 2310, 6)])        # rows of exactly 33: the first mid length
+def test_pack_csr_row_length_classes(mode_order, dims, nnz, seed, csr_path):
+    d = dims if mode_order == (0, 1) else (dims[1], dims[0])
+    coords, val = synth.random_coo(dims, nnz, seed)
+    if mode_order == (1, 0):
+        coords = [coords[1], coords[0]]
+    check_pack(coords, val, d, mode_order, (D, CU))
+    check_pack(coords, val.float(), d, mode_order, (D, CU))
+
+
+def test_pack_csr_histogram_path_reports_errors(monkeypatch):
+    monkeypatch.setenv("COMET_PACK_CSR", "1")
+    r = torch.tensor([0, 1, 1, 5], dtype=torch.int32, device="cuda")
+    c = torch.tensor([0, 1, 1, 2], dtype=torch.int32, device="cuda")
+    v = torch.ones(4, dtype=torch.float64, device="cuda")
+    with pytest.raises(comet.CometError) as e:
+        comet.pack([r[:3], c[:3]], v[:3], (4, 4), (0, 1), (D, CU))
+    assert comet.binding.STATUS_NAMES[e.value.status] == "COMET_ERR_DUPLICATE_COORD"
+    with pytest.raises(comet.CometError) as e:
+        comet.pack([r, c], v, (4, 4), (0, 1), (D, CU))
+    assert comet.binding.STATUS_NAMES[e.value.status] == "COMET_ERR_COORD_OUT_OF_RANGE"
+    # duplicates inside a long row (the shared-memory sorts check neighbours too)
+    g = np.random.default_rng(1)
+    cols = torch.from_numpy(g.permutation(9000)[:5000].astype(np.int32)).cuda()
+    cols[4999] = cols[17]
+    rows = torch.zeros(5000, dtype=torch.int32, device="cuda")
+    with pytest.raises(comet.CometError) as e:
+        comet.pack([rows, cols], torch.ones(5000, dtype=torch.float64, device="cuda"), (1, 9000), (0, 1), (D, CU))
+    assert comet.binding.STATUS_NAMES[e.value.status] == "COMET_ERR_DUPLICATE_COORD"
+    cols2 = torch.from_numpy(g.permutation(3000)[:700].astype(np.int32)).cuda()
+    cols2[699] = cols2[5]
+    with pytest.raises(comet.CometError) as e:
+        comet.pack([torch.zeros(700, dtype=torch.int32, device="cuda"), cols2], torch.ones(700, dtype=torch.float64, device="cuda"),
+                   (1, 3000), (0, 1), (D, CU))
+    assert comet.binding.STATUS_NAMES[e.value.status] == "COMET_ERR_DUPLICATE_COORD"
 
 
 @pytest.mark.parametrize("attr", FORMATS_3D)
@@ -196,6 +256,16 @@ def test_pack_sum_duplicates_is_a_no_op_on_distinct_cells_and_handles_empty_and_
     assert np.array_equal(got.val.cpu().numpy(), want.val.astype(np.float32))   # summed in double, rounded once
 
 
+def test_pack_csr_histogram_flag_gives_the_same_tensor():
+    dims = (300, 200)
+    coords, val = synth.random_coo(dims, 5000, 7)
+    a = comet.pack([c.cuda() for c in coords], val.cuda(), dims, (0, 1), (D, CU))
+    b = comet.pack([c.cuda() for c in coords], val.cuda(), dims, (0, 1), (D, CU), csr_histogram=True)
+    assert torch.equal(a.val, b.val) and torch.equal(a.pos(1), b.pos(1)) and torch.equal(a.crd(1), b.crd(1))
+    c3 = comet.pack([c.cuda() for c in coords], val.cuda(), dims, (0, 1), (CU, CU), csr_histogram=True)   # ignored here
+    assert c3.attr == (CU, CU)
+
+
 def test_pack_ex_rejects_unknown_flags():
     import ctypes as C
     h = comet.default_handle()
@@ -204,6 +274,6 @@ def test_pack_ex_rejects_unknown_flags():
     crd = (C.c_void_p * 2)(0, 0)
     mo = (C.c_int32 * 2)(0, 1)
     at = (C.c_int32 * 2)(D, CU)
-    st = h.lib.comet_pack_ex(h._h, C.c_int32(2), dims, C.c_int64(0), crd, None, C.c_int(0), mo, at, C.c_uint32(6), None,
+    st = h.lib.comet_pack_ex(h._h, C.c_int32(2), dims, C.c_int64(0), crd, None, C.c_int(0), mo, at, C.c_uint32(12), None,
                              C.byref(out))
     assert st == -1
