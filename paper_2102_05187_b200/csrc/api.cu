@@ -174,17 +174,19 @@ extern "C" comet_status_t comet_spmm(comet_handle_t handle, const comet_sptensor
   cudaStream_t s = (cudaStream_t)stream;
   const int64_t rows = A->dims[A->mode_order[0]];
   if (is_fmt(A, 2, COMET_D, COMET_CU))
-    return seg_gather(ctx, A->dtype, A->pos[1] + 1, A->crd[1], A->val, rows, A->nnz, B, ldb, R, C, ldc, nullptr, rows, s);
+    return seg_gather(ctx, A->dtype, A->pos[1] + 1, A->crd[1], A->val, rows, A->nnz, B, ldb, R, C, ldc, nullptr, rows,
+                      A->dims[A->mode_order[1]], s);
   if (is_fmt(A, 2, COMET_CU, COMET_CU)) {
     if (A->crd_len[0] == 0) return zero_rows(ctx, C, A->dtype, rows, R, ldc, s);
     return seg_gather(ctx, A->dtype, A->pos[1] + 1, A->crd[1], A->val, A->crd_len[0], A->nnz, B, ldb, R, C, ldc, A->crd[0],
-                      rows, s);
+                      rows, 0, s);
   }
   if (is_fmt(A, 2, COMET_CN, COMET_S)) {
     int32_t *pos = nullptr;
     st = coo_rows(ctx, A, rows, s, &pos);
     if (st != COMET_OK) return st;
-    st = seg_gather(ctx, A->dtype, pos + 1, A->crd[1], A->val, rows, A->nnz, B, ldb, R, C, ldc, nullptr, rows, s);
+    st = seg_gather(ctx, A->dtype, pos + 1, A->crd[1], A->val, rows, A->nnz, B, ldb, R, C, ldc, nullptr, rows,
+                    A->dims[A->mode_order[1]], s);
     ctx_free(ctx, pos, s);
     return st;
   }
@@ -516,7 +518,7 @@ extern "C" comet_status_t comet_ttm(comet_handle_t handle, const comet_sptensor_
   if (Y->dtype != X->dtype) return COMET_ERR_INVALID_ARG;
   if (misaligned(U, X->dtype)) return COMET_ERR_MISALIGNED;
   Context *ctx = reinterpret_cast<Context *>(handle);
-  return seg_gather(ctx, X->dtype, fiber_pos + 1, X->crd[last], X->val, F, X->nnz, U, ldu, R, Y->val, R, nullptr, F,
+  return seg_gather(ctx, X->dtype, fiber_pos + 1, X->crd[last], X->val, F, X->nnz, U, ldu, R, Y->val, R, nullptr, F, 0,
                     (cudaStream_t)stream);
 }
 

@@ -12,6 +12,7 @@
 #include "common.cuh"
 #include "kernels.cuh"
 #include "walk.cuh"
+#include "spmm_heavy.cuh"
 
 #ifndef COMET_PF_GATHER
 #define COMET_PF_GATHER 4      // row gathers in flight per worker (SpMM, TTM); measured best with 4 CTAs/SM
@@ -39,10 +40,12 @@ struct SegGatherArgs {
   double *carry_val;        // num_tiles x carry_ld
   int32_t *carry_seg;       // num_tiles: segment the carry belongs to, -1 if none
   int32_t carry_ld;
+  int32_t skip_len;         // > 0: segments of at least this many entries are somebody else's (the long-row
+                            //      path of SpMM): neither walked nor stored here. Never below tile_items.
 };
 
 // What the walker does with one leaf entry: close the segments that end in front of it, accumulate.
-template <class T, int LPN, int CPL, int VEC, bool MAPPED>
+template <class T, int LPN, int CPL, int VEC, bool MAPPED, bool PASS_THROUGH = false>
 struct SegGatherPolicy {
   using L = Lanes<T, LPN, CPL, VEC>;
   static constexpr int kPF = COMET_PF_GATHER;
@@ -63,10 +66,12 @@ struct SegGatherPolicy {
   int32_t next_end;         // leaf position where the open segment ends (-1: no segment left)
   int32_t base, rel_end;    // chunk base and next_end relative to it
   int32_t last_flush;       // leaf position of the latest flush (entries at or after it are still in acc)
+  uint64_t pass;            // PASS_THROUGH: L2 evict-first policy of the gathers (the other role's block of B stays)
 
   __device__ __forceinline__ SegGatherPolicy(const SegGatherArgs &args, const L &lanes, int64_t i0, int32_t j0)
       : a(args), ln(lanes), base(j0), last_flush(j0) {
     ln.zero(acc);
+    if (PASS_THROUGH) pass = l2_policy_evict_first();
     val = static_cast<const T *>(a.val);
     bcol = reinterpret_cast<const char *>(static_cast<const T *>(a.B) + ln.col0);
     ldb_bytes = (int32_t)(a.ldb * sizeof(T));
@@ -83,7 +88,8 @@ struct SegGatherPolicy {
     e.a = ld_stream(a.crd + j);
   }
   __device__ __forceinline__ void prefetch(int32_t c, int32_t, Slot &s) const {
-    ln.gather(reinterpret_cast<const T *>(bcol + (int64_t)c * ldb_bytes), s.r);
+    if (PASS_THROUGH) ln.gather_hint(reinterpret_cast<const T *>(bcol + (int64_t)c * ldb_bytes), s.r, pass);
+    else ln.gather(reinterpret_cast<const T *>(bcol + (int64_t)c * ldb_bytes), s.r);
   }
   __device__ __forceinline__ void begin_chunk(int32_t b) { base = b; rel_end = next_end - b; }
 
@@ -113,13 +119,21 @@ struct SegGatherPolicy {
   }
 };
 
-template <class T, int LPN, int CPL, int VEC, bool MAPPED>
+// HEAVY: the first h.heavy_ctas CTAs of the grid work on the long rows of an SpMM (spmm_heavy.cuh) while the
+// others walk the general tiles and skip those rows. The two roles are bound by different things (the long rows
+// by the L2 -> L1 fill rate, the rest by DRAM latency), so sharing the SMs between them is faster than running
+// one after the other.
+template <class T, int LPN, int CPL, int VEC, bool MAPPED, bool HEAVY>
 __global__ void __launch_bounds__(kBlockThreads, (CPL * VEC * sizeof(T) <= 16 ? COMET_MINB_GATHER : 2))
-seg_gather_kernel(const SegGatherArgs a) {
+seg_gather_kernel(const SegGatherArgs a, const HeavyArgs h) {
   using L = Lanes<T, LPN, CPL, VEC>;
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  if (HEAVY && (int)blockIdx.x < h.heavy_ctas) {
+    heavy_role<T, LPN, CPL, VEC>(h, smem_raw);
+    return;
+  }
   const int worker = threadIdx.x / LPN;
-  const int64_t tile = (int64_t)blockIdx.x * L::kWorkers + worker;
+  const int64_t tile = (int64_t)(blockIdx.x - (HEAVY ? h.heavy_ctas : 0)) * L::kWorkers + worker;
   if (tile >= a.num_tiles) return;                       // whole groups leave together
   const uint32_t smem = smem_u32(smem_raw) + worker * RingLayout<L, false>::kWorkerBytes;
   const L ln(a.R);
@@ -127,11 +141,31 @@ seg_gather_kernel(const SegGatherArgs a) {
   const int64_t total = a.M + a.N;
   const int64_t d0 = tile * a.tile_items;
   const int64_t d1 = (d0 + a.tile_items < total) ? d0 + a.tile_items : total;
-  const int64_t i0 = merge_path_segments_coop<LPN>(a.seg_end, a.M, a.N, d0, ln.g, ln.mask);
+  int64_t i0 = merge_path_segments_coop<LPN>(a.seg_end, a.M, a.N, d0, ln.g, ln.mask);
   const int64_t i1 = merge_path_segments_coop<LPN>(a.seg_end, a.M, a.N, d1, ln.g, ln.mask);
-  const int32_t j0 = (int32_t)(d0 - i0), j1 = (int32_t)(d1 - i1);
+  int32_t j0 = (int32_t)(d0 - i0), j1 = (int32_t)(d1 - i1);
+  if (a.skip_len > 0) {
+    // A long segment holds more entries than a tile, so it can only be the one open at the tile's start or the
+    // one open at its end. Its entries are left out; its end marker (if it is in this tile) stores nothing.
+    if (i0 < a.M) {
+      const int32_t end0 = __ldg(a.seg_end + i0);
+      const int32_t start0 = i0 > 0 ? __ldg(a.seg_end + i0 - 1) : 0;
+      if (end0 - start0 >= a.skip_len) {
+        if (i0 >= i1) {                                      // the whole tile lies inside the long segment
+          if (ln.g == 0) a.carry_seg[tile] = -1;
+          return;
+        }
+        i0 += 1;
+        j0 = end0;
+      }
+    }
+    if (i1 < a.M) {
+      const int32_t start1 = i1 > 0 ? __ldg(a.seg_end + i1 - 1) : 0;
+      if (__ldg(a.seg_end + i1) - start1 >= a.skip_len && start1 < j1) j1 = start1 > j0 ? start1 : j0;
+    }
+  }
 
-  SegGatherPolicy<T, LPN, CPL, VEC, MAPPED> p(a, ln, i0, j0);
+  SegGatherPolicy<T, LPN, CPL, VEC, MAPPED, HEAVY> p(a, ln, i0, j0);
   walk_tile(ln, p, j0, j1, smem);
   while (p.segment() < i1) p.flush(j1);                  // end markers that close the tile
 
@@ -199,34 +233,65 @@ int32_t choose_tile_items(int64_t total_items, int workers_per_block) {
   return (int32_t)t;
 }
 
-template <class T, int LPN, int CPL, int VEC, bool MAPPED>
-static comet_status_t launch_mapped(Context *ctx, const SegGatherArgs &a, int64_t blocks, cudaStream_t stream) {
+template <class T, int LPN, int CPL, int VEC, bool MAPPED, bool HEAVY>
+static comet_status_t launch_mapped(Context *ctx, const SegGatherArgs &a, const HeavyArgs &h, int64_t blocks,
+                                    cudaStream_t stream) {
   using L = Lanes<T, LPN, CPL, VEC>;
   constexpr size_t smem = RingLayout<L, false>::kBlockBytes;
-  auto kernel = seg_gather_kernel<T, LPN, CPL, VEC, MAPPED>;
+  auto kernel = seg_gather_kernel<T, LPN, CPL, VEC, MAPPED, HEAVY>;
   if (smem > 48 * 1024)
     COMET_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  kernel<<<(unsigned)blocks, kBlockThreads, smem, stream>>>(a);
+  kernel<<<(unsigned)(blocks + (HEAVY ? h.heavy_ctas : 0)), kBlockThreads, smem, stream>>>(a, h);
   COMET_LAUNCH_CHECK(ctx);
   return COMET_OK;
 }
 
+// The shapes whose rows are 256, 512 or 1024 bytes carry the long-row role of SpMM.
+template <class T, int LPN, int CPL, int VEC> constexpr bool kHeavyShape =
+    VEC * sizeof(T) == 16 && (LPN * CPL * VEC * sizeof(T) == 256 || LPN * CPL * VEC * sizeof(T) == 512 ||
+                              LPN * CPL * VEC * sizeof(T) == 1024) && LPN >= 16;
+
+static size_t carry_bytes(int64_t num_tiles, int32_t carry_ld) {
+  return align_up((size_t)num_tiles * carry_ld * sizeof(double), 256) + align_up((size_t)num_tiles * sizeof(int32_t), 256);
+}
+
+// `heavy` (optional): the long-row plan of an SpMM; its scratch precedes the carries of this launch.
 template <class T, int LPN, int CPL, int VEC>
-static comet_status_t launch_one(Context *ctx, SegGatherArgs a, cudaStream_t stream) {
+static comet_status_t launch_one(Context *ctx, SegGatherArgs a, HeavyArgs *heavy, cudaStream_t stream) {
   constexpr int WORKERS = kBlockThreads / LPN;
   const int64_t total = a.M + a.N;
   a.tile_items = choose_tile_items(total, WORKERS);
   a.num_tiles = ceil_div(total, a.tile_items);
   a.carry_ld = (int32_t)align_up((size_t)a.R, 2);
   const size_t val_bytes = align_up((size_t)a.num_tiles * a.carry_ld * sizeof(double), 256);
-  const size_t seg_bytes = align_up((size_t)a.num_tiles * sizeof(int32_t), 256);
-  char *scratch = (char *)scratch_get(ctx, val_bytes + seg_bytes, stream);
+  size_t heavy_bytes = 0;
+  HeavyArgs h{};
+  if (kHeavyShape<T, LPN, CPL, VEC> && heavy && !a.out_row)
+    heavy_bytes = spmm_heavy_plan(sizeof(T) == 4 ? COMET_F32 : COMET_F64, a.M, a.N, heavy->cols, a.B, a.ldb, a.R, a.C, a.ldc,
+                                  a.tile_items, &h);
+  char *scratch = (char *)scratch_get(ctx, heavy_bytes + carry_bytes(a.num_tiles, a.carry_ld), stream);
   if (!scratch) return COMET_ERR_ALLOC;
-  a.carry_val = (double *)scratch;
-  a.carry_seg = (int32_t *)(scratch + val_bytes);
+  a.carry_val = (double *)(scratch + heavy_bytes);
+  a.carry_seg = (int32_t *)(scratch + heavy_bytes + val_bytes);
   const int64_t blocks = ceil_div(a.num_tiles, WORKERS);
-  comet_status_t st = a.out_row ? launch_mapped<T, LPN, CPL, VEC, true>(ctx, a, blocks, stream)
-                                : launch_mapped<T, LPN, CPL, VEC, false>(ctx, a, blocks, stream);
+  comet_status_t st;
+  if constexpr (kHeavyShape<T, LPN, CPL, VEC>) {
+    if (heavy_bytes) {
+      st = spmm_heavy_prepare(ctx, &h, a.seg_end - 1, a.crd, a.val, scratch, stream);
+      if (st != COMET_OK) return st;
+      a.skip_len = h.threshold;
+      st = launch_mapped<T, LPN, CPL, VEC, false, true>(ctx, a, h, blocks, stream);
+      if (st != COMET_OK) return st;
+      st = spmm_heavy_finish(ctx, h, sizeof(T) == 4 ? COMET_F32 : COMET_F64, stream);
+      if (st != COMET_OK) return st;
+      carry_fixup_launch(sizeof(T) == 4 ? COMET_F32 : COMET_F64, a.carry_val, a.carry_seg, a.num_tiles, a.R, a.carry_ld, a.C,
+                         a.ldc, a.out_row, stream);
+      COMET_LAUNCH_CHECK(ctx);
+      return COMET_OK;
+    }
+  }
+  st = a.out_row ? launch_mapped<T, LPN, CPL, VEC, true, false>(ctx, a, h, blocks, stream)
+                 : launch_mapped<T, LPN, CPL, VEC, false, false>(ctx, a, h, blocks, stream);
   if (st != COMET_OK) return st;
   carry_fixup_launch(sizeof(T) == 4 ? COMET_F32 : COMET_F64, a.carry_val, a.carry_seg, a.num_tiles, a.R, a.carry_ld, a.C,
                      a.ldc, a.out_row, stream);
@@ -241,7 +306,10 @@ static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 template <class T>
 static comet_status_t seg_gather_typed(Context *ctx, const int32_t *seg_end, const int32_t *crd, const T *val,
                                        int64_t M, int64_t N, const T *B, int64_t ldb, int64_t R, T *C, int64_t ldc,
-                                       const int32_t *out_row, int64_t out_rows, cudaStream_t stream) {
+                                       const int32_t *out_row, int64_t out_rows, int64_t b_rows, cudaStream_t stream) {
+  HeavyArgs hint{};                                        // SpMM on [D,CU] with a known B: long rows by column phases
+  hint.cols = b_rows;
+  HeavyArgs *heavy = (!out_row && b_rows > 0 && R <= 128) ? &hint : nullptr;
   constexpr int PER = 16 / sizeof(T);                      // elements per 128-bit piece
   const bool vec_ok = aligned16(B) && aligned16(C) && (ldb % PER == 0) && (ldc % PER == 0);
   int64_t done = 0;
@@ -256,16 +324,16 @@ static comet_status_t seg_gather_typed(Context *ctx, const int32_t *seg_end, con
     a.R = (int32_t)chunk;
     const bool v = vec_ok && done % PER == 0;
     const int64_t pieces = chunk / PER;                    // 128-bit pieces per row when chunk is a multiple
-    if (v && chunk % PER == 0 && pieces == 64) st = launch_one<T, 32, 2, PER>(ctx, a, stream);
-    else if (v && chunk % PER == 0 && pieces == 32) st = launch_one<T, 32, 1, PER>(ctx, a, stream);
-    else if (v && chunk % PER == 0 && pieces == 16) st = launch_one<T, 16, 1, PER>(ctx, a, stream);
-    else if (v && chunk % PER == 0 && pieces == 8) st = launch_one<T, 8, 1, PER>(ctx, a, stream);
-    else if (v && chunk % PER == 0 && pieces == 4) st = launch_one<T, 4, 1, PER>(ctx, a, stream);
-    else if (v && chunk % PER == 0 && pieces == 2) st = launch_one<T, 2, 1, PER>(ctx, a, stream);
-    else if (v && chunk % PER == 0 && pieces == 1) st = launch_one<T, 1, 1, PER>(ctx, a, stream);
-    else if (chunk > 64) st = launch_one<T, 32, 4, 1>(ctx, a, stream);
-    else if (chunk > 32) st = launch_one<T, 32, 2, 1>(ctx, a, stream);
-    else st = launch_one<T, 32, 1, 1>(ctx, a, stream);
+    if (v && chunk % PER == 0 && pieces == 64) st = launch_one<T, 32, 2, PER>(ctx, a, heavy, stream);
+    else if (v && chunk % PER == 0 && pieces == 32) st = launch_one<T, 32, 1, PER>(ctx, a, heavy, stream);
+    else if (v && chunk % PER == 0 && pieces == 16) st = launch_one<T, 16, 1, PER>(ctx, a, heavy, stream);
+    else if (v && chunk % PER == 0 && pieces == 8) st = launch_one<T, 8, 1, PER>(ctx, a, heavy, stream);
+    else if (v && chunk % PER == 0 && pieces == 4) st = launch_one<T, 4, 1, PER>(ctx, a, heavy, stream);
+    else if (v && chunk % PER == 0 && pieces == 2) st = launch_one<T, 2, 1, PER>(ctx, a, heavy, stream);
+    else if (v && chunk % PER == 0 && pieces == 1) st = launch_one<T, 1, 1, PER>(ctx, a, heavy, stream);
+    else if (chunk > 64) st = launch_one<T, 32, 4, 1>(ctx, a, heavy, stream);
+    else if (chunk > 32) st = launch_one<T, 32, 2, 1>(ctx, a, heavy, stream);
+    else st = launch_one<T, 32, 1, 1>(ctx, a, heavy, stream);
     if (st != COMET_OK) return st;
     done += a.R;
   }
@@ -274,14 +342,14 @@ static comet_status_t seg_gather_typed(Context *ctx, const int32_t *seg_end, con
 
 comet_status_t seg_gather(Context *ctx, int dtype, const int32_t *seg_end, const int32_t *crd, const void *val,
                           int64_t M, int64_t N, const void *B, int64_t ldb, int64_t R, void *C, int64_t ldc,
-                          const int32_t *out_row, int64_t out_rows, cudaStream_t stream) {
+                          const int32_t *out_row, int64_t out_rows, int64_t b_rows, cudaStream_t stream) {
   if (ldb >= (1ll << 28)) return COMET_ERR_INDEX_OVERFLOW;      // row offsets are formed as int32 bytes * int32 index
   if (M == 0) return out_row ? zero_rows(ctx, C, dtype, out_rows, R, ldc, stream) : COMET_OK;
   if (dtype == COMET_F32)
     return seg_gather_typed<float>(ctx, seg_end, crd, (const float *)val, M, N, (const float *)B, ldb, R, (float *)C, ldc,
-                                   out_row, out_rows, stream);
+                                   out_row, out_rows, b_rows, stream);
   return seg_gather_typed<double>(ctx, seg_end, crd, (const double *)val, M, N, (const double *)B, ldb, R, (double *)C,
-                                  ldc, out_row, out_rows, stream);
+                                  ldc, out_row, out_rows, b_rows, stream);
 }
 
 }  // namespace comet

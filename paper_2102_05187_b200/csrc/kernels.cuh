@@ -6,11 +6,13 @@
 namespace comet {
 
 // out[row(s), 0..R) = sum over leaf entries p of segment s of val[p] * B[crd[p], 0..R)   (SpMM, TTM)
-// seg_end[s] = leaf position where segment s ends. out_row == NULL: row(s) = s; otherwise row(s) =
-// out_row[s] (ascending) and all other rows below out_rows are zero-filled.
+// seg_end[s] = leaf position where segment s ends; seg_end - 1 must be readable and hold 0 (seg_end = pos + 1).
+// out_row == NULL: row(s) = s; otherwise row(s) = out_row[s] (ascending) and all other rows below out_rows are
+// zero-filled. b_rows = number of rows of B (0: unknown; only used to decide on the long-row path of SpMM).
 comet_status_t seg_gather(Context *ctx, int dtype, const int32_t *seg_end, const int32_t *crd, const void *val,
                           int64_t M, int64_t N, const void *B, int64_t ldb, int64_t R, void *C, int64_t ldc,
-                          const int32_t *out_row, int64_t out_rows, cudaStream_t stream);
+                          const int32_t *out_row, int64_t out_rows, int64_t b_rows, cudaStream_t stream);
+
 
 // y[row(s)] = sum over leaf entries p of segment s of val[p] * x[crd[p]]                    (SpMV, TTV)
 comet_status_t seg_dot(Context *ctx, int dtype, const int32_t *seg_end, const int32_t *crd, const void *val, int64_t M,

@@ -73,9 +73,24 @@ __device__ __forceinline__ void sts_s32(uint32_t addr, int32_t v) {
 // gathers keep their program order relative to the ring reads: exactly the rolling window is in flight
 // (the scheduler otherwise hoists loads of far-ahead entries and spills).
 template <class T, int VEC> struct Piece;
+// L2 eviction policies for the gathers of a kernel whose CTAs play two roles at once: rows that are re-used out
+// of L2 are kept (evict_last) while rows that are read once pass through (evict_first).
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
 template <> struct Piece<double, 2> {
   static __device__ __forceinline__ void load(const double *p, double (&d)[2]) {
     asm volatile("ld.global.nc.v2.f64 {%0, %1}, [%2];" : "=d"(d[0]), "=d"(d[1]) : "l"(p));
+  }
+  static __device__ __forceinline__ void load_hint(const double *p, double (&d)[2], uint64_t pol) {
+    asm volatile("ld.global.nc.L2::cache_hint.v2.f64 {%0, %1}, [%2], %3;" : "=d"(d[0]), "=d"(d[1]) : "l"(p), "l"(pol));
   }
   static __device__ __forceinline__ void store_stream(double *p, const double (&d)[2]) {
     __stcs(reinterpret_cast<double2 *>(p), make_double2(d[0], d[1]));
@@ -90,6 +105,10 @@ template <> struct Piece<double, 1> {
 template <> struct Piece<float, 4> {
   static __device__ __forceinline__ void load(const float *p, float (&d)[4]) {
     asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3]) : "l"(p));
+  }
+  static __device__ __forceinline__ void load_hint(const float *p, float (&d)[4], uint64_t pol) {
+    asm volatile("ld.global.nc.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3]) : "l"(p), "l"(pol));
   }
   static __device__ __forceinline__ void store_stream(float *p, const double (&d)[4]) {
     __stcs(reinterpret_cast<float4 *>(p), make_float4((float)d[0], (float)d[1], (float)d[2], (float)d[3]));
@@ -138,6 +157,15 @@ template <class T_, int LPN_, int CPL_, int VEC_> struct Lanes {
 #pragma unroll
     for (int t = 0; t < CPL; ++t)
       if (ok[t]) Piece<T, VEC>::load(row + t * kStride, dst[t]);
+  }
+  // the same with an L2 eviction policy (128-bit pieces only; the other shapes never carry two roles)
+  __device__ __forceinline__ void gather_hint(const T *row, T (&dst)[CPL][VEC], uint64_t pol) const {
+    if constexpr (VEC * sizeof(T) == 16) {
+#pragma unroll
+      for (int t = 0; t < CPL; ++t) Piece<T, VEC>::load_hint(row + t * kStride, dst[t], pol);
+    } else {
+      gather(row, dst);
+    }
   }
   __device__ __forceinline__ void store_row(T *row, const double (&acc)[CPL][VEC]) const {
 #pragma unroll
