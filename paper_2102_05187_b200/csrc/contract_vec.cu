@@ -177,6 +177,8 @@ seg_gather_kernel(const SegGatherArgs a, const HeavyArgs h) {
 
 // Adds the carries onto the stored rows. Tiles that stopped inside the same segment are consecutive;
 // the first of such a run sums the run in tile order and updates the row (the only writer of it now).
+// A heavy segment spans hundreds of tiles, so the run is read eight tiles at a time with all loads in
+// flight together (the additions keep the tile order).
 template <class T>
 __global__ void carry_fixup_kernel(const double *__restrict__ carry_val, const int32_t *__restrict__ carry_seg,
                                    int64_t num_tiles, int32_t R, int32_t carry_ld, T *__restrict__ C,
@@ -188,8 +190,23 @@ __global__ void carry_fixup_kernel(const double *__restrict__ carry_val, const i
   const int32_t seg = carry_seg[tile];
   if (seg < 0) return;
   if (tile > 0 && carry_seg[tile - 1] == seg) return;
-  double sum = 0.0;
-  for (int64_t t = tile; t < num_tiles && carry_seg[t] == seg; ++t) sum += carry_val[t * carry_ld + c];
+  double sum = carry_val[tile * carry_ld + c];
+  bool more = true;
+  for (int64_t t = tile + 1; more; t += 8) {
+    int32_t s[8];
+    double v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const bool in = t + u < num_tiles;
+      s[u] = in ? __ldg(carry_seg + t + u) : -2;
+      v[u] = in ? __ldcs(carry_val + (t + u) * carry_ld + c) : 0.0;
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      more = more && s[u] == seg;
+      if (more) sum += v[u];
+    }
+  }
   const int64_t row = out_row ? (int64_t)out_row[seg] : (int64_t)seg;
   C[row * ldc + c] = (T)((double)C[row * ldc + c] + sum);
 }

@@ -8,6 +8,8 @@
 // consecutive leaf entries with a rolling window of row gathers in flight. A worker stores the output rows that END in its tile (and zero-fills the
 // rows between consecutive stored rows, so no memset is needed), and writes the partial sum of the
 // row it stops in to a carry slot that the fix-up kernel adds in tile order (deterministic).
+#include <stdlib.h>
+
 #include "common.cuh"
 #include "kernels.cuh"
 #include "walk.cuh"
@@ -16,10 +18,13 @@
 #define COMET_PF_COO 2        // entries in flight per worker, two row gathers each
 #endif
 #ifndef COMET_PF_CSF
-#define COMET_PF_CSF 4
+#define COMET_PF_CSF 2       // entries in flight per worker (a Q row each, a P row where a fiber closes)
 #endif
 #ifndef COMET_MINB_COO
 #define COMET_MINB_COO 4
+#endif
+#ifndef COMET_CSF_ROLLED_TAIL
+#define COMET_CSF_ROLLED_TAIL true
 #endif
 #ifndef COMET_MINB_CSF
 #define COMET_MINB_CSF 4
@@ -45,6 +50,7 @@ struct MttkrpArgs {
   double *carry_val;
   int32_t *carry_seg;
   int32_t carry_ld;
+  const int32_t *part_fiber, *part_slice;   // CSF: per tile boundary, from the partition kernel (num_tiles + 1 each)
 };
 
 // ------------------------------------------------------------------------------------------- COO
@@ -136,13 +142,40 @@ __global__ void __launch_bounds__(kBlockThreads, (CPL * VEC * sizeof(T) <= 16 ? 
 }
 
 // ------------------------------------------------------------------------------------------- CSF
-template <class T, int LPN, int CPL, int VEC>
+// Fibers are short (a few entries, most of them one), so what is done per FIBER decides the speed. The fibers
+// and slices of a tile are therefore looked at once, before the walk and by all lanes at once: a worker scans the
+// fiber ends that fall into its tile (coalesced reads of the level-2 positions and of the level-1 coordinates)
+// and leaves, in a shared-memory array with one word per leaf entry of the tile, the P row index at the LAST
+// entry of every fiber (-1 elsewhere); a second scan over the slices of the tile sets the top bit at the last
+// entry of every slice. The walk then finds everything it needs in the staged entry: an entry that closes a
+// fiber has that fiber's P row gathered together with its own Q row (same window, same distance ahead), closing
+// a fiber is "slice sum += fiber sum * P row", closing a slice is one row store. No positions are followed and
+// nothing is looked up entry by entry.
+constexpr int32_t kNoEnd = -1;                      // flag word: no fiber ends at this entry
+constexpr uint32_t kSliceEnd = 0x80000000u;         // flag word: P row index, top bit set if the slice ends too
+                                                    // (a coordinate is below 2^31 - 1, so the two never collide)
+constexpr int kCsfTileCap = 512;                    // leaf entries per tile: 16 mask words
+constexpr int kCsfMaskWords = kCsfTileCap / 32;
+constexpr int kCsfWorkerBytes = 3 * kCsfMaskWords * 4;   // fiber-end bits, slice-end bits, fiber ends in front of each word
+
+__device__ __forceinline__ void atom_or_shared(uint32_t addr, uint32_t bits) {
+  asm volatile("red.shared.or.b32 [%0], %1;" ::"r"(addr), "r"(bits) : "memory");
+}
+
+// EXPAND: when the fibers are so short that most entries close one (mean length below 4), following the fibers
+// costs more than it saves. The staging then hands EVERY entry the P row index of its fiber (the number of fiber
+// ends in front of an entry is its fiber's number), both rows are gathered per entry, and the walk is the one of
+// the sorted-COO kernel: slice sum += (x * P row) * Q row, a row store where a slice ends. The P rows of a
+// fiber's later entries are L1 hits.
+template <class T, int LPN, int CPL, int VEC, bool EXPAND>
 struct CsfPolicy {
   using L = Lanes<T, LPN, CPL, VEC>;
   static constexpr int kPF = COMET_PF_CSF;
   static constexpr bool kAux = false;
-  static constexpr bool kFullUnroll = false;   // the fiber/slice epilogue is long: keep the body small
-  struct Slot { T r[CPL][VEC]; };
+  static constexpr bool kFullUnroll = true;
+  static constexpr bool kRolledTail = COMET_CSF_ROLLED_TAIL;
+  static constexpr bool kEntryConsume = true;
+  struct Slot { T r[CPL][VEC]; T p[CPL][VEC]; };           // Q row of the entry; P row of its fiber if it closes one
 
   const MttkrpArgs &a;
   const L &ln;
@@ -151,130 +184,202 @@ struct CsfPolicy {
   T *ocol;
   const T *val;
   double tac[CPL][VEC], aac[CPL][VEC];   // open fiber sum, open slice sum
-  T prow[CPL][VEC];                      // P row of the open fiber
-  T pnext[CPL][VEC];                     // P row of the fiber after it: fetched one fiber ahead, so that a fold
-                                         // never waits for its gather (fibers are a few entries long)
-  int32_t end1;                          // leaf position where the fiber after the open one ends
-  // cursors instead of indices: the per-fiber path is executed once per fiber and per worker (divergently),
-  // so it is kept to pointer bumps and 32-bit compares
-  const int32_t *endp;                   // seg_end2 + open fiber
-  const int32_t *c1p;                    // crd1 + open fiber
-  int32_t fibers_left;                   // fibers from the open one to the last
-  int32_t to_slice_end;                  // fibers from the open one to the end of the open slice
+  uint32_t ends, slices, before;         // shared addresses of the tile's three word arrays
+  int32_t j0, f0;
   int32_t s;                             // open slice
-  int32_t next_end;                      // leaf position where the open fiber ends
-  int32_t base, rel_end;
-  int32_t last_fold;                     // leaf position of the latest fold (entries at or after it are in tac)
+  int32_t f_open;                        // the fiber that is still open behind the tile's last fiber end
   bool a_dirty;
 
-  __device__ __forceinline__ CsfPolicy(const MttkrpArgs &args, const L &lanes, int64_t f0, int64_t s0, int32_t j0)
-      : a(args), ln(lanes), s((int32_t)s0), base(j0), last_fold(j0), a_dirty(false) {
+  // The look at the tile's fibers and slices (see above). f0 = first fiber that ends behind j0, s0 = its slice.
+  __device__ __forceinline__ CsfPolicy(const MttkrpArgs &args, const L &lanes, int64_t f0_, int64_t s0, int32_t j0_, int32_t j1,
+                                       uint32_t smem_words)
+      : a(args), ln(lanes), ends(smem_words), slices(smem_words + kCsfMaskWords * 4), before(smem_words + 2 * kCsfMaskWords * 4),
+        j0(j0_), f0((int32_t)f0_), s((int32_t)s0), a_dirty(false) {
     ln.zero(tac);
     ln.zero(aac);
-#pragma unroll
-    for (int t = 0; t < CPL; ++t)
-#pragma unroll
-      for (int k = 0; k < VEC; ++k) { prow[t][k] = (T)0; pnext[t][k] = (T)0; }
     pcol = reinterpret_cast<const char *>(static_cast<const T *>(a.P) + ln.col0);
     qcol = reinterpret_cast<const char *>(static_cast<const T *>(a.Q) + ln.col0);
     ldp_bytes = (int32_t)(a.ldp * sizeof(T));
     ldq_bytes = (int32_t)(a.ldq * sizeof(T));
     ocol = static_cast<T *>(a.out) + ln.col0;
     val = static_cast<const T *>(a.val);
-    endp = a.seg_end2 + f0;
-    c1p = a.crd1 + f0;
-    fibers_left = (int32_t)(a.F - f0);
-    next_end = fibers_left > 0 ? __ldg(endp) : -1;
-    end1 = fibers_left > 1 ? __ldg(endp + 1) : -1;
-    rel_end = next_end - base;
-    to_slice_end = s < a.S ? (int32_t)(__ldg(a.pos1 + s + 1) - f0) : -1;
-    if (fibers_left > 0) ln.gather(reinterpret_cast<const T *>(pcol + (int64_t)__ldg(c1p) * ldp_bytes), prow);
-    fetch_ahead();
+    for (int w = ln.g; w < 2 * kCsfMaskWords; w += LPN) sts_s32(ends + w * 4, 0);
+    ln.sync();
+    int32_t closed = 0;                                    // fibers that end inside the tile
+    for (int64_t k = f0_ + ln.g;; k += LPN) {
+      const int32_t e = k < a.F ? __ldg(a.seg_end2 + k) : 0x7fffffff;
+      const bool in = e <= j1;
+      if (in) atom_or_shared(ends + ((e - 1 - j0) >> 5) * 4, 1u << ((e - 1 - j0) & 31));
+      const int got = __popc(__ballot_sync(ln.mask, in) & ln.mask);
+      closed += got;
+      if (got != LPN) break;                               // ends ascend: a lane outside means the scan is over
+    }
+    f_open = f0 + closed;
+    for (int64_t k = s0 + ln.g;; k += LPN) {               // slice k ends with fiber pos1[k + 1] - 1
+      const int64_t last = k < a.S ? (int64_t)__ldg(a.pos1 + k + 1) - 1 : -1;
+      const bool in = last >= 0 && last < f_open;
+      if (in) {
+        const int32_t q = __ldg(a.seg_end2 + last) - 1 - j0;
+        atom_or_shared(slices + (q >> 5) * 4, 1u << (q & 31));
+      }
+      if (__popc(__ballot_sync(ln.mask, in) & ln.mask) != LPN) break;
+    }
+    ln.sync();
+    for (int w = ln.g; w < kCsfMaskWords; w += LPN) {
+      int32_t cnt = 0;
+      for (int x = 0; x < w; ++x) cnt += __popc((uint32_t)lds_s32(ends + x * 4));
+      sts_s32(before + w * 4, cnt);
+    }
+    ln.sync();
   }
-  __device__ __forceinline__ int64_t fiber() const { return a.F - fibers_left; }
-  __device__ __forceinline__ void fetch_ahead() {        // start fetching the P row of the fiber after the open one
-    if (fibers_left > 1) ln.gather(reinterpret_cast<const T *>(pcol + (int64_t)__ldg(c1p + 1) * ldp_bytes), pnext);
+  __device__ __forceinline__ void begin_chunk(int32_t) {}
+  // the flag word of leaf entry j: the P row index of its fiber if it is the fiber's last entry
+  __device__ __forceinline__ int32_t flag_of(int32_t j) const {
+    const int32_t q = j - j0;
+    const uint32_t w = (uint32_t)lds_s32(ends + (q >> 5) * 4);
+    const uint32_t bit = 1u << (q & 31);
+    if (!EXPAND && !(w & bit)) return kNoEnd;
+    const int32_t f = f0 + lds_s32(before + (q >> 5) * 4) + __popc(w & (bit - 1u));
+    const uint32_t row = (uint32_t)__ldg(a.crd1 + f);
+    return (int32_t)(((uint32_t)lds_s32(slices + (q >> 5) * 4) & bit) ? (row | kSliceEnd) : row);
   }
   __device__ __forceinline__ void fetch(int32_t j, Entry16 &e, int32_t &) const {
     e.v = (double)ld_stream(val + j);
     e.a = ld_stream(a.crd2 + j);
+    e.b = flag_of(j);
   }
-  __device__ __forceinline__ void prefetch(int32_t ck, int32_t, Slot &sl) const {
+  __device__ __forceinline__ void prefetch(int32_t ck, int32_t flag, Slot &sl) const {
     ln.gather(reinterpret_cast<const T *>(qcol + (int64_t)ck * ldq_bytes), sl.r);
+    if (EXPAND || flag != kNoEnd)
+      ln.gather(reinterpret_cast<const T *>(pcol + (int64_t)(int32_t)((uint32_t)flag & ~kSliceEnd) * ldp_bytes), sl.p);
   }
-  __device__ __forceinline__ void begin_chunk(int32_t b) { base = b; rel_end = next_end - b; }
-
-  __device__ __forceinline__ void fold(int32_t j) {      // aac += tac * P[crd1[f], :]
+  __device__ __forceinline__ void fold(const T (&prow)[CPL][VEC]) {      // aac += tac * P[crd1[f], :]
 #pragma unroll
     for (int t = 0; t < CPL; ++t)
       if (ln.ok[t])
 #pragma unroll
         for (int k = 0; k < VEC; ++k) { aac[t][k] = fma(tac[t][k], (double)prow[t][k], aac[t][k]); tac[t][k] = 0.0; }
     a_dirty = true;
-    last_fold = j;
   }
-  __device__ __forceinline__ void close_slice() {        // the slice is complete: this worker owns its row
-    const int64_t row = __ldg(a.crd0 + s);
-    const int64_t lo = s > 0 ? (int64_t)__ldg(a.crd0 + s - 1) + 1 : 0;
-    ln.zero_rows(ocol, a.ldo, lo, row);
-    ln.store_row(ocol + row * a.ldo, aac);
-    if (s == a.S - 1) ln.zero_rows(ocol, a.ldo, row + 1, a.rows);
+  // The slice is complete: this worker owns its row. (The rows that no slice owns are zero-filled by a kernel of
+  // their own, so that this stays short.)
+  __device__ __forceinline__ void close_slice() {
+    ln.store_row(ocol + (int64_t)__ldg(a.crd0 + s) * a.ldo, aac);
     ln.zero(aac);
     a_dirty = false;
     ++s;
-    to_slice_end = s < a.S ? __ldg(a.pos1 + s + 1) - __ldg(a.pos1 + s) : -1;
   }
-  __device__ __forceinline__ void end_fiber(int32_t j) {
-    fold(j);
-    ++endp;
-    ++c1p;
-    --fibers_left;
-    next_end = end1;                                     // loaded one fiber ago
-    end1 = fibers_left > 1 ? __ldg(endp + 1) : -1;
-    rel_end = next_end - base;
+  __device__ __forceinline__ void consume_entry(int, const Entry16 &e, Slot &sl) {
+    if (EXPAND) {
 #pragma unroll
-    for (int t = 0; t < CPL; ++t)
+      for (int t = 0; t < CPL; ++t)
+        if (ln.ok[t])
 #pragma unroll
-      for (int k = 0; k < VEC; ++k) prow[t][k] = pnext[t][k];
-    fetch_ahead();
-    if (--to_slice_end == 0) close_slice();
+          for (int k = 0; k < VEC; ++k) aac[t][k] = fma(e.v * (double)sl.p[t][k], (double)sl.r[t][k], aac[t][k]);
+      if (e.b < 0) close_slice();
+      return;
+    }
+    ln.fma_rows(e.v, sl.r, tac);
+    if (e.b != kNoEnd) {
+      fold(sl.p);
+      if (e.b < 0) close_slice();
+    }
   }
-  __device__ __forceinline__ void consume(int q, double v, int32_t, Slot &sl) {
-    while (rel_end == q) end_fiber(base + q);
-    ln.fma_rows(v, sl.r, tac);
+  // After the walk of [j0, j1): the entries behind the last fiber end belong to a fiber that goes on in the next
+  // tile; they contribute through distributivity.
+  __device__ __forceinline__ void finish(int32_t j1) {
+    const int32_t q = j1 - 1 - j0;
+    if (EXPAND) {                                          // the slice sum is open unless the last entry closed a slice
+      a_dirty = !(((uint32_t)lds_s32(slices + (q >> 5) * 4) >> (q & 31)) & 1u);
+      return;
+    }
+    if (((uint32_t)lds_s32(ends + (q >> 5) * 4) >> (q & 31)) & 1u) return;     // the tile stops at a fiber end
+    T prow[CPL][VEC];
+    ln.gather(reinterpret_cast<const T *>(pcol + (int64_t)__ldg(a.crd1 + f_open) * ldp_bytes), prow);
+    fold(prow);
   }
 };
 
-template <class T, int LPN, int CPL, int VEC>
+// Tile boundaries of the CSF kernel, a thread per boundary: the merge-path split of (fiber-end markers, leaf
+// positions) at item t * tile_items, then the slice of the first fiber whose entries reach into the tile. The
+// slice is stored complemented when that fiber is the one after the split's (its end marker is the next item).
+__global__ void __launch_bounds__(kBlockThreads) csf_partition_kernel(const int32_t *__restrict__ seg_end2,
+                                                                      const int32_t *__restrict__ pos1, int64_t S, int64_t F,
+                                                                      int64_t N, int32_t tile_items, int64_t num_tiles,
+                                                                      int32_t *__restrict__ part_fiber,
+                                                                      int32_t *__restrict__ part_slice) {
+  const int64_t t = (int64_t)blockIdx.x * kBlockThreads + threadIdx.x;
+  if (t > num_tiles) return;
+  const int64_t total = F + N;
+  const int64_t d = t * tile_items < total ? t * tile_items : total;
+  int64_t f = merge_path_segments(seg_end2, F, N, d);
+  part_fiber[t] = (int32_t)f;
+  const bool skip = f < F && (int64_t)__ldg(seg_end2 + f) == d - f;
+  if (skip) ++f;
+  int64_t lo = 0, hi = S;                                  // slices that end at or before fiber f (every slice is non-empty)
+  while (lo < hi) {
+    const int64_t mid = (lo + hi) >> 1;
+    if ((int64_t)__ldg(pos1 + mid + 1) <= f) lo = mid + 1; else hi = mid;
+  }
+  part_slice[t] = skip ? ~(int32_t)lo : (int32_t)lo;
+}
+
+// Zero-fills the output rows that no slice owns: the rows between the coordinates of consecutive slices, before
+// the first and behind the last. A warp looks at 32 slices at a time and clears the gaps it finds together.
+template <class T>
+__global__ void __launch_bounds__(kBlockThreads) zero_unowned_rows_kernel(const int32_t *__restrict__ crd0, int64_t S, int64_t rows,
+                                                                          T *__restrict__ out, int64_t ldo, int32_t R) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = ((int64_t)blockIdx.x * kBlockThreads + threadIdx.x) >> 5;
+  const int64_t s = warp * 32 + lane;                      // gap s lies in front of slice s; gap S behind the last slice
+  int64_t lo = 0, hi = 0;
+  if (s <= S) {
+    lo = s > 0 ? (int64_t)__ldg(crd0 + s - 1) + 1 : 0;
+    hi = s < S ? (int64_t)__ldg(crd0 + s) : rows;
+  }
+  unsigned todo = __ballot_sync(0xffffffffu, hi > lo);
+  while (todo) {
+    const int src = __ffs(todo) - 1;
+    todo &= todo - 1;
+    const int64_t a = __shfl_sync(0xffffffffu, lo, src), b = __shfl_sync(0xffffffffu, hi, src);
+    for (int64_t i = (a * R) + lane; i < b * R; i += 32) {
+      const int64_t r = i / R;
+      out[r * ldo + (i - r * R)] = (T)0;
+    }
+  }
+}
+
+template <class T, int LPN, int CPL, int VEC, bool EXPAND>
 __global__ void __launch_bounds__(kBlockThreads, (CPL * VEC * sizeof(T) <= 16 ? COMET_MINB_CSF : 2)) mttkrp_csf_kernel(const MttkrpArgs a) {
   using L = Lanes<T, LPN, CPL, VEC>;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int worker = threadIdx.x / LPN;
   const int64_t tile = (int64_t)blockIdx.x * L::kWorkers + worker;
   if (tile >= a.num_tiles) return;
-  using P = CsfPolicy<T, LPN, CPL, VEC>;
+  using P = CsfPolicy<T, LPN, CPL, VEC, EXPAND>;
   const uint32_t smem = smem_u32(smem_raw) + worker * RingLayout<L, false>::kWorkerBytes;
+  const uint32_t flags = smem_u32(smem_raw) + (uint32_t)RingLayout<L, false>::kBlockBytes + worker * kCsfWorkerBytes;
   const L ln(a.R);
 
-  // tile = a span of the merge list of fiber-end markers and leaf positions
+  // A tile is a span of the merge list of fiber-end markers and leaf positions (equal work per tile: an entry
+  // costs a gather, a fiber another one). It owns the leaf entries of the span and the fibers whose LAST entry
+  // is among them.
+  // Where the tile starts (fiber, slice) was found by the partition kernel: a worker is sequential, so dependent
+  // searches at the head of every tile would cost it a third of its time.
   const int64_t total = a.F + a.N;
   const int64_t d0 = tile * a.tile_items;
   const int64_t d1 = (d0 + a.tile_items < total) ? d0 + a.tile_items : total;
-  const int64_t f0 = merge_path_segments_coop<LPN>(a.seg_end2, a.F, a.N, d0, ln.g, ln.mask);
-  const int64_t f1 = merge_path_segments_coop<LPN>(a.seg_end2, a.F, a.N, d1, ln.g, ln.mask);
+  const int64_t f0 = __ldg(a.part_fiber + tile), f1 = __ldg(a.part_fiber + tile + 1);
   const int32_t j0 = (int32_t)(d0 - f0), j1 = (int32_t)(d1 - f1);
-
-  // slice that holds fiber f0: the number of slices that end at or before it (every slice is non-empty)
-  int64_t lo = 0, hi = a.S;
-  while (lo < hi) {
-    const int64_t mid = (lo + hi) >> 1;
-    if ((int64_t)__ldg(a.pos1 + mid + 1) <= f0) lo = mid + 1; else hi = mid;
+  if (j0 >= j1) {                                          // nothing but an end marker: its fiber was closed by the tile before
+    if (ln.g == 0) a.carry_seg[tile] = -1;
+    return;
   }
-
-  P p(a, ln, f0, lo, j0);
+  const int32_t s0 = __ldg(a.part_slice + tile);
+  // the first fiber of the tile: the one the partition found, unless all its entries lie in earlier tiles
+  P p(a, ln, f0 + (s0 < 0 ? 1 : 0), s0 < 0 ? ~s0 : s0, j0, j1, flags);
   walk_tile(ln, p, j0, j1, smem);
-  while (p.fiber() < f1) p.end_fiber(j1);
-  if (j1 > p.last_fold) p.fold(j1);                      // an unfinished fiber contributes through distributivity
+  p.finish(j1);
   const bool carry = p.a_dirty && p.s < a.S;
   if (ln.g == 0) a.carry_seg[tile] = carry ? (int32_t)p.s : -1;
   if (carry) ln.store_carry(a.carry_val + tile * a.carry_ld + ln.col0, p.aac);
@@ -287,19 +392,34 @@ template <bool CSF, class T, int LPN, int CPL, int VEC>
 static comet_status_t launch_mttkrp(Context *ctx, MttkrpArgs a, cudaStream_t stream) {
   constexpr int WORKERS = kBlockThreads / LPN;
   const int64_t total = CSF ? a.F + a.N : a.N;
+  using L = Lanes<T, LPN, CPL, VEC>;
   a.tile_items = choose_tile_items(total, WORKERS);
+  if (CSF && a.tile_items > kCsfTileCap) a.tile_items = kCsfTileCap;          // one mask bit per leaf entry of a tile
   a.num_tiles = ceil_div(total, a.tile_items);
   a.carry_ld = (int32_t)align_up((size_t)a.R, 2);
   const size_t val_bytes = align_up((size_t)a.num_tiles * a.carry_ld * sizeof(double), 256);
   const size_t seg_bytes = align_up((size_t)a.num_tiles * sizeof(int32_t), 256);
-  char *scratch = (char *)scratch_get(ctx, val_bytes + seg_bytes, stream);
+  const size_t part_bytes = CSF ? align_up((size_t)(a.num_tiles + 1) * sizeof(int32_t), 256) : 0;
+  char *scratch = (char *)scratch_get(ctx, val_bytes + seg_bytes + 2 * part_bytes, stream);
   if (!scratch) return COMET_ERR_ALLOC;
   a.carry_val = (double *)scratch;
   a.carry_seg = (int32_t *)(scratch + val_bytes);
+  if (CSF) {
+    int32_t *pf = (int32_t *)(scratch + val_bytes + seg_bytes), *ps = (int32_t *)(scratch + val_bytes + seg_bytes + part_bytes);
+    csf_partition_kernel<<<(unsigned)ceil_div(a.num_tiles + 1, kBlockThreads), kBlockThreads, 0, stream>>>(
+        a.seg_end2, a.pos1, a.S, a.F, a.N, a.tile_items, a.num_tiles, pf, ps);
+    COMET_LAUNCH_CHECK(ctx);
+    a.part_fiber = pf;
+    a.part_slice = ps;
+  }
   const unsigned blocks = (unsigned)ceil_div(a.num_tiles, WORKERS);
-  using L = Lanes<T, LPN, CPL, VEC>;
-  constexpr size_t smem = CSF ? RingLayout<L, false>::kBlockBytes : RingLayout<L, true>::kBlockBytes;
-  auto kernel = CSF ? mttkrp_csf_kernel<T, LPN, CPL, VEC> : mttkrp_coo_kernel<T, LPN, CPL, VEC>;
+  constexpr size_t smem = CSF ? RingLayout<L, false>::kBlockBytes + (size_t)WORKERS * kCsfWorkerBytes
+                              : RingLayout<L, true>::kBlockBytes;
+  // CSF with short fibers (mean length below 4): the per-entry form; COMET_CSF_FORM=fold / expand forces one
+  bool expand = CSF && a.N < 4 * a.F;
+  if (const char *e = getenv("COMET_CSF_FORM")) expand = CSF && (e[0] == 'e' ? true : (e[0] == 'f' ? false : expand));
+  auto kernel = !CSF ? mttkrp_coo_kernel<T, LPN, CPL, VEC>
+                     : (expand ? mttkrp_csf_kernel<T, LPN, CPL, VEC, true> : mttkrp_csf_kernel<T, LPN, CPL, VEC, false>);
   if (smem > 48 * 1024)
     COMET_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   kernel<<<blocks, kBlockThreads, smem, stream>>>(a);
@@ -364,6 +484,12 @@ comet_status_t mttkrp_csf(Context *ctx, int dtype, const int32_t *pos1, const in
   a.pos1 = pos1; a.crd0 = crd0; a.crd1 = crd1; a.seg_end2 = pos2 + 1; a.crd2 = crd2; a.val = val;
   a.S = S; a.F = F; a.N = N; a.rows = rows;
   a.P = P; a.ldp = ldp; a.Q = Q; a.ldq = ldq; a.out = out; a.ldo = ldo;
+  {                                                        // rows that no slice owns (all R columns at once)
+    const unsigned blocks = (unsigned)ceil_div(S + 1, kBlockThreads);
+    if (dtype == COMET_F32) zero_unowned_rows_kernel<float><<<blocks, kBlockThreads, 0, stream>>>(crd0, S, rows, (float *)out, ldo, (int32_t)R);
+    else zero_unowned_rows_kernel<double><<<blocks, kBlockThreads, 0, stream>>>(crd0, S, rows, (double *)out, ldo, (int32_t)R);
+    COMET_LAUNCH_CHECK(ctx);
+  }
   return dtype == COMET_F32 ? mttkrp_chunks<true, float>(ctx, a, R, stream) : mttkrp_chunks<true, double>(ctx, a, R, stream);
 }
 

@@ -203,45 +203,93 @@ template <class L, bool AUX> struct RingLayout {
   static constexpr size_t kBlockBytes = (size_t)L::kWorkers * kWorkerBytes;
 };
 
-// One chunk: positions 0..n-1 of the ring half at shared address `cur`; `nxt` is the other half.
-// kFullUnroll policies get the whole chunk unrolled (ring offsets and positions are immediates); the
-// others (heavy per-segment work, where code size matters more) get a loop of kPF-wide unrolled steps.
+// A policy that declares `static constexpr bool kPositional = true` is told WHERE the entry it prefetches sits
+// (position `at` of the current or of the next chunk) through prefetch_at(at, in_current_chunk, a, b, slot):
+// for policies that keep per-chunk information about the entries (the CSF fiber-end masks).
+template <class P, class = void> struct policy_is_positional { static constexpr bool value = false; };
+template <class P> struct policy_is_positional<P, decltype((void)P::kPositional)> { static constexpr bool value = P::kPositional; };
+
+// A policy that declares `static constexpr bool kTwoSpeed = true` has two ways to consume an entry: the full
+// consume(), and consume_plain() for the chunks for which plain_chunk() says that the rare, long part of
+// consume() cannot happen (end_plain_chunk() then settles the bookkeeping for the whole chunk). Only the plain
+// form is unrolled; the full form runs as a loop, so the code stays small enough for the instruction cache.
+template <class P, class = void> struct policy_is_two_speed { static constexpr bool value = false; };
+template <class P> struct policy_is_two_speed<P, decltype((void)P::kTwoSpeed)> { static constexpr bool value = P::kTwoSpeed; };
+
+// kEntryConsume: the policy wants the whole staged entry (value and both coordinate words, one 128-bit read)
+// when it consumes it, through consume_entry(q, entry, slot): for flags that travel in the coordinate words.
+template <class P, class = void> struct policy_consumes_entry { static constexpr bool value = false; };
+template <class P> struct policy_consumes_entry<P, decltype((void)P::kEntryConsume)> { static constexpr bool value = P::kEntryConsume; };
+
+template <class P, class = void> struct policy_rolls_tail { static constexpr bool value = false; };
+template <class P> struct policy_rolls_tail<P, decltype((void)P::kRolledTail)> { static constexpr bool value = P::kRolledTail; };
+
+// One chunk, unrolled: positions 0..n-1 of the ring half at shared address `cur`; `nxt` is the other half. Ring
+// offsets and positions are immediates.
+template <class L, class Policy, bool TAIL, bool PLAIN>
+__device__ __forceinline__ void walk_chunk_unrolled(Policy &p, typename Policy::Slot (&win)[Policy::kPF], uint32_t cur,
+                                                    uint32_t nxt, uint32_t cur_aux, uint32_t nxt_aux, int n) {
+  constexpr int kChunk = L::kChunk, kPF = Policy::kPF;
+#pragma unroll
+  for (int q = 0; q < kChunk; ++q) {
+    if (TAIL && q >= n) break;
+    if constexpr (PLAIN) p.consume_plain(q, lds_f64(cur + q * 16), win[q % kPF]);
+    else if constexpr (policy_consumes_entry<Policy>::value) p.consume_entry(q, lds_entry(cur + q * 16), win[q % kPF]);
+    else p.consume(q, lds_f64(cur + q * 16), Policy::kAux ? lds_s32(cur_aux + q * 4) : 0, win[q % kPF]);
+    // refill the slot with the entry kPF ahead (it may sit in the next chunk's half of the ring);
+    // the last, partial chunk only looks ahead inside itself
+    if (TAIL && q + kPF >= n) continue;
+    const bool in_cur = q + kPF < kChunk;
+    const int at = in_cur ? q + kPF : q + kPF - kChunk;
+    int32_t ca, cb;
+    lds_coords((in_cur ? cur : nxt) + at * 16, ca, cb);
+    if constexpr (policy_is_positional<Policy>::value) p.prefetch_at(at, in_cur, ca, cb, win[q % kPF]);
+    else p.prefetch(ca, cb, win[q % kPF]);
+  }
+}
+
+// One chunk as a loop of kPF-wide unrolled steps (for heavy per-segment work, where code size matters more).
+template <class L, class Policy, bool TAIL>
+__device__ __forceinline__ void walk_chunk_rolled(Policy &p, typename Policy::Slot (&win)[Policy::kPF], uint32_t cur,
+                                                  uint32_t nxt, uint32_t cur_aux, uint32_t nxt_aux, int n) {
+  constexpr int kChunk = L::kChunk, kPF = Policy::kPF;
+  // the two halves are adjacent in shared memory: position q + kPF of `cur` wraps into `nxt`
+  const uint32_t lo = cur < nxt ? cur : nxt, lo_aux = cur_aux < nxt_aux ? cur_aux : nxt_aux;
+  const int off = cur < nxt ? 0 : kChunk;
+#pragma unroll 1
+  for (int q0 = 0; q0 < (TAIL ? n : kChunk); q0 += kPF) {
+#pragma unroll
+    for (int u = 0; u < kPF; ++u) {
+      const int q = q0 + u;
+      if (TAIL && q >= n) break;
+      const int r = off + q;
+      if constexpr (policy_consumes_entry<Policy>::value) p.consume_entry(q, lds_entry(lo + r * 16), win[u]);
+      else p.consume(q, lds_f64(lo + r * 16), Policy::kAux ? lds_s32(lo_aux + r * 4) : 0, win[u]);
+      if (TAIL && q + kPF >= n) continue;
+      int32_t ca, cb;
+      lds_coords(lo + ((r + kPF) & (2 * kChunk - 1)) * 16, ca, cb);
+      if constexpr (policy_is_positional<Policy>::value) p.prefetch_at((q + kPF) & (kChunk - 1), q + kPF < kChunk, ca, cb, win[u]);
+      else p.prefetch(ca, cb, win[u]);
+    }
+  }
+}
+
 template <class L, class Policy, bool TAIL>
 __device__ __forceinline__ void walk_chunk(Policy &p, typename Policy::Slot (&win)[Policy::kPF], uint32_t cur,
                                            uint32_t nxt, uint32_t cur_aux, uint32_t nxt_aux, int n) {
-  constexpr int kChunk = L::kChunk, kPF = Policy::kPF;
-  if (Policy::kFullUnroll) {
-#pragma unroll
-    for (int q = 0; q < kChunk; ++q) {
-      if (TAIL && q >= n) break;
-      p.consume(q, lds_f64(cur + q * 16), Policy::kAux ? lds_s32(cur_aux + q * 4) : 0, win[q % kPF]);
-      // refill the slot with the entry kPF ahead (it may sit in the next chunk's half of the ring);
-      // the last, partial chunk only looks ahead inside itself
-      if (TAIL && q + kPF >= n) continue;
-      const bool in_cur = q + kPF < kChunk;
-      const int at = in_cur ? q + kPF : q + kPF - kChunk;
-      int32_t ca, cb;
-      lds_coords((in_cur ? cur : nxt) + at * 16, ca, cb);
-      p.prefetch(ca, cb, win[q % kPF]);
+  if constexpr (policy_is_two_speed<Policy>::value) {
+    if (!TAIL && p.plain_chunk()) {
+      walk_chunk_unrolled<L, Policy, false, true>(p, win, cur, nxt, cur_aux, nxt_aux, n);
+      p.end_plain_chunk();
+    } else {
+      walk_chunk_rolled<L, Policy, TAIL>(p, win, cur, nxt, cur_aux, nxt_aux, n);
     }
+  } else if constexpr (Policy::kFullUnroll) {
+    // kRolledTail: the one partial chunk of a tile runs as a loop, so that only one copy of the unrolled body exists
+    if constexpr (TAIL && policy_rolls_tail<Policy>::value) walk_chunk_rolled<L, Policy, true>(p, win, cur, nxt, cur_aux, nxt_aux, n);
+    else walk_chunk_unrolled<L, Policy, TAIL, false>(p, win, cur, nxt, cur_aux, nxt_aux, n);
   } else {
-    // the two halves are adjacent in shared memory: position q + kPF of `cur` wraps into `nxt`
-    const uint32_t lo = cur < nxt ? cur : nxt, lo_aux = cur_aux < nxt_aux ? cur_aux : nxt_aux;
-    const int off = cur < nxt ? 0 : kChunk;
-#pragma unroll 1
-    for (int q0 = 0; q0 < (TAIL ? n : kChunk); q0 += kPF) {
-#pragma unroll
-      for (int u = 0; u < kPF; ++u) {
-        const int q = q0 + u;
-        if (TAIL && q >= n) break;
-        const int r = off + q;
-        p.consume(q, lds_f64(lo + r * 16), Policy::kAux ? lds_s32(lo_aux + r * 4) : 0, win[u]);
-        if (TAIL && q + kPF >= n) continue;
-        int32_t ca, cb;
-        lds_coords(lo + ((r + kPF) & (2 * kChunk - 1)) * 16, ca, cb);
-        p.prefetch(ca, cb, win[u]);
-      }
-    }
+    walk_chunk_rolled<L, Policy, TAIL>(p, win, cur, nxt, cur_aux, nxt_aux, n);
   }
 }
 
@@ -283,7 +331,8 @@ __device__ __forceinline__ void walk_tile(const L &ln, Policy &p, int32_t j0, in
   for (int u = 0; u < kPF; ++u) {
     int32_t ca, cb;
     lds_coords(smem + u * 16, ca, cb);
-    p.prefetch(ca, cb, win[u]);
+    if constexpr (policy_is_positional<Policy>::value) p.prefetch_at(u, true, ca, cb, win[u]);
+    else p.prefetch(ca, cb, win[u]);
   }
 
   int half = 0;
