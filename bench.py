@@ -21,8 +21,10 @@ same workload and prints the same JSON line with "impl": "reference".
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
+import re
 import statistics
 import subprocess
 import sys
@@ -80,6 +82,49 @@ def model(op, fmt, case, t):
             return n * 20 + dense, 3 * n * case.R
         return n * 12 + F * 8 + Sn * 8 + dense, 2 * n * case.R + 2 * F * case.R
     raise ValueError(op)
+
+
+def roofline_obj(nbytes, ms, peak, peak_kind, kernel, traffic=None, **extra):
+    """The roofline object of one kernel group: algorithmic bytes per call / CUDA-event time of the call."""
+    gbs = nbytes / ms / 1e6
+    out = {"kernel": kernel, "bound": "hbm", "achieved": round(gbs, 1), "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+           "frac": round(gbs / peak, 4), "frac_of_8000": round(gbs / NOMINAL_GBS, 4), "us_per_call": round(ms * 1e3, 1),
+           "algorithmic_bytes": int(nbytes), "traffic": traffic}
+    out.update(extra)
+    return out
+
+
+SPMM_SOURCES = ("contract_vec.cu", "spmm_heavy.cu", "spmm_heavy.cuh", "walk.cuh", "common.cuh")
+SPMM_PROFILE = os.path.join("profiles", "spmm_config2.md")
+
+
+def source_digest(names):
+    h = hashlib.sha256()
+    for n in names:
+        with open(os.path.join(ROOT, "paper_2102_05187_b200", "csrc", n), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def spmm_traffic_from_profile():
+    """DRAM bytes per comet_spmm call on the full workload, from the ncu summary under profiles/. The summary
+    records the digest of the kernel sources it was taken with; if the sources have changed since, the figure is
+    dropped (null) instead of being carried over to code it was not measured on."""
+    info = {"profile": SPMM_PROFILE, "source_digest": source_digest(SPMM_SOURCES)}
+    try:
+        text = open(os.path.join(ROOT, SPMM_PROFILE)).read()
+        traffic = float(re.search(r"traffic_bytes_per_call:\s*([0-9.eE+]+)", text).group(1))
+        digest = re.search(r"source_digest:\s*([0-9a-f]+)", text).group(1)
+        commit = re.search(r"commit:\s*([0-9a-f]+)", text)
+        info["profile_commit"] = commit.group(1) if commit else None
+        info["profile_source_digest"] = digest
+        if digest != info["source_digest"]:
+            info["stale"] = "kernel sources changed since the capture"
+            return None, info
+        return traffic, info
+    except Exception as e:                                  # no summary, or not in the expected form
+        info["stale"] = f"no usable profile summary ({type(e).__name__})"
+        return None, info
 
 
 def index_bytes(t):
@@ -170,7 +215,7 @@ def flush_l2(buf):
     buf.add_(1)
 
 
-def per_kernel(comet, handle, steps, warm, peak):
+def per_kernel(comet, handle, steps, warm, peak, peak_kind="measured"):
     """Every workload at full size: pack time and contraction time per op and format."""
     out = []
     l2buf = torch.zeros(192 << 20, dtype=torch.uint8, device="cuda")      # > 126 MB L2
@@ -251,6 +296,8 @@ def per_kernel(comet, handle, steps, warm, peak):
             "l2": "flushed between repetitions" if small else "inputs larger than L2",
             "pack_us_median": round(pmed * 1e3, 1), "pack_compulsory_bytes": pbytes,
             "pack_GBps": round(pbytes / pmed / 1e6, 1),
+            "roofline": roofline_obj(nbytes, med, peak, peak_kind, f"comet_{op} ({fmt}) on {case.name}"),
+            "pack_roofline": roofline_obj(pbytes, pmed, peak, peak_kind, f"comet_pack -> {fmt} on {case.name}"),
         })
         if op == "mttkrp" and fmt == "csf":
             # the two other modes of the SAME packed tensor (atomic accumulation, nothing re-packed)
@@ -266,6 +313,7 @@ def per_kernel(comet, handle, steps, warm, peak):
                     "frac_of_8000": round(nbytes / med / 1e6 / NOMINAL_GBS, 4),
                     "frac_of_peak": round(nbytes / med / 1e6 / peak, 4), "GFLOPs": round(flops / med / 1e6, 1),
                     "l2": "inputs larger than L2", "accumulation": "atomic adds (order not fixed)",
+                    "roofline": roofline_obj(nbytes, med, peak, peak_kind, f"comet_mttkrp mode {mode + 1} of the root-packed csf"),
                 })
                 del Fm, Am
         del T
@@ -283,6 +331,27 @@ def cpu_baseline_sample(case, frac_rows):
     v = case.val[keep].cpu().numpy()
     B = case.dense["B"].cpu().numpy()
     return (rows, case.dims[1]), [ci, cj], v, B
+
+
+def timed_cpu_baseline(dims, coords, val, B, reps=3):
+    """The oracle's SpMM loop with double accumulators (-O3 -march=native): one thread and all the threads this
+    process may use; mean of `reps` runs each. Bytes = the compulsory bytes of the SpMM on the sample."""
+    from oracle import timed_baseline
+    n = len(val)
+    nbytes = n * 12 + (dims[0] + 1) * 4 + B.size * 8 + dims[0] * B.shape[1] * 8
+    threads = timed_baseline.host_threads()
+    out = {"host_threads": threads, "reps": reps, "what": "SpMM only, COO loops with double accumulators, gcc -O3 -march=native"}
+    for label, t in (("threads_1", 1), ("threads_all", threads)):
+        timed_baseline.spmm(coords, val, dims, B, t)       # warm-up (page faults of the output)
+        ts = []
+        for _ in range(reps):
+            t0 = time.perf_counter()
+            timed_baseline.spmm(coords, val, dims, B, t)
+            ts.append(time.perf_counter() - t0)
+        mean = sum(ts) / len(ts)
+        out[label] = {"threads": t, "seconds": round(mean, 4), "GBps": round(nbytes / mean / 1e9, 3),
+                      "GFLOPs": round(2 * n * B.shape[1] / mean / 1e9, 2)}
+    return out
 
 
 def oracle_step(dims, coords, val, B):
@@ -390,14 +459,13 @@ def run_ours(args):
     A.free()
 
     spmm_med = statistics.median(spmm_ms)
-    roofline = {
-        "kernel": "comet_spmm (seg_gather_kernel<32,1,2> + carry fix-up)", "bound": "hbm",
-        "achieved": round(spmm_bytes / spmm_med / 1e6, 1), "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-        "frac": round(spmm_bytes / spmm_med / 1e6 / peak, 4), "frac_of_8000": round(spmm_bytes / spmm_med / 1e6 / NOMINAL_GBS, 4),
-        "us_per_launch": round(spmm_med * 1e3, 1), "algorithmic_bytes": spmm_bytes,
-        "traffic": TRAFFIC_SPMM_C2 if args.scale == 1.0 else None,
-        "note": "gather-bound: 64-column rows of B (537 MB, 4x the L2) are gathered nnz times, so DRAM traffic is 7.2x the algorithmic bytes and sits at the measured copy bandwidth",
-    }
+    traffic, traffic_info = spmm_traffic_from_profile() if args.scale == 1.0 else (None, {"stale": "not the full workload"})
+    roofline = roofline_obj(
+        spmm_bytes, spmm_med, peak, peak_kind,
+        "comet_spmm: seg_gather_kernel<32,1,2> with two CTA roles (long rows by column blocks of B | general tiles), "
+        "3 analysis kernels, 2 fix-ups", traffic=traffic, traffic_source=traffic_info,
+        note="gather-bound: the 64-column rows of B (537 MB, 4x the L2) are gathered nnz times; the long rows are "
+             "processed by column blocks so that their gathers hit L2, the short rows still pull their rows from DRAM")
 
     result = {
         "metric": "effective HBM GB/s of the SpMM path (compulsory bytes / time); per-kernel GB/s and GFLOP/s in `kernels`",
@@ -419,24 +487,21 @@ def run_ours(args):
     }
 
     if rank == 0 and not args.headline_only and world == 1:
-        result["kernels"] = per_kernel(comet, handle, max(3, min(args.steps, 25)), max(3, args.warmup), peak)
+        result["kernels"] = per_kernel(comet, handle, max(3, min(args.steps, 25)), max(3, args.warmup), peak, peak_kind)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        dims_s, coords_s, val_s, B_s = cpu_baseline_sample(case, args.cpu_rows)
+        dims_s, coords_s, val_s, B_s = cpu_baseline_sample(case, args.sample_rows)
         dt, nbytes = oracle_step(dims_s, coords_s, val_s, B_s)
         result["cpu_baseline"] = {"value": round(nbytes / dt / 1e9, 4), "unit": "GB/s", "cores": 1, "kind": "oracle",
-                                  "seconds": round(dt, 2),
+                                  "seconds": round(dt, 2), "host_cores": len(os.sched_getaffinity(0)),
                                   "sample": f"rows 0..{dims_s[0] - 1} of the workload ({len(val_s)} nnz), "
-                                            "oracle.pack + oracle.spmm, one thread"}
+                                            "oracle.pack + oracle.spmm (long double sums), one thread; the same sample "
+                                            "as --impl reference",
+                                  "timed_double": timed_cpu_baseline(dims_s, coords_s, val_s, B_s)}
     if rank == 0:
         print(json.dumps(result))
     if dist:
         dist.barrier()
         dist.destroy_process_group()
-
-
-# DRAM bytes per launch of the SpMM gather kernel at full size, from the ncu capture summarised in
-# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum).
-TRAFFIC_SPMM_C2 = 9.47e9
 
 
 # --------------------------------------------------------------------------------------------- reference arm
@@ -445,7 +510,7 @@ def run_reference(args):
     if rank != 0:
         return
     case = synth.make(2, scale=args.scale, device="cpu")
-    dims_s, coords_s, val_s, B_s = cpu_baseline_sample(case, args.ref_rows)
+    dims_s, coords_s, val_s, B_s = cpu_baseline_sample(case, args.sample_rows)
     for _ in range(args.warmup):
         oracle_step(dims_s, coords_s, val_s, B_s)
     times = []
@@ -465,7 +530,8 @@ def run_reference(args):
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": "configs[1] CSR SpMM (bounded row sample for the CPU oracle)",
                    "step": "oracle.pack(COO->CSR) + oracle.spmm", "nnz": len(val_s), "R": case.R, "seed": case.seed},
-        "cpu_baseline": {"value": round(value, 4), "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": round(value, 4), "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample,
+                         "host_cores": len(os.sched_getaffinity(0))},
         "e2e": {"value": round(value, 4), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
@@ -479,10 +545,17 @@ def main():
     ap.add_argument("--scale", type=float, default=1.0, help="workload scale (1.0 is the only reported one)")
     ap.add_argument("--headline-only", action="store_true", help="skip the per-kernel table")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-rows", type=float, default=0.25, help="fraction of rows in the CPU-baseline sample")
-    ap.add_argument("--ref-rows", type=float, default=1.0 / 16, help="fraction of rows per step of --impl reference")
+    ap.add_argument("--sample-rows", type=float, default=1.0 / 8,
+                    help="fraction of the rows in the CPU sample (the cpu_baseline leg and --impl reference use the same one)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # plain `python bench.py --gpus N`: start the N replicas (one process per GPU) and hand over to them
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(29500 + os.getpid() % 2000), os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd))
+    if "WORLD_SIZE" in os.environ and int(os.environ["WORLD_SIZE"]) != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} does not match the launcher's WORLD_SIZE={os.environ['WORLD_SIZE']}")
     if args.impl == "reference":
         run_reference(args)
     else:

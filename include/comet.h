@@ -10,8 +10,8 @@
  *   D  (dense)                pos = [dim] (1 entry), no crd; position = parent_position*dim + coordinate
  *   CU (compressed, unique)   crd = the distinct coordinates under each parent position, ascending;
  *                             pos has parents+1 entries: children of parent p are crd[pos[p] .. pos[p+1])
- *                             (Table 1: "for i from pos[m] to pos[m+1] { idx = crd[i] }", m = the
- *                             position produced by the level above, 0 at the first level)
+ *                             (the loop form of Table 1: pos is indexed by the position that the level above
+ *                             produced, 0 at the first level, and brackets that parent's range of crd)
  *   CN (compressed, nonunique) first level only: crd = every entry's coordinate, pos = [0, nnz]
  *   S  (singleton)            crd[p] = coordinate of the entry at parent position p, no pos
  *
@@ -24,9 +24,14 @@
  *     OVERWRITTEN (C = A.B, not +=); rows / fibers without a stored entry become +0.0.
  *   - Dense operands are row-major with an explicit leading dimension in elements.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream). Contractions
- *     are asynchronous on that stream and never synchronise; comet_pack and the *_symbolic calls
- *     synchronise the stream once to learn data-dependent sizes.
- *   - A handle caches scratch memory and may be used from one stream at a time.
+ *     are asynchronous on that stream; comet_pack and the *_symbolic calls synchronise the stream
+ *     once to learn data-dependent sizes. Exceptions, all on the host side of a contraction call:
+ *     the handle's scratch grows on demand, and the call that grows it waits for the stream before the
+ *     old buffer is released (so the first call, or the first larger one, may synchronise);
+ *     comet_spmv / comet_spmm on a [CN,S] matrix allocate and release a row index on every call;
+ *     a call on another stream than the handle's previous call first waits for that previous stream.
+ *   - A handle caches scratch memory and device counters: one call at a time. Calls on one handle
+ *     from several host threads, or overlapping on the GPU, are not supported (use a handle each).
  *   - Errors are return codes; nothing aborts, throws or traps. Errors detectable on the host are
  *     returned before anything is launched.
  *   - Limits: nnz, every extent and every pos value must be < 2^31 - 1 (int32 indices); leading
@@ -66,6 +71,18 @@ typedef enum {
 } comet_status_t;
 
 #define COMET_MAX_ORDER 4
+
+/* Tuning variables read from the environment (for experiments and tests; the defaults are the measured best):
+ *   COMET_TILE_ITEMS=n          items (leaf entries + segment ends) per tile of the matrix-operand kernels
+ *   COMET_SEG_DOT_KERNEL=name   SpMV/TTV kernel: resident | stream | stream2 (default: chosen by size)
+ *   COMET_STREAM_SPAN=n         entries per span of the SpMV/TTV stream kernels (multiple of 128)
+ *   COMET_PACK_CSR=1|0          forces / forbids the histogram CSR packing of comet_pack_ex (COMET_PACK_CSR_HISTOGRAM)
+ *   COMET_SEG_PARTITION=0       matrix-operand kernels search their tile boundaries themselves (no pre-pass)
+ *   COMET_CSF_FORM=fold|expand  root-mode CSF MTTKRP: per-fiber or per-entry form (default: by mean fiber length)
+ *   COMET_SPMM_LONG_ROWS=0      comet_spmm without the long-row path; COMET_SPMM_LONG_ROW, _LONG_TILE, _PIECE,
+ *                               _BLOCK_MB, _BLOCKS, _LONG_CTAS, _LONG_MIN_NNZ, _LONG_MIN_B_MB: its threshold
+ *                               (entries), tile and piece sizes, block size / count of B, CTAs of the long-row
+ *                               role, and the matrix / operand sizes from which it switches itself on */
 
 /* The sparse tensor descriptor (a plain struct the caller may also fill in by hand for arrays it
  * built itself; run comet_validate on such a tensor before contracting it). */
@@ -249,7 +266,8 @@ comet_status_t comet_reorder(comet_handle_t handle, int32_t order, const int64_t
  * scratch from an allocator; this entry point needs neither. It calls no cudaMalloc, cudaFree or
  * any other allocating routine, directly or through a library.
  *
- * Same result as comet_spmv for A = [D,CU] with fp64 values (other formats or fp32: COMET_ERR_UNSUPPORTED_FORMAT). The caller
+ * The same product as comet_spmv for A = [D,CU] with fp64 values, equal to it up to rounding (the two tile the
+ * matrix differently); other formats or fp32: COMET_ERR_UNSUPPORTED_FORMAT. The caller
  * still passes the inputs and the output (device pointers, y has dims[mode_order[0]] entries and is
  * fully overwritten). The per-tile carry slots live in a fixed 768 KiB device array that is part of
  * the library image: every GPU that loads the library holds it until the process exits.

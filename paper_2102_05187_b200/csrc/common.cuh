@@ -21,6 +21,9 @@ struct Context {
   int32_t *h_pinned;                      // small pinned buffer for device->host size reads
   int32_t *d_status;                      // device words written by checking kernels
   int64_t launches;                       // kernels launched through this handle (for accounting)
+  cudaStream_t last_stream;               // stream of the latest call that used the scratch or the counters
+  bool has_last_stream;
+  bool counters_dirty;                    // a CUDA call failed: the device counters may not be back at zero
 };
 
 // Grows the cached scratch buffer to at least `bytes` and returns it (NULL on allocation failure).

@@ -13,7 +13,7 @@ static void *default_alloc(void *, size_t bytes, void *) {
 static void default_free(void *, void *p, void *) { if (p) cudaFree(p); }
 
 comet_status_t cuda_fail(Context *ctx, cudaError_t e) {
-  if (ctx) ctx->last_cuda_error = (int)e;
+  if (ctx) { ctx->last_cuda_error = (int)e; ctx->counters_dirty = true; }
   cudaGetLastError();   // clear the sticky-less error state
   return COMET_ERR_CUDA;
 }
@@ -25,7 +25,23 @@ void ctx_free(Context *ctx, void *p, cudaStream_t stream) {
   if (p) ctx->allocator.free(ctx->allocator.ctx, p, (void *)stream);
 }
 
+// The scratch and the device counters (words 32..35 of d_status, which the kernels that use them leave at zero)
+// belong to one call at a time. Two things could break that silently and are made safe here, where every
+// contraction passes: a call on ANOTHER stream than the handle's previous call waits for that stream first (its
+// kernels may still be using both), and after any failed CUDA call the counters are cleared before the next use
+// (a kernel that did not run to its end may not have put them back).
+static void ctx_enter(Context *ctx, cudaStream_t stream) {
+  if (ctx->has_last_stream && ctx->last_stream != stream) cudaStreamSynchronize(ctx->last_stream);
+  ctx->last_stream = stream;
+  ctx->has_last_stream = true;
+  if (ctx->counters_dirty && ctx->d_status) {
+    if (cudaMemsetAsync(ctx->d_status + 32, 0, 4 * sizeof(int32_t), stream) == cudaSuccess) ctx->counters_dirty = false;
+    else cudaGetLastError();
+  }
+}
+
 void *scratch_get(Context *ctx, size_t bytes, cudaStream_t stream) {
+  ctx_enter(ctx, stream);
   if (bytes <= ctx->scratch_bytes && ctx->scratch) return ctx->scratch;
   if (ctx->scratch) {
     // work queued on the stream may still read the old buffer
@@ -58,6 +74,9 @@ extern "C" comet_status_t comet_create(comet_handle_t *handle, const comet_alloc
   else ctx->allocator = comet_allocator_t{comet::default_alloc, comet::default_free, nullptr};
   ctx->device = dev;
   ctx->last_cuda_error = 0;
+  ctx->has_last_stream = false;
+  ctx->last_stream = nullptr;
+  ctx->counters_dirty = false;
   ctx->launches = 0;
   ctx->scratch = nullptr;
   ctx->scratch_bytes = 0;

@@ -831,10 +831,10 @@ extern "C" comet_status_t comet_spmv_static(const comet_sptensor_t *A, const voi
   const int m0 = A->mode_order[0], m1 = A->mode_order[1];
   if (!((m0 == 0 && m1 == 1) || (m0 == 1 && m1 == 0))) return COMET_ERR_INVALID_ARG;
   const int64_t M = A->dims[m0], N = A->nnz;
-  if (M < 0 || N < 0 || !A->pos[1] || A->pos_len[1] != M + 1 || (N > 0 && (!A->crd[1] || !A->val)))
-    return COMET_ERR_INVALID_ARG;
-  if ((reinterpret_cast<uintptr_t>(x) & 7) || (reinterpret_cast<uintptr_t>(y) & 7)) return COMET_ERR_MISALIGNED;
+  if (M < 0 || N < 0) return COMET_ERR_INVALID_ARG;
   if (M + N > kStaticMaxItems) return COMET_ERR_WORKSPACE;      // beyond the fixed scratch: use comet_spmv
+  if (!A->pos[1] || A->pos_len[1] != M + 1 || (N > 0 && (!A->crd[1] || !A->val))) return COMET_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(x) & 7) || (reinterpret_cast<uintptr_t>(y) & 7)) return COMET_ERR_MISALIGNED;
   if (M == 0) return COMET_OK;
 
   void *scratch = nullptr;

@@ -40,6 +40,7 @@ struct SegGatherArgs {
   double *carry_val;        // num_tiles x carry_ld
   int32_t *carry_seg;       // num_tiles: segment the carry belongs to, -1 if none
   int32_t carry_ld;
+  const int32_t *part;      // num_tiles + 1 merge-path splits (segments in front of each tile boundary), or NULL
   int32_t skip_len;         // > 0: segments of at least this many entries are somebody else's (the long-row
                             //      path of SpMM): neither walked nor stored here. Never below tile_items.
 };
@@ -141,8 +142,10 @@ seg_gather_kernel(const SegGatherArgs a, const HeavyArgs h) {
   const int64_t total = a.M + a.N;
   const int64_t d0 = tile * a.tile_items;
   const int64_t d1 = (d0 + a.tile_items < total) ? d0 + a.tile_items : total;
-  int64_t i0 = merge_path_segments_coop<LPN>(a.seg_end, a.M, a.N, d0, ln.g, ln.mask);
-  const int64_t i1 = merge_path_segments_coop<LPN>(a.seg_end, a.M, a.N, d1, ln.g, ln.mask);
+  // the splits come from the partition kernel when there is one: a worker is sequential, and two dependent
+  // searches at the head of every tile are a sizeable part of a short tile
+  int64_t i0 = a.part ? (int64_t)__ldg(a.part + tile) : merge_path_segments_coop<LPN>(a.seg_end, a.M, a.N, d0, ln.g, ln.mask);
+  const int64_t i1 = a.part ? (int64_t)__ldg(a.part + tile + 1) : merge_path_segments_coop<LPN>(a.seg_end, a.M, a.N, d1, ln.g, ln.mask);
   int32_t j0 = (int32_t)(d0 - i0), j1 = (int32_t)(d1 - i1);
   if (a.skip_len > 0) {
     // A long segment holds more entries than a tile, so it can only be the one open at the tile's start or the
@@ -173,6 +176,17 @@ seg_gather_kernel(const SegGatherArgs a, const HeavyArgs h) {
   const bool carry = seg < a.M && j1 > p.last_flush;     // leaf entries of a segment that ends in a later tile
   if (ln.g == 0) a.carry_seg[tile] = carry ? (int32_t)seg : -1;
   if (carry) ln.store_carry(a.carry_val + tile * a.carry_ld + ln.col0, p.acc);
+}
+
+// Merge-path split at every tile boundary, a thread per boundary.
+__global__ void __launch_bounds__(kBlockThreads) seg_partition_kernel(const int32_t *__restrict__ seg_end, int64_t M, int64_t N,
+                                                                      int32_t tile_items, int64_t num_tiles,
+                                                                      int32_t *__restrict__ part) {
+  const int64_t t = (int64_t)blockIdx.x * kBlockThreads + threadIdx.x;
+  if (t > num_tiles) return;
+  const int64_t total = M + N;
+  const int64_t d = t * tile_items < total ? t * tile_items : total;
+  part[t] = (int32_t)merge_path_segments(seg_end, M, N, d);
 }
 
 // Adds the carries onto the stored rows. Tiles that stopped inside the same segment are consecutive;
@@ -286,10 +300,19 @@ static comet_status_t launch_one(Context *ctx, SegGatherArgs a, HeavyArgs *heavy
   if (kHeavyShape<T, LPN, CPL, VEC> && heavy && !a.out_row)
     heavy_bytes = spmm_heavy_plan(sizeof(T) == 4 ? COMET_F32 : COMET_F64, a.M, a.N, heavy->cols, a.B, a.ldb, a.R, a.C, a.ldc,
                                   a.tile_items, &h);
-  char *scratch = (char *)scratch_get(ctx, heavy_bytes + carry_bytes(a.num_tiles, a.carry_ld), stream);
+  static const bool use_part = !(getenv("COMET_SEG_PARTITION") && atoi(getenv("COMET_SEG_PARTITION")) == 0);
+  const size_t part_bytes = use_part && a.num_tiles >= 1024 ? align_up((size_t)(a.num_tiles + 1) * sizeof(int32_t), 256) : 0;
+  char *scratch = (char *)scratch_get(ctx, heavy_bytes + carry_bytes(a.num_tiles, a.carry_ld) + part_bytes, stream);
   if (!scratch) return COMET_ERR_ALLOC;
   a.carry_val = (double *)(scratch + heavy_bytes);
   a.carry_seg = (int32_t *)(scratch + heavy_bytes + val_bytes);
+  if (part_bytes) {
+    int32_t *part = (int32_t *)(scratch + heavy_bytes + carry_bytes(a.num_tiles, a.carry_ld));
+    seg_partition_kernel<<<(unsigned)ceil_div(a.num_tiles + 1, kBlockThreads), kBlockThreads, 0, stream>>>(a.seg_end, a.M, a.N,
+                                                                                                         a.tile_items, a.num_tiles, part);
+    COMET_LAUNCH_CHECK(ctx);
+    a.part = part;
+  }
   const int64_t blocks = ceil_div(a.num_tiles, WORKERS);
   comet_status_t st;
   if constexpr (kHeavyShape<T, LPN, CPL, VEC>) {

@@ -330,3 +330,17 @@ def test_order_n_mttkrp_is_the_three_order_function_on_three_order_input(mode):
     a3, n3 = oracle.mttkrp(c, v, dims, mode, F)
     an, nn = oracle.mttkrp_n(c, v, dims, mode, F)
     assert np.array_equal(a3, an) and np.array_equal(n3, nn)
+
+
+def test_timed_baseline_agrees_with_the_parity_oracle():
+    """The benchmark's timed CPU loop (double accumulators, 1 and several threads) against the long-double oracle."""
+    from oracle import timed_baseline
+    dims, R = (300, 200), 16
+    coords, val = synth.random_coo(dims, 5000, 21)
+    c, v = [x.numpy() for x in coords], val.numpy()
+    B = synth.random_dense((dims[1], R), 21).numpy()
+    want, norm = oracle.spmm(c, v, dims, B)
+    for threads in (1, 3):
+        got = timed_baseline.spmm(c, v, dims, B, threads)
+        assert np.all(np.abs(got - want) <= 1e-12 * norm)
+    assert timed_baseline.host_threads() >= 1
