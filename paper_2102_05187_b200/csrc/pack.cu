@@ -648,7 +648,7 @@ extern "C" comet_status_t comet_pack_ex(comet_handle_t handle, int32_t order, co
   int64_t n = nnz;                     // entries the level pass sees (fewer after duplicates are merged)
   const int64_t sort_tiles = ceil_div(n > 0 ? n : 1, kSortTile);
   int64_t level_tiles = ceil_div(n > 0 ? n : 1, kLevelTile);
-  const int64_t table_len = 256 * sort_tiles;
+  const int64_t table_len = radix_sort_table_words(n);
   const int64_t counts_len = (int64_t)COMET_MAX_ORDER * level_tiles;
 
   TempBlocks tmp(ctx, s);
