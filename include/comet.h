@@ -128,11 +128,19 @@ int64_t comet_kernel_launches(comet_handle_t handle);
  *   h_coo_crd[order]    HOST array of DEVICE pointers, one int32[nnz] coordinate array per mode
  *   coo_val             DEVICE, nnz values, copied bitwise into leaf order
  *   h_mode_order[order] a permutation of 0..order-1; h_attr[order] one comet_attr_t per level
- * Supported attribute tuples: [CN,S,...,S], [CU,...,CU], [D,CU,...,CU] (orders 2..4), provided the
+ * Supported attribute tuples: [CN,S,...,S], [CU,...,CU], [D,CU,...,CU] (orders 2..4), and [D,S] for a matrix, which
+ * asks for ELLPACK (below), provided the
  * coordinate bit widths (ceil(log2(extent)) per mode) sum to <= 63. Input order is arbitrary; duplicates and out-of-range
  * coordinates are detected on the device and reported (COMET_ERR_DUPLICATE_COORD,
  * COMET_ERR_COORD_OUT_OF_RANGE); `out` is then left zeroed. On success `out` owns its arrays
- * (allocated through the handle's allocator) until comet_sptensor_free. Synchronises `stream` once. */
+ * (allocated through the handle's allocator) until comet_sptensor_free. Synchronises `stream` once.  *
+ * ELLPACK (named in the Tensor Storage Format section among the formats the four attributes compose; the paper
+ * does not spell the composition out, this is the reading used): order 2 with h_attr = {COMET_D, COMET_S} gives a
+ * descriptor of THREE levels [D, D, S]: the rows (dense), K slots per row (dense; listed as a third "mode" of
+ * extent K = the longest row: dims[2] = K, mode_order = {row mode, 2, column mode}), and one singleton column
+ * coordinate per slot. pos[0] = [rows], pos[1] = [K], crd[2] and val hold rows * K entries (nnz = rows * K): a row's
+ * entries first, columns ascending, then padding with column -1 and value 0. comet_spmv, comet_spmm and
+ * comet_elementwise_mul accept it. Synchronises `stream` twice more than the CSR packing it goes through. */
 comet_status_t comet_pack(comet_handle_t handle, int32_t order, const int64_t *h_dims, int64_t nnz,
                           const int32_t *const *h_coo_crd, const void *coo_val, comet_dtype_t dtype,
                           const int32_t *h_mode_order, const int32_t *h_attr, void *stream,
@@ -256,6 +264,17 @@ comet_status_t comet_mttkrp(comet_handle_t handle, const comet_sptensor_t *X, in
 comet_status_t comet_reorder(comet_handle_t handle, int32_t order, const int64_t *h_dims, int64_t nnz,
                              const int32_t *const *h_coo_crd, int32_t iterations, int32_t *const *h_new_label,
                              void *stream);
+
+/* Element-wise product with a dense operand (Language section: `*` between operands whose indices are not
+ * contraction indices is element-wise): C = A .* B, sparse with A's structure. out_val[p] = val[p] * B[coordinates
+ * of A's leaf position p]; out_val (device, A->nnz values of A's dtype, caller-allocated, may be A->val itself)
+ * is the value array of a tensor that otherwise shares A's level arrays. B is dense over A's modes: element
+ * (i_0, i_1, ...) in MODE order (not storage order) sits at B[sum_m i_m * h_strides[m]] (h_strides: host array,
+ * one non-negative element stride per mode). Any attribute tuple the descriptor may hold, of order 1..4, and
+ * ELLPACK (two strides; padding slots give 0). Asynchronous on `stream`; a caller-built A is trusted as in the
+ * contractions. */
+comet_status_t comet_elementwise_mul(comet_handle_t handle, const comet_sptensor_t *A, const void *B,
+                                     const int64_t *h_strides, void *out_val, void *stream);
 
 /* CSR SpMV without any allocation (the paper has no counterpart; this exists for deployment only).
  *

@@ -5,5 +5,5 @@ TTV, TTM and MTTKRP as hand-written sm_100a CUDA kernels behind a C ABI (include
 This package is the thin Python binding of that library; see `binding` for the calls.
 """
 from .binding import (D, CU, CN, S, CometError, Handle, SpTensor, default_handle, load_library, pack, validate,  # noqa: F401
-                      spmv, spmm, spmm_from_host, ttv_symbolic, ttv, ttm_symbolic, ttm, mttkrp, reorder, EXPORTS,
-                      LIB_PATH)
+                      spmv, spmm, elementwise_mul, spmm_from_host, ttv_symbolic, ttv, ttm_symbolic, ttm, mttkrp, reorder,
+                      EXPORTS, LIB_PATH)

@@ -51,6 +51,7 @@ EXPORTS = [
     "comet_pack",
     "comet_sptensor_free", "comet_validate", "comet_spmv", "comet_spmm", "comet_ttv_symbolic", "comet_ttv",
     "comet_ttm_symbolic", "comet_ttm", "comet_mttkrp", "comet_spmv_static", "comet_pack_ex", "comet_ttm_symbolic_ex", "comet_reorder",
+    "comet_elementwise_mul",
 ]
 
 
@@ -344,6 +345,24 @@ def spmm(A: SpTensor, B: torch.Tensor, out: torch.Tensor | None = None) -> torch
                                  _ptr(out), C.c_int64(out.stride(0)), _stream_ptr())
     A.handle.check(st, "comet_spmm")
     return out
+
+
+def elementwise_mul(A: SpTensor, B: torch.Tensor, out_val: torch.Tensor | None = None) -> SpTensor:
+    """C = A .* B for a dense B over A's modes (any strides): a tensor that shares A's level arrays (A must
+    outlive it) and owns its values."""
+    _require_cuda(B)
+    dt = _same_dtype(A, B, out_val)
+    modes = 2 if A.attr == (D, D, S) else A.c.order
+    assert B.dim() == modes
+    if out_val is None:
+        out_val = torch.empty(A.c.nnz, dtype=dt, device=B.device)
+    strides = (C.c_int64 * MAX_ORDER)(*[int(x) for x in B.stride()], *([0] * (MAX_ORDER - modes)))
+    st = A.handle.lib.comet_elementwise_mul(A.handle._h, C.byref(A.c), _ptr(B), strides, _ptr(out_val), _stream_ptr())
+    A.handle.check(st, "comet_elementwise_mul")
+    s = SpTensorStruct.from_buffer_copy(A.c)
+    s.val = out_val.data_ptr() if out_val.numel() else 0
+    s.owner = None
+    return SpTensor(A.handle, s, keep=[A, out_val])
 
 
 def ttv_symbolic(X: SpTensor, mode: int, out_attr=None) -> SpTensor:

@@ -141,6 +141,12 @@ extern "C" comet_status_t comet_sptensor_free(comet_handle_t handle, comet_spten
 extern "C" comet_status_t comet_spmv(comet_handle_t handle, const comet_sptensor_t *A, const void *x, void *y,
                                      void *stream) {
   if (!handle || !x || !y) return COMET_ERR_INVALID_ARG;
+  if (is_ellpack(A)) {
+    const comet_status_t es = ell_check(A);
+    if (es != COMET_OK) return es;
+    if (misaligned(x, A->dtype) || misaligned(y, A->dtype)) return COMET_ERR_MISALIGNED;
+    return ell_spmv(reinterpret_cast<Context *>(handle), A, x, y, (cudaStream_t)stream);
+  }
   comet_status_t st = check_tensor(A, 2);
   if (st != COMET_OK) return st;
   if (misaligned(x, A->dtype) || misaligned(y, A->dtype)) return COMET_ERR_MISALIGNED;
@@ -167,6 +173,12 @@ extern "C" comet_status_t comet_spmv(comet_handle_t handle, const comet_sptensor
 extern "C" comet_status_t comet_spmm(comet_handle_t handle, const comet_sptensor_t *A, const void *B, int64_t R,
                                      int64_t ldb, void *C, int64_t ldc, void *stream) {
   if (!handle || !B || !C || R < 1 || ldb < R || ldc < R) return COMET_ERR_INVALID_ARG;
+  if (is_ellpack(A)) {
+    const comet_status_t es = ell_check(A);
+    if (es != COMET_OK) return es;
+    if (misaligned(B, A->dtype) || misaligned(C, A->dtype)) return COMET_ERR_MISALIGNED;
+    return ell_spmm(reinterpret_cast<Context *>(handle), A, B, ldb, R, C, ldc, (cudaStream_t)stream);
+  }
   comet_status_t st = check_tensor(A, 2);
   if (st != COMET_OK) return st;
   if (misaligned(B, A->dtype) || misaligned(C, A->dtype)) return COMET_ERR_MISALIGNED;
@@ -520,6 +532,26 @@ extern "C" comet_status_t comet_ttm(comet_handle_t handle, const comet_sptensor_
   Context *ctx = reinterpret_cast<Context *>(handle);
   return seg_gather(ctx, X->dtype, fiber_pos + 1, X->crd[last], X->val, F, X->nnz, U, ldu, R, Y->val, R, nullptr, F, 0,
                     (cudaStream_t)stream);
+}
+
+// ------------------------------------------------------------------------------------------ element-wise
+extern "C" comet_status_t comet_elementwise_mul(comet_handle_t handle, const comet_sptensor_t *A, const void *B,
+                                                const int64_t *h_strides, void *out_val, void *stream) {
+  if (!handle || !A || !h_strides) return COMET_ERR_INVALID_ARG;
+  comet_status_t st;
+  int modes = A->order;
+  if (is_ellpack(A)) {
+    st = ell_check(A);
+    modes = 2;
+  } else {
+    st = check_tensor(A, A->order);
+  }
+  if (st != COMET_OK) return st;
+  if (A->nnz > 0 && (!B || !out_val)) return COMET_ERR_INVALID_ARG;
+  if (misaligned(B, A->dtype) || misaligned(out_val, A->dtype)) return COMET_ERR_MISALIGNED;
+  for (int m = 0; m < modes; ++m)
+    if (h_strides[m] < 0) return COMET_ERR_INVALID_ARG;
+  return elementwise_mul(reinterpret_cast<Context *>(handle), A, B, h_strides, out_val, (cudaStream_t)stream);
 }
 
 // ------------------------------------------------------------------------------------------ MTTKRP

@@ -67,6 +67,19 @@ comet_status_t pack_csr_fast(Context *ctx, int dtype, const int32_t *row, const 
                              int64_t rows, int64_t cols, int32_t *pos_out, int32_t *crd_out, void *val_out,
                              int *fallback, cudaStream_t s);
 
+// ELLPACK [D,D,S] (ellpack.cu): conversion from a CSR tensor (arrays allocated into `owner`; synchronises), the
+// descriptor test and the two products.
+comet_status_t ell_from_csr(Context *ctx, const comet_sptensor_t *csr, void *owner, comet_sptensor_t *out, cudaStream_t s);
+bool is_ellpack(const comet_sptensor_t *A);
+comet_status_t ell_check(const comet_sptensor_t *A);
+comet_status_t ell_spmv(Context *ctx, const comet_sptensor_t *A, const void *x, void *y, cudaStream_t s);
+comet_status_t ell_spmm(Context *ctx, const comet_sptensor_t *A, const void *B, int64_t ldb, int64_t R, void *C, int64_t ldc,
+                        cudaStream_t s);
+
+// out[p] = val[p] * B[coordinates of leaf position p] (elementwise.cu); h_strides: element stride of every MODE in B.
+comet_status_t elementwise_mul(Context *ctx, const comet_sptensor_t *A, const void *B, const int64_t *h_strides, void *out,
+                               cudaStream_t s);
+
 int32_t choose_tile_items(int64_t total_items, int workers_per_block);
 
 // Block list of a library-owned tensor (what comet_sptensor_free releases).

@@ -575,10 +575,29 @@ extern "C" comet_status_t comet_pack_ex(comet_handle_t handle, int32_t order, co
     if (nnz > 0 && !h_coo_crd[l]) return COMET_ERR_INVALID_ARG;
   }
   if (nnz > 0 && !coo_val) return COMET_ERR_INVALID_ARG;
-  if (!supported_attrs(order, h_attr)) return COMET_ERR_UNSUPPORTED_FORMAT;
-
   Context *ctx = reinterpret_cast<Context *>(handle);
   cudaStream_t s = (cudaStream_t)stream;
+
+  // A singleton level under a dense one asks for ELLPACK: packed as CSR first, then the rows are spread over
+  // K slots each (ellpack.cu). The result has three levels, [D, D, S].
+  if (order == 2 && h_attr[0] == COMET_D && h_attr[1] == COMET_S) {
+    const int32_t csr_attr[2] = {COMET_D, COMET_CU};
+    comet_sptensor_t csr;
+    comet_status_t st = comet_pack_ex(handle, 2, h_dims, nnz, h_coo_crd, coo_val, dtype, h_mode_order, csr_attr,
+                                      flags & ~(uint32_t)COMET_PACK_CSR_HISTOGRAM, stream, &csr);
+    if (st != COMET_OK) return st;
+    void *owner = owner_new();
+    st = owner ? ell_from_csr(ctx, &csr, owner, out, s) : COMET_ERR_ALLOC;
+    comet_sptensor_free(handle, &csr, stream);
+    if (st != COMET_OK) {
+      if (owner) owner_release(ctx, owner, s);
+      memset(out, 0, sizeof(*out));
+      return st;
+    }
+    out->owner = owner;
+    return COMET_OK;
+  }
+  if (!supported_attrs(order, h_attr)) return COMET_ERR_UNSUPPORTED_FORMAT;
 
   // CSR of a matrix with a dense row level: the row structure is a histogram, so the full sort is not needed
   // (pack_csr.cu). On request only (COMET_PACK_CSR_HISTOGRAM): it wins on matrices whose rows are of similar
