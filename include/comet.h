@@ -192,7 +192,8 @@ comet_status_t comet_spmm(comet_handle_t handle, const comet_sptensor_t *A, cons
                           void *C, int64_t ldc, void *stream);
 
 /* TTV  Y = X x_n v  (SpTTV definition; `mode` = n, 0-based, must be the mode of X's LAST level).
- * X: 3 levels, [CU,CU,CU] (CSF) or [CN,S,S] (sorted COO), or 4 levels, [CU,CU,CU,CU] (CSF). The result
+ * X: 3 levels, [CU,CU,CU] (CSF) or [CN,S,S] (sorted COO), or 4 levels, [CU,CU,CU,CU] (CSF) or [CN,S,S,S] (sorted
+ * COO; its symbolic call derives the compressed levels by packing the entries once more). The result
  * is sparse, one order lower: comet_ttv_symbolic builds its structure over the kept modes in storage
  * order (Y's modes are renumbered 0..order-2) with h_out_attr[order-1] level attributes: {D,CU} (CSR) or
  * {CU,CU} (DCSR) for a 3-order X, {CU,CU,CU} (CSF) for a 4-order X; values are then (re)computed by
@@ -254,7 +255,7 @@ comet_status_t comet_mttkrp(comet_handle_t handle, const comet_sptensor_t *X, in
  * indices are re-numbered in ascending key order, ties in the order of their current numbers. One iteration is
  * a step for every mode in turn.
  *   h_coo_crd[order]    HOST array of DEVICE pointers: int32[nnz] coordinates per mode (COO, any order;
- *                       duplicates allowed); orders 2 and 3
+ *                       duplicates allowed); orders 2 to 4
  *   h_new_label[order]  HOST array of DEVICE pointers: int32[dims[m]] OUT, new_label[m][x] = the new number of
  *                       original index x (a permutation of 0..dims[m]-1; the identity for iterations = 0)
  * The caller applies it: coordinates become new_label[m][c], row j of a dense operand indexed by mode m moves to

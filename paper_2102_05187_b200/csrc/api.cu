@@ -217,7 +217,8 @@ static comet_status_t check_last_mode(const comet_sptensor_t *X, int32_t mode) {
   if (mode < 0 || mode >= X->order) return COMET_ERR_INVALID_ARG;
   bool csf = true;
   for (int l = 0; l < X->order; ++l) csf = csf && X->attr[l] == COMET_CU;
-  if (!csf && !is_fmt(X, 3, COMET_CN, COMET_S, COMET_S)) return COMET_ERR_UNSUPPORTED_FORMAT;
+  const bool coo4 = X->order == 4 && X->attr[0] == COMET_CN && X->attr[1] == COMET_S && X->attr[2] == COMET_S && X->attr[3] == COMET_S;
+  if (!csf && !coo4 && !is_fmt(X, 3, COMET_CN, COMET_S, COMET_S)) return COMET_ERR_UNSUPPORTED_FORMAT;
   if (X->mode_order[X->order - 1] != mode) return COMET_ERR_UNSUPPORTED_FORMAT;   // re-pack with the contracted mode last
   return COMET_OK;
 }
@@ -261,15 +262,43 @@ __global__ void coo_levels_kernel(const int32_t *__restrict__ c0, const int32_t 
 struct CooAsCsf {
   comet_sptensor_t t;       // CSF-shaped view: derived upper levels + the COO tensor's leaf arrays
   int32_t *pos2;            // fiber boundaries (F + 1); handed to the result, which the numeric call reads
-  void *temps[4];           // pos0, crd0, pos1, crd1 of the view
+  void *temps[6];           // the upper levels of the view: pos0, crd0, pos1, crd1 (and pos2, crd2 for order 4)
 };
 
 static void coo_view_release(Context *ctx, CooAsCsf *v, bool keep_pos2, cudaStream_t s) {
-  for (int i = 0; i < 4; ++i) if (v->temps[i]) ctx_free(ctx, v->temps[i], s);
+  for (int i = 0; i < 6; ++i) if (v->temps[i]) ctx_free(ctx, v->temps[i], s);
   if (!keep_pos2 && v->pos2) ctx_free(ctx, v->pos2, s);
 }
 
+// 4-order sorted COO [CN,S,S,S]: the three upper CSF levels come from the packing itself (the entries are sorted
+// once more, which a symbolic call can afford); the leaf level stays the COO tensor's own last coordinate array
+// and values, whose order is the packed order.
+static comet_status_t coo4_as_csf(Context *ctx, const comet_sptensor_t *X, cudaStream_t s, CooAsCsf *v) {
+  memset(v, 0, sizeof(*v));
+  const int32_t *by_mode[4];
+  for (int l = 0; l < 4; ++l) by_mode[X->mode_order[l]] = X->crd[l];
+  const int32_t attr[4] = {COMET_CU, COMET_CU, COMET_CU, COMET_CU};
+  comet_sptensor_t P;
+  comet_status_t st = comet_pack(reinterpret_cast<comet_handle_t>(ctx), 4, X->dims, X->nnz, by_mode, X->val,
+                                 (comet_dtype_t)X->dtype, X->mode_order, attr, (void *)s, &P);
+  if (st != COMET_OK) return st;
+  // take the level arrays over from the packed tensor; its leaf coordinates and values are not needed
+  Owner *po = static_cast<Owner *>(P.owner);
+  for (int b = 0; b < po->count; ++b)
+    if (po->blocks[b] == (void *)P.crd[3] || po->blocks[b] == P.val) ctx_free(ctx, po->blocks[b], s);
+  delete po;
+  v->temps[0] = P.pos[0]; v->temps[1] = P.crd[0]; v->temps[2] = P.pos[1]; v->temps[3] = P.crd[1];
+  v->temps[4] = P.pos[2]; v->temps[5] = P.crd[2];
+  v->pos2 = P.pos[3];
+  v->t = P;
+  v->t.owner = nullptr;
+  v->t.crd[3] = X->crd[3]; v->t.crd_len[3] = X->nnz;
+  v->t.val = X->val; v->t.nnz = X->nnz;
+  return COMET_OK;
+}
+
 static comet_status_t coo_as_csf(Context *ctx, const comet_sptensor_t *X, cudaStream_t s, CooAsCsf *v) {
+  if (X->order == 4) return coo4_as_csf(ctx, X, s, v);
   memset(v, 0, sizeof(*v));
   const int64_t n = X->nnz;
   int64_t S = 0, F = 0;
@@ -330,8 +359,18 @@ static comet_status_t coo_as_csf(Context *ctx, const comet_sptensor_t *X, cudaSt
 // levels) holds pos2, owned by Y. The numeric call finds them there.
 static void stash_fiber_pos(comet_sptensor_t *Y, Owner *o, int slot, CooAsCsf *v) {
   o->blocks[o->count++] = v->pos2;
-  Y->pos[slot] = v->pos2;
-  Y->pos_len[slot] = v->t.pos_len[2];
+  if (slot < COMET_MAX_ORDER) {
+    Y->pos[slot] = v->pos2;
+    Y->pos_len[slot] = v->t.pos_len[v->t.order - 1];
+  } else {                               // all four pos slots are Y's own (4-order TTM): the dense last level has no crd
+    Y->crd[COMET_MAX_ORDER - 1] = v->pos2;
+    Y->crd_len[COMET_MAX_ORDER - 1] = v->t.pos_len[v->t.order - 1];
+  }
+}
+static const int32_t *stashed_fiber_pos(const comet_sptensor_t *Y, int slot, int64_t *len) {
+  if (slot < COMET_MAX_ORDER) { *len = Y->pos_len[slot]; return Y->pos[slot]; }
+  *len = Y->crd_len[COMET_MAX_ORDER - 1];
+  return Y->crd[COMET_MAX_ORDER - 1];
 }
 
 // Copies X's upper levels (all but the last) into the same levels of Y, device to device.
@@ -407,7 +446,7 @@ extern "C" comet_status_t comet_ttv_symbolic(comet_handle_t handle, const comet_
     if (!Y->val) st = COMET_ERR_ALLOC;
   }
   if (from_coo) {
-    if (st == COMET_OK) stash_fiber_pos(Y, o, 2, &view);
+    if (st == COMET_OK) stash_fiber_pos(Y, o, out_order, &view);
     coo_view_release(ctx, &view, st == COMET_OK, s);
   }
   if (st != COMET_OK) { release(ctx, o, s); memset(Y, 0, sizeof(*Y)); return st; }
@@ -423,8 +462,9 @@ extern "C" comet_status_t comet_ttv(comet_handle_t handle, const comet_sptensor_
   // fibers: X's level-2 pos for CSF; for COO the boundaries that the symbolic call left in Y's spare slot
   const bool from_coo = X->attr[0] == COMET_CN;
   const int last = X->order - 1;
-  const int32_t *fiber_pos = from_coo ? Y->pos[2] : X->pos[last];
-  const int64_t F = from_coo ? Y->pos_len[2] - 1 : X->crd_len[last - 1];
+  int64_t stashed = 0;
+  const int32_t *fiber_pos = from_coo ? stashed_fiber_pos(Y, last, &stashed) : X->pos[last];
+  const int64_t F = from_coo ? stashed - 1 : X->crd_len[last - 1];
   if (!fiber_pos || F < 0) return COMET_ERR_INVALID_ARG;
   if (Y->order != last || Y->nnz != F || (Y->nnz > 0 && !Y->val)) return COMET_ERR_INVALID_ARG;
   if (Y->dtype != X->dtype) return COMET_ERR_INVALID_ARG;
@@ -508,7 +548,7 @@ extern "C" comet_status_t comet_ttm_symbolic_ex(comet_handle_t handle, const com
     }
   }
   if (from_coo) {
-    if (st == COMET_OK) stash_fiber_pos(Y, o, 3, &view);
+    if (st == COMET_OK) stash_fiber_pos(Y, o, X->order, &view);
     coo_view_release(ctx, &view, st == COMET_OK, s);
   }
   if (st != COMET_OK) { release(ctx, o, s); memset(Y, 0, sizeof(*Y)); return st; }
@@ -523,8 +563,9 @@ extern "C" comet_status_t comet_ttm(comet_handle_t handle, const comet_sptensor_
   if (st != COMET_OK) return st;
   const bool from_coo = X->attr[0] == COMET_CN;
   const int last = X->order - 1;
-  const int32_t *fiber_pos = from_coo ? Y->pos[3] : X->pos[last];
-  const int64_t F = from_coo ? Y->pos_len[3] - 1 : X->crd_len[last - 1];
+  int64_t stashed = 0;
+  const int32_t *fiber_pos = from_coo ? stashed_fiber_pos(Y, X->order, &stashed) : X->pos[last];
+  const int64_t F = from_coo ? stashed - 1 : X->crd_len[last - 1];
   if (!fiber_pos || F < 0) return COMET_ERR_INVALID_ARG;
   if (Y->order != X->order || Y->nnz != F * R || (Y->nnz > 0 && !Y->val)) return COMET_ERR_INVALID_ARG;
   if (Y->dtype != X->dtype) return COMET_ERR_INVALID_ARG;

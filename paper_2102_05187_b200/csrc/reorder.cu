@@ -74,7 +74,7 @@ extern "C" comet_status_t comet_reorder(comet_handle_t handle, int32_t order, co
                                         const int32_t *const *h_coo_crd, int32_t iterations,
                                         int32_t *const *h_new_label, void *stream) {
   if (!handle || !h_dims || !h_coo_crd || !h_new_label || nnz < 0 || iterations < 0) return COMET_ERR_INVALID_ARG;
-  if (order < 2 || order > 3) return COMET_ERR_UNSUPPORTED_FORMAT;
+  if (order < 2 || order > COMET_MAX_ORDER) return COMET_ERR_UNSUPPORTED_FORMAT;
   if (nnz > 2147483647ll - 1024) return COMET_ERR_INDEX_OVERFLOW;
   int64_t max_dim = 0;
   for (int m = 0; m < order; ++m) {
@@ -137,7 +137,8 @@ extern "C" comet_status_t comet_reorder(comet_handle_t handle, int32_t order, co
       while (bits < 64 && (span[m] >> bits) != 0) ++bits;
       reorder_init_keys_kernel<<<(unsigned)ceil_div(d, 256), 256, 0, s>>>(ka, pa, d, span[m]);
       if (order == 2) reorder_min_keys_kernel<2><<<(unsigned)ceil_div(nnz, 256), 256, 0, s>>>(r, m, nnz, (unsigned long long *)ka);
-      else reorder_min_keys_kernel<3><<<(unsigned)ceil_div(nnz, 256), 256, 0, s>>>(r, m, nnz, (unsigned long long *)ka);
+      else if (order == 3) reorder_min_keys_kernel<3><<<(unsigned)ceil_div(nnz, 256), 256, 0, s>>>(r, m, nnz, (unsigned long long *)ka);
+      else reorder_min_keys_kernel<4><<<(unsigned)ceil_div(nnz, 256), 256, 0, s>>>(r, m, nnz, (unsigned long long *)ka);
       ctx->launches += 2;
       cudaError_t e = cudaGetLastError();
       if (e != cudaSuccess) { st = cuda_fail(ctx, e); break; }

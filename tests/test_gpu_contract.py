@@ -258,6 +258,45 @@ def test_ttv_ttm_order4_csf(dims, nnz, seed, mode, tile_items):
 
 
 @pytest.mark.parametrize("dims,nnz,seed", ORDER4_CASES)
+@pytest.mark.parametrize("mode", [0, 3])
+def test_ttv_ttm_order4_from_sorted_coo(dims, nnz, seed, mode):
+    """4-order tensors in sorted COO [CN,S,S,S], contracted mode stored last: the symbolic call derives the three
+    upper CSF levels (bit-exact against the oracle's CSF packing), the values against the order-N oracle."""
+    coords, val = synth.random_coo(dims, nnz, seed)
+    c, v = _np(coords), val.numpy()
+    kept = [m for m in range(4) if m != mode]
+    mode_order = (kept[2], kept[0], kept[1], mode)
+    X = upload_packed(oracle.pack(c, v, dims, mode_order, (CN, S, S, S)))
+    csf = oracle.pack(c, v, dims, mode_order, (CU, CU, CU, CU))
+    # the oracle lists fibers by increasing MODE; the storage lists them in (kept[2], kept[0], kept[1]) order
+    keys, want, norm = oracle.ttm_n(c, v, dims, mode, synth.random_dense((dims[mode],), seed).numpy())
+    k0 = keys // (dims[kept[1]] * dims[kept[2]])
+    k1 = (keys // dims[kept[2]]) % dims[kept[1]]
+    k2 = keys % dims[kept[2]]
+    stored = np.lexsort((k1, k0, k2)) if len(keys) else np.zeros(0, dtype=np.int64)
+    vec = synth.random_dense((dims[mode],), seed).numpy()
+    Y = comet.ttv_symbolic(X, mode)
+    assert Y.attr == (CU, CU, CU) and Y.c.nnz == len(keys)
+    for l in range(3):
+        assert_equal_arrays(Y.pos(l), csf.pos[l], f"coo4 ttv pos{l}")
+        assert_equal_arrays(Y.crd(l), csf.crd[l], f"coo4 ttv crd{l}")
+    Y.val.fill_(float("nan"))
+    comet.ttv(X, mode, dev(vec), Y)
+    assert_close(Y.val, want[stored, 0], norm[stored, 0], what="ttv order 4 from coo")
+    for R in (1, 16, 5):
+        U = synth.random_dense((dims[mode], R), seed + 1).numpy()
+        _, wantm, normm = oracle.ttm_n(c, v, dims, mode, U)
+        Z = comet.ttm_symbolic(X, mode, R)
+        assert Z.attr == (CU, CU, CU, D) and Z.pos(3).tolist() == [R]
+        Z.val.fill_(float("nan"))
+        comet.ttm(X, mode, dev(U), Z)
+        assert_close(Z.val.reshape(-1, R), wantm[stored], normm[stored], what=f"ttm order 4 from coo R={R}")
+        for l in range(3):
+            assert_equal_arrays(Z.pos(l), csf.pos[l], f"coo4 ttm pos{l}")
+            assert_equal_arrays(Z.crd(l), csf.crd[l], f"coo4 ttm crd{l}")
+
+
+@pytest.mark.parametrize("dims,nnz,seed", ORDER4_CASES)
 @pytest.mark.parametrize("mode_order", [(0, 1, 2, 3), (3, 1, 0, 2)])
 @pytest.mark.parametrize("attr", [(CN, S, S, S), (CU, CU, CU, CU)])
 def test_mttkrp_order4_every_mode(dims, nnz, seed, mode_order, attr):
@@ -298,12 +337,14 @@ def test_order4_packed_on_the_device_then_contracted():
     c, v = _np(coords), val.numpy()
     X = comet.pack([t.cuda() for t in coords], val.cuda(), dims, (3, 1, 0, 2), (CU, CU, CU, CU))
     vec = synth.random_dense((dims[2],), 9).numpy()
-    _, want, norm = oracle.ttm_n(c, v, dims, 2, vec)
-    # oracle keys are in increasing MODE order (0,1,3); the stored order is (3,1,0): compare as sets of fibers
+    keys, want, norm = oracle.ttm_n(c, v, dims, 2, vec)
+    # oracle keys are in increasing MODE order (0,1,3); the stored order is (3,1,0): bring the oracle's fibers into
+    # the stored order and compare fiber by fiber with each fiber's own normaliser
+    k0, k1, k3 = keys // (dims[1] * dims[3]), (keys // dims[3]) % dims[1], keys % dims[3]
+    stored = np.lexsort((k0, k1, k3))
     Y = comet.ttv(X, 2, dev(vec))
     assert Y.c.nnz == len(want)
-    got = Y.val.cpu().numpy()
-    assert abs(np.sort(got) - np.sort(want[:, 0])).max() <= 1e-12 * norm.max()
+    assert_close(Y.val, want[stored, 0], norm[stored, 0], what="ttv of a device-packed 4-order tensor")
 
 
 @pytest.mark.parametrize("dims,nnz,seed", TENSOR_CASES)

@@ -30,7 +30,8 @@ def _check(coords, dims, iterations):
 
 @pytest.mark.parametrize("dims,nnz,seed", [((7, 5), 12, 1), ((1, 9), 4, 2), ((40, 30), 300, 3), ((300, 200), 5000, 4),
                                            ((50, 50), 0, 5), ((20, 18, 16), 900, 6), ((1, 30, 30), 300, 7),
-                                           ((2000, 5, 7), 500, 8), ((3000, 100), 400, 9)])
+                                           ((2000, 5, 7), 500, 8), ((3000, 100), 400, 9),
+                                           ((9, 8, 7, 6), 400, 10), ((40, 3, 1, 25), 600, 11)])
 @pytest.mark.parametrize("iterations", [0, 1, 2, 4])
 def test_labels_equal_the_oracle(dims, nnz, seed, iterations):
     coords, _ = synth.random_coo(dims, nnz, seed)
@@ -75,5 +76,5 @@ def test_bad_coordinates_and_orders_are_reported():
         comet.reorder([dev(np.array([0, 5], dtype=np.int32)), dev(np.array([0, 1], dtype=np.int32))], (3, 3), 2)
     assert comet.binding.STATUS_NAMES[e.value.status] == "COMET_ERR_COORD_OUT_OF_RANGE"
     with pytest.raises(comet.CometError) as e:
-        comet.reorder([dev(np.zeros(2, dtype=np.int32))] * 4, (2, 2, 2, 2), 1)
+        comet.reorder([dev(np.zeros(2, dtype=np.int32))], (2,), 1)               # a vector has nothing to reorder by
     assert e.value.status == -2

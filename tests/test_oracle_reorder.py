@@ -4,6 +4,7 @@ hand, and recover a band hidden by random relabelling (the effect the paper's se
 import numpy as np
 
 import oracle
+import synth
 from oracle.reorder import reorder, window_columns
 
 
@@ -79,3 +80,23 @@ def test_three_order_tensors_use_the_tuple_of_the_other_modes():
     c2 = np.array([5, 3, 9])
     l0, l1, l2 = reorder([c0, c1, c2], (3, 2, 10), 1)
     assert l0.tolist() == [2, 1, 0]                   # keys (1,5), (1,3), (0,9) -> order: index 2, index 1, index 0
+
+
+def test_four_order_tensors_keep_the_contraction():
+    """Order 4: the labels are permutations and an order-4 tensor-times-vector is unchanged up to the relabelling."""
+    dims = (6, 5, 4, 7)
+    coords, val = synth.random_coo(dims, 200, 12)
+    c, v = [x.numpy() for x in coords], val.numpy()
+    lab = reorder(c, dims, 3)
+    for m, d in enumerate(dims):
+        assert sorted(lab[m].tolist()) == list(range(d))
+    x = synth.random_dense((dims[3],), 12).numpy()
+    dense = np.zeros(dims)
+    dense[tuple(c)] = v
+    want = np.einsum("ijkl,l->ijk", dense, x)
+    relabelled = np.zeros(dims)
+    relabelled[tuple(lab[m][c[m]] for m in range(4))] = v
+    xp = np.zeros_like(x)
+    xp[lab[3]] = x
+    got = np.einsum("ijkl,l->ijk", relabelled, xp)
+    assert np.allclose(got[np.ix_(lab[0], lab[1], lab[2])], want, rtol=0, atol=1e-12)
