@@ -267,3 +267,39 @@ def test_large_matrix_268m_entries():
     want, norm = oracle.spmv(c, v, dims, x.cpu().numpy(), rows=rows)
     rel = assert_close(y[torch.from_numpy(rows).cuda()], want, norm, what="268M-entry spmv")
     print(f"268M entries: worst normalised error {rel:.2e}")
+
+
+def test_full_fp32_c2_spmm_and_c5_coo_mttkrp():
+    """fp32 values at full size (the long-row path of SpMM and the tiled COO MTTKRP): the oracle is fed the same
+    float32 numbers widened to double; both the stated 1e-5 tolerance and the rounding bound of two float roundings
+    (the store and one carry addition) must hold."""
+    case = synth.make(2, device="cuda")
+    v32, B32 = case.val.float(), case.dense["B"].float()
+    A = comet.pack(case.coords, v32, case.dims, (0, 1), (D, CU))
+    C = torch.full((case.dims[0], case.R), float("nan"), dtype=torch.float32, device="cuda")
+    comet.spmm(A, B32, C)
+    lengths = torch.bincount(case.coords[0].long(), minlength=case.dims[0])
+    rows = sample_rows(case.dims[0], 12, always=torch.topk(lengths, 4).indices.tolist() + [0, case.dims[0] - 1])
+    c = [x.cpu().numpy() for x in case.coords]
+    want, norm = oracle.spmm(c, v32.double().cpu().numpy(), case.dims, B32.double().cpu().numpy(), rows=rows)
+    got = C[torch.from_numpy(rows).cuda()].double()
+    assert_close(got, want, norm, tol=1e-5, what="C2 spmm fp32")
+    assert_close(got, want, norm, tol=3 * 2.0 ** -24, what="C2 spmm fp32 (rounding bound)")
+    del A, C, case
+    torch.cuda.empty_cache()
+
+    case = synth.make(5, device="cuda")
+    v32 = case.val.float()
+    Fd = [None, case.dense["B"].float(), case.dense["C"].float()]
+    X = comet.pack(case.coords, v32, case.dims, (0, 1, 2), (CN, S, S))
+    out = torch.full((case.dims[0], case.R), float("nan"), dtype=torch.float32, device="cuda")
+    comet.mttkrp(X, 0, Fd, out)
+    counts = torch.bincount(case.coords[0].long(), minlength=case.dims[0])
+    rows = sample_rows(case.dims[0], 15, always=torch.topk(counts, 4).indices.tolist() + [0, case.dims[0] - 1])
+    del X
+    c = [x.cpu().numpy() for x in case.coords]
+    want, norm = oracle.mttkrp(c, v32.double().cpu().numpy(), case.dims, 0,
+                               [None, Fd[1].double().cpu().numpy(), Fd[2].double().cpu().numpy()], rows=rows)
+    got = out[torch.from_numpy(rows).cuda()].double()
+    assert_close(got, want, norm, tol=1e-5, what="C5 coo mttkrp fp32")
+    assert_close(got, want, norm, tol=3 * 2.0 ** -24, what="C5 coo mttkrp fp32 (rounding bound)")
