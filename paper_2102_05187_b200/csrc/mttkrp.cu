@@ -174,8 +174,8 @@ struct CsfPolicy {
   static constexpr bool kAux = false;
   static constexpr bool kFullUnroll = true;
   static constexpr bool kRolledTail = COMET_CSF_ROLLED_TAIL;
-  static constexpr bool kEntryConsume = true;
-  struct Slot { T r[CPL][VEC]; T p[CPL][VEC]; };           // Q row of the entry; P row of its fiber if it closes one
+  static constexpr bool kSlotCarries = true;               // value and flag word travel in the window slot
+  struct Slot { T r[CPL][VEC]; T p[CPL][VEC]; double v; int32_t flag; };   // Q row of the entry; P row of its fiber if it closes one
 
   const MttkrpArgs &a;
   const L &ln;
@@ -191,8 +191,8 @@ struct CsfPolicy {
   bool a_dirty;
 
   // The look at the tile's fibers and slices (see above). f0 = first fiber that ends behind j0, s0 = its slice.
-  __device__ __forceinline__ CsfPolicy(const MttkrpArgs &args, const L &lanes, int64_t f0_, int64_t s0, int32_t j0_, int32_t j1,
-                                       uint32_t smem_words)
+  __device__ __forceinline__ CsfPolicy(const MttkrpArgs &args, const L &lanes, int64_t f0_, int64_t f_open_, int64_t s0,
+                                       int64_t s_open, int32_t j0_, uint32_t smem_words)
       : a(args), ln(lanes), ends(smem_words), slices(smem_words + kCsfMaskWords * 4), before(smem_words + 2 * kCsfMaskWords * 4),
         j0(j0_), f0((int32_t)f0_), s((int32_t)s0), a_dirty(false) {
     ln.zero(tac);
@@ -205,27 +205,19 @@ struct CsfPolicy {
     val = static_cast<const T *>(a.val);
     for (int w = ln.g; w < 2 * kCsfMaskWords; w += LPN) sts_s32(ends + w * 4, 0);
     ln.sync();
-    int32_t closed = 0;                                    // fibers that end inside the tile
-    for (int64_t k = f0_ + ln.g;; k += LPN) {
-      const int32_t e = k < a.F ? __ldg(a.seg_end2 + k) : 0x7fffffff;
-      const bool in = e <= j1;
-      if (in) atom_or_shared(ends + ((e - 1 - j0) >> 5) * 4, 1u << ((e - 1 - j0) & 31));
-      const int got = __popc(__ballot_sync(ln.mask, in) & ln.mask);
-      closed += got;
-      if (got != LPN) break;                               // ends ascend: a lane outside means the scan is over
+    // the fibers f0 .. f_open-1 end inside the tile, the slices s0 .. s_open-1 with them (both bounds come from the
+    // partition, so the two scans have known lengths and their loads do not wait for one another)
+    f_open = (int32_t)f_open_;
+    for (int64_t k = f0_ + ln.g; k < f_open_; k += LPN) {
+      const int32_t q = __ldg(a.seg_end2 + k) - 1 - j0;
+      atom_or_shared(ends + (q >> 5) * 4, 1u << (q & 31));
     }
-    f_open = f0 + closed;
-    for (int64_t k = s0 + ln.g;; k += LPN) {               // slice k ends with fiber pos1[k + 1] - 1
-      const int64_t last = k < a.S ? (int64_t)__ldg(a.pos1 + k + 1) - 1 : -1;
-      const bool in = last >= 0 && last < f_open;
-      if (in) {
-        const int32_t q = __ldg(a.seg_end2 + last) - 1 - j0;
-        atom_or_shared(slices + (q >> 5) * 4, 1u << (q & 31));
-      }
-      if (__popc(__ballot_sync(ln.mask, in) & ln.mask) != LPN) break;
+    for (int64_t k = s0 + ln.g; k < s_open; k += LPN) {    // slice k ends with fiber pos1[k + 1] - 1
+      const int32_t q = __ldg(a.seg_end2 + __ldg(a.pos1 + k + 1) - 1) - 1 - j0;
+      atom_or_shared(slices + (q >> 5) * 4, 1u << (q & 31));
     }
     ln.sync();
-    for (int w = ln.g; w < kCsfMaskWords; w += LPN) {
+    for (int w = ln.g; w < kCsfMaskWords; w += LPN) {      // fiber ends in front of each word
       int32_t cnt = 0;
       for (int x = 0; x < w; ++x) cnt += __popc((uint32_t)lds_s32(ends + x * 4));
       sts_s32(before + w * 4, cnt);
@@ -248,7 +240,10 @@ struct CsfPolicy {
     e.a = ld_stream(a.crd2 + j);
     e.b = flag_of(j);
   }
-  __device__ __forceinline__ void prefetch(int32_t ck, int32_t flag, Slot &sl) const {
+  __device__ __forceinline__ void prefetch_entry(const Entry16 &e, Slot &sl) const {
+    const int32_t ck = e.a, flag = e.b;
+    sl.v = e.v;
+    sl.flag = flag;
     ln.gather(reinterpret_cast<const T *>(qcol + (int64_t)ck * ldq_bytes), sl.r);
     if (EXPAND || flag != kNoEnd)
       ln.gather(reinterpret_cast<const T *>(pcol + (int64_t)(int32_t)((uint32_t)flag & ~kSliceEnd) * ldp_bytes), sl.p);
@@ -269,7 +264,8 @@ struct CsfPolicy {
     a_dirty = false;
     ++s;
   }
-  __device__ __forceinline__ void consume_entry(int, const Entry16 &e, Slot &sl) {
+  __device__ __forceinline__ void consume_slot(int, Slot &sl) {
+    struct { double v; int32_t b; } e{sl.v, sl.flag};
     if (EXPAND) {
 #pragma unroll
       for (int t = 0; t < CPL; ++t)
@@ -375,9 +371,11 @@ __global__ void __launch_bounds__(kBlockThreads, (CPL * VEC * sizeof(T) <= 16 ? 
     if (ln.g == 0) a.carry_seg[tile] = -1;
     return;
   }
-  const int32_t s0 = __ldg(a.part_slice + tile);
-  // the first fiber of the tile: the one the partition found, unless all its entries lie in earlier tiles
-  P p(a, ln, f0 + (s0 < 0 ? 1 : 0), s0 < 0 ? ~s0 : s0, j0, j1, flags);
+  // The partition stores the slice complemented when the split's fiber has all its entries in front of the split
+  // (its end marker is the next item): that fiber belongs to the tile before. So this tile owns the fibers from
+  // its own corrected start to the next tile's corrected start, and the slices likewise.
+  const int32_t s0 = __ldg(a.part_slice + tile), s1 = __ldg(a.part_slice + tile + 1);
+  P p(a, ln, f0 + (s0 < 0 ? 1 : 0), f1 + (s1 < 0 ? 1 : 0), s0 < 0 ? ~s0 : s0, s1 < 0 ? ~s1 : s1, j0, flags);
   walk_tile(ln, p, j0, j1, smem);
   p.finish(j1);
   const bool carry = p.a_dirty && p.s < a.S;

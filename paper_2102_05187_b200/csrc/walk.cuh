@@ -221,6 +221,12 @@ template <class P> struct policy_is_two_speed<P, decltype((void)P::kTwoSpeed)> {
 template <class P, class = void> struct policy_consumes_entry { static constexpr bool value = false; };
 template <class P> struct policy_consumes_entry<P, decltype((void)P::kEntryConsume)> { static constexpr bool value = P::kEntryConsume; };
 
+// kSlotCarries: the policy keeps what it needs of an entry (value, flags) in the window slot, filled when the
+// entry's rows are requested: prefetch_entry(entry, slot) gets the whole staged entry (one 128-bit read) and
+// consume_slot(q, slot) reads nothing from shared memory. One shared-memory read per entry instead of two.
+template <class P, class = void> struct policy_slot_carries { static constexpr bool value = false; };
+template <class P> struct policy_slot_carries<P, decltype((void)P::kSlotCarries)> { static constexpr bool value = P::kSlotCarries; };
+
 template <class P, class = void> struct policy_rolls_tail { static constexpr bool value = false; };
 template <class P> struct policy_rolls_tail<P, decltype((void)P::kRolledTail)> { static constexpr bool value = P::kRolledTail; };
 
@@ -233,7 +239,8 @@ __device__ __forceinline__ void walk_chunk_unrolled(Policy &p, typename Policy::
 #pragma unroll
   for (int q = 0; q < kChunk; ++q) {
     if (TAIL && q >= n) break;
-    if constexpr (PLAIN) p.consume_plain(q, lds_f64(cur + q * 16), win[q % kPF]);
+    if constexpr (policy_slot_carries<Policy>::value) p.consume_slot(q, win[q % kPF]);
+    else if constexpr (PLAIN) p.consume_plain(q, lds_f64(cur + q * 16), win[q % kPF]);
     else if constexpr (policy_consumes_entry<Policy>::value) p.consume_entry(q, lds_entry(cur + q * 16), win[q % kPF]);
     else p.consume(q, lds_f64(cur + q * 16), Policy::kAux ? lds_s32(cur_aux + q * 4) : 0, win[q % kPF]);
     // refill the slot with the entry kPF ahead (it may sit in the next chunk's half of the ring);
@@ -241,10 +248,14 @@ __device__ __forceinline__ void walk_chunk_unrolled(Policy &p, typename Policy::
     if (TAIL && q + kPF >= n) continue;
     const bool in_cur = q + kPF < kChunk;
     const int at = in_cur ? q + kPF : q + kPF - kChunk;
-    int32_t ca, cb;
-    lds_coords((in_cur ? cur : nxt) + at * 16, ca, cb);
-    if constexpr (policy_is_positional<Policy>::value) p.prefetch_at(at, in_cur, ca, cb, win[q % kPF]);
-    else p.prefetch(ca, cb, win[q % kPF]);
+    if constexpr (policy_slot_carries<Policy>::value) {
+      p.prefetch_entry(lds_entry((in_cur ? cur : nxt) + at * 16), win[q % kPF]);
+    } else {
+      int32_t ca, cb;
+      lds_coords((in_cur ? cur : nxt) + at * 16, ca, cb);
+      if constexpr (policy_is_positional<Policy>::value) p.prefetch_at(at, in_cur, ca, cb, win[q % kPF]);
+      else p.prefetch(ca, cb, win[q % kPF]);
+    }
   }
 }
 
@@ -263,13 +274,18 @@ __device__ __forceinline__ void walk_chunk_rolled(Policy &p, typename Policy::Sl
       const int q = q0 + u;
       if (TAIL && q >= n) break;
       const int r = off + q;
-      if constexpr (policy_consumes_entry<Policy>::value) p.consume_entry(q, lds_entry(lo + r * 16), win[u]);
+      if constexpr (policy_slot_carries<Policy>::value) p.consume_slot(q, win[u]);
+      else if constexpr (policy_consumes_entry<Policy>::value) p.consume_entry(q, lds_entry(lo + r * 16), win[u]);
       else p.consume(q, lds_f64(lo + r * 16), Policy::kAux ? lds_s32(lo_aux + r * 4) : 0, win[u]);
       if (TAIL && q + kPF >= n) continue;
-      int32_t ca, cb;
-      lds_coords(lo + ((r + kPF) & (2 * kChunk - 1)) * 16, ca, cb);
-      if constexpr (policy_is_positional<Policy>::value) p.prefetch_at((q + kPF) & (kChunk - 1), q + kPF < kChunk, ca, cb, win[u]);
-      else p.prefetch(ca, cb, win[u]);
+      if constexpr (policy_slot_carries<Policy>::value) {
+        p.prefetch_entry(lds_entry(lo + ((r + kPF) & (2 * kChunk - 1)) * 16), win[u]);
+      } else {
+        int32_t ca, cb;
+        lds_coords(lo + ((r + kPF) & (2 * kChunk - 1)) * 16, ca, cb);
+        if constexpr (policy_is_positional<Policy>::value) p.prefetch_at((q + kPF) & (kChunk - 1), q + kPF < kChunk, ca, cb, win[u]);
+        else p.prefetch(ca, cb, win[u]);
+      }
     }
   }
 }
@@ -329,10 +345,14 @@ __device__ __forceinline__ void walk_tile(const L &ln, Policy &p, int32_t j0, in
   typename Policy::Slot win[kPF];
 #pragma unroll
   for (int u = 0; u < kPF; ++u) {
-    int32_t ca, cb;
-    lds_coords(smem + u * 16, ca, cb);
-    if constexpr (policy_is_positional<Policy>::value) p.prefetch_at(u, true, ca, cb, win[u]);
-    else p.prefetch(ca, cb, win[u]);
+    if constexpr (policy_slot_carries<Policy>::value) {
+      p.prefetch_entry(lds_entry(smem + u * 16), win[u]);
+    } else {
+      int32_t ca, cb;
+      lds_coords(smem + u * 16, ca, cb);
+      if constexpr (policy_is_positional<Policy>::value) p.prefetch_at(u, true, ca, cb, win[u]);
+      else p.prefetch(ca, cb, win[u]);
+    }
   }
 
   int half = 0;
