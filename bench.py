@@ -215,8 +215,9 @@ def flush_l2(buf):
     buf.add_(1)
 
 
-def per_kernel(comet, handle, steps, warm, peak, peak_kind="measured"):
-    """Every workload at full size: pack time and contraction time per op and format."""
+def per_kernel(comet, handle, steps, warm, peak, peak_kind="measured", scale=1.0, only=None):
+    """Every workload (at full size unless `scale`): pack time and contraction time per op and format. `only`:
+    restrict to these config numbers (profiling runs)."""
     out = []
     l2buf = torch.zeros(192 << 20, dtype=torch.uint8, device="cuda")      # > 126 MB L2
     plans = [(1, "spmv", "csr", (0, 1), (D, CU)), (2, "spmm", "csr", (0, 1), (D, CU)),
@@ -224,8 +225,10 @@ def per_kernel(comet, handle, steps, warm, peak, peak_kind="measured"):
              (5, "mttkrp", "coo", (0, 1, 2), (CN, S, S)), (5, "mttkrp", "csf", (0, 1, 2), (CU, CU, CU))]
     case = None
     for cfg, op, fmt, order, attr in plans:
+        if only and cfg not in only:
+            continue
         if case is None or case.name[:2] != f"C{cfg}":
-            case = synth.make(cfg, device="cuda")
+            case = synth.make(cfg, scale=scale, device="cuda")
         coords, val = case.coords, case.val
         small = cfg in (1, 3)              # working set near or below L2: flush between repetitions
 
@@ -364,6 +367,18 @@ def oracle_step(dims, coords, val, B):
     nbytes = bytes_pack(n, 2, 4 * (dims[0] + 2 + n)) + n * 12 + (dims[0] + 1) * 4 + B.size * 8 + dims[0] * B.shape[1] * 8
     del pk
     return dt, nbytes
+
+
+def run_kernels_only(args):
+    """--kernels-only: the per-workload table alone (optionally scaled down and restricted), for profiling runs."""
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    import paper_2102_05187_b200 as comet
+    handle = comet.Handle()
+    peak, peak_kind = measured_peak()
+    only = [int(x) for x in args.configs.split(",")] if args.configs else None
+    table = per_kernel(comet, handle, max(1, args.steps), max(1, args.warmup), peak, peak_kind, args.kernels_scale, only)
+    print(json.dumps({"kernels": table, "scale": args.kernels_scale}))
 
 
 def run_ours(args):
@@ -544,10 +559,16 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--scale", type=float, default=1.0, help="workload scale (1.0 is the only reported one)")
     ap.add_argument("--headline-only", action="store_true", help="skip the per-kernel table")
+    ap.add_argument("--kernels-only", action="store_true", help="only the per-workload table (profiling runs)")
+    ap.add_argument("--kernels-scale", type=float, default=1.0, help="workload scale of --kernels-only")
+    ap.add_argument("--configs", default="", help="comma-separated config numbers for --kernels-only (default: all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sample-rows", type=float, default=1.0 / 8,
                     help="fraction of the rows in the CPU sample (the cpu_baseline leg and --impl reference use the same one)")
     args = ap.parse_args()
+    if args.kernels_only:
+        run_kernels_only(args)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         # plain `python bench.py --gpus N`: start the N replicas (one process per GPU) and hand over to them
