@@ -30,6 +30,13 @@ comet_status_t mttkrp_csf(Context *ctx, int dtype, const int32_t *pos1, const in
                           int64_t N, int64_t rows, const void *P, int64_t ldp, const void *Q, int64_t ldq,
                           int64_t R, void *out, int64_t ldo, cudaStream_t stream);
 
+// CSF with the output mode stored at level 1, on the tiled walker (mttkrp.cu): fp64, R a power of two up to 64 and
+// aligned operands; COMET_ERR_UNSUPPORTED_FORMAT otherwise (take mttkrp_scatter then). P = the ROOT mode's factor.
+comet_status_t mttkrp_csf_level1(Context *ctx, int dtype, const int32_t *pos1, const int32_t *crd0, const int32_t *crd1,
+                                 const int32_t *pos2, const int32_t *crd2, const void *val, int64_t S, int64_t F, int64_t N,
+                                 int64_t rows, const void *P, int64_t ldp, const void *Q, int64_t ldq, int64_t R, void *out,
+                                 int64_t ldo, cudaStream_t stream);
+
 // MTTKRP with the output mode NOT stored first, by atomic accumulation (see mttkrp_scatter.cu). kind 0: COO,
 // crd0 = output-mode coordinates and crd1 / crd2 those of A's / B's modes; kind 1 / 2: CSF, output mode at
 // level 1 / 2, A = the root mode's factor, B = the factor of the remaining mode.

@@ -51,6 +51,7 @@ struct MttkrpArgs {
   int32_t *carry_seg;
   int32_t carry_ld;
   const int32_t *part_fiber, *part_slice;   // CSF: per tile boundary, from the partition kernel (num_tiles + 1 each)
+  bool level1;                              // CSF: the output mode is the one stored at level 1 (atomic accumulation)
 };
 
 // ------------------------------------------------------------------------------------------- COO
@@ -167,8 +168,16 @@ __device__ __forceinline__ void atom_or_shared(uint32_t addr, uint32_t bits) {
 // ends in front of an entry is its fiber's number), both rows are gathered per entry, and the walk is the one of
 // the sorted-COO kernel: slice sum += (x * P row) * Q row, a row store where a slice ends. The P rows of a
 // fiber's later entries are L1 hits.
-template <class T, int LPN, int CPL, int VEC, bool EXPAND>
+// FORM 2 (kCsfLevel1): the OUTPUT mode is the one stored at level 1. The walk is the same; a fiber's sum, times the
+// row of the root mode's factor (P here, one row per slice), is added to output row crd1[fiber] with atomic adds
+// (the rows of one output index are spread over the whole tensor, so no tile owns one); nothing is carried from
+// tile to tile. Sums are double; the output must be zero when the kernel starts.
+constexpr int kCsfFold = 0, kCsfExpand = 1, kCsfLevel1 = 2;
+
+template <class T, int LPN, int CPL, int VEC, int FORM>
 struct CsfPolicy {
+  static constexpr bool EXPAND = FORM == kCsfExpand;
+  static constexpr bool LEVEL1 = FORM == kCsfLevel1;
   using L = Lanes<T, LPN, CPL, VEC>;
   static constexpr int kPF = COMET_PF_CSF;
   static constexpr bool kAux = false;
@@ -184,6 +193,7 @@ struct CsfPolicy {
   T *ocol;
   const T *val;
   double tac[CPL][VEC], aac[CPL][VEC];   // open fiber sum, open slice sum
+  T arow[CPL][VEC];                      // LEVEL1: the root factor's row of the open slice
   uint32_t ends, slices, before;         // shared addresses of the tile's three word arrays
   int32_t j0, f0;
   int32_t s;                             // open slice
@@ -203,6 +213,7 @@ struct CsfPolicy {
     ldq_bytes = (int32_t)(a.ldq * sizeof(T));
     ocol = static_cast<T *>(a.out) + ln.col0;
     val = static_cast<const T *>(a.val);
+    if (LEVEL1 && s < a.S) ln.gather(reinterpret_cast<const T *>(pcol + (int64_t)__ldg(a.crd0 + s) * ldp_bytes), arow);
     for (int w = ln.g; w < 2 * kCsfMaskWords; w += LPN) sts_s32(ends + w * 4, 0);
     ln.sync();
     // the fibers f0 .. f_open-1 end inside the tile, the slices s0 .. s_open-1 with them (both bounds come from the
@@ -245,7 +256,7 @@ struct CsfPolicy {
     sl.v = e.v;
     sl.flag = flag;
     ln.gather(reinterpret_cast<const T *>(qcol + (int64_t)ck * ldq_bytes), sl.r);
-    if (EXPAND || flag != kNoEnd)
+    if (!LEVEL1 && (EXPAND || flag != kNoEnd))
       ln.gather(reinterpret_cast<const T *>(pcol + (int64_t)(int32_t)((uint32_t)flag & ~kSliceEnd) * ldp_bytes), sl.p);
   }
   __device__ __forceinline__ void fold(const T (&prow)[CPL][VEC]) {      // aac += tac * P[crd1[f], :]
@@ -264,8 +275,28 @@ struct CsfPolicy {
     a_dirty = false;
     ++s;
   }
+  // LEVEL1: out[row, :] += tac * arow (atomic), tac = 0
+  __device__ __forceinline__ void scatter_fiber(int32_t row) {
+    double *dst = reinterpret_cast<double *>(a.out) + (int64_t)row * a.ldo + ln.col0;
+#pragma unroll
+    for (int t = 0; t < CPL; ++t)
+      if (ln.ok[t])
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) {
+          atomicAdd(dst + t * L::kStride + k, tac[t][k] * (double)arow[t][k]);
+          tac[t][k] = 0.0;
+        }
+  }
   __device__ __forceinline__ void consume_slot(int, Slot &sl) {
     struct { double v; int32_t b; } e{sl.v, sl.flag};
+    if (LEVEL1) {
+      ln.fma_rows(e.v, sl.r, tac);
+      if (e.b != kNoEnd) {
+        scatter_fiber((int32_t)((uint32_t)e.b & ~kSliceEnd));
+        if (e.b < 0 && ++s < a.S) ln.gather(reinterpret_cast<const T *>(pcol + (int64_t)__ldg(a.crd0 + s) * ldp_bytes), arow);
+      }
+      return;
+    }
     if (EXPAND) {
 #pragma unroll
       for (int t = 0; t < CPL; ++t)
@@ -290,6 +321,7 @@ struct CsfPolicy {
       return;
     }
     if (((uint32_t)lds_s32(ends + (q >> 5) * 4) >> (q & 31)) & 1u) return;     // the tile stops at a fiber end
+    if (LEVEL1) { scatter_fiber(__ldg(a.crd1 + f_open)); return; }
     T prow[CPL][VEC];
     ln.gather(reinterpret_cast<const T *>(pcol + (int64_t)__ldg(a.crd1 + f_open) * ldp_bytes), prow);
     fold(prow);
@@ -345,14 +377,14 @@ __global__ void __launch_bounds__(kBlockThreads) zero_unowned_rows_kernel(const 
   }
 }
 
-template <class T, int LPN, int CPL, int VEC, bool EXPAND>
+template <class T, int LPN, int CPL, int VEC, int FORM>
 __global__ void __launch_bounds__(kBlockThreads, (CPL * VEC * sizeof(T) <= 16 ? COMET_MINB_CSF : 2)) mttkrp_csf_kernel(const MttkrpArgs a) {
   using L = Lanes<T, LPN, CPL, VEC>;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int worker = threadIdx.x / LPN;
   const int64_t tile = (int64_t)blockIdx.x * L::kWorkers + worker;
   if (tile >= a.num_tiles) return;
-  using P = CsfPolicy<T, LPN, CPL, VEC, EXPAND>;
+  using P = CsfPolicy<T, LPN, CPL, VEC, FORM>;
   const uint32_t smem = smem_u32(smem_raw) + worker * RingLayout<L, false>::kWorkerBytes;
   const uint32_t flags = smem_u32(smem_raw) + (uint32_t)RingLayout<L, false>::kBlockBytes + worker * kCsfWorkerBytes;
   const L ln(a.R);
@@ -368,7 +400,7 @@ __global__ void __launch_bounds__(kBlockThreads, (CPL * VEC * sizeof(T) <= 16 ? 
   const int64_t f0 = __ldg(a.part_fiber + tile), f1 = __ldg(a.part_fiber + tile + 1);
   const int32_t j0 = (int32_t)(d0 - f0), j1 = (int32_t)(d1 - f1);
   if (j0 >= j1) {                                          // nothing but an end marker: its fiber was closed by the tile before
-    if (ln.g == 0) a.carry_seg[tile] = -1;
+    if (FORM != kCsfLevel1 && ln.g == 0) a.carry_seg[tile] = -1;
     return;
   }
   // The partition stores the slice complemented when the split's fiber has all its entries in front of the split
@@ -378,6 +410,7 @@ __global__ void __launch_bounds__(kBlockThreads, (CPL * VEC * sizeof(T) <= 16 ? 
   P p(a, ln, f0 + (s0 < 0 ? 1 : 0), f1 + (s1 < 0 ? 1 : 0), s0 < 0 ? ~s0 : s0, s1 < 0 ? ~s1 : s1, j0, flags);
   walk_tile(ln, p, j0, j1, smem);
   p.finish(j1);
+  if (FORM == kCsfLevel1) return;                          // everything went out through atomic adds
   const bool carry = p.a_dirty && p.s < a.S;
   if (ln.g == 0) a.carry_seg[tile] = carry ? (int32_t)p.s : -1;
   if (carry) ln.store_carry(a.carry_val + tile * a.carry_ld + ln.col0, p.aac);
@@ -417,11 +450,15 @@ static comet_status_t launch_mttkrp(Context *ctx, MttkrpArgs a, cudaStream_t str
   bool expand = CSF && a.N < 4 * a.F;
   if (const char *e = getenv("COMET_CSF_FORM")) expand = CSF && (e[0] == 'e' ? true : (e[0] == 'f' ? false : expand));
   auto kernel = !CSF ? mttkrp_coo_kernel<T, LPN, CPL, VEC>
-                     : (expand ? mttkrp_csf_kernel<T, LPN, CPL, VEC, true> : mttkrp_csf_kernel<T, LPN, CPL, VEC, false>);
+                     : (expand ? mttkrp_csf_kernel<T, LPN, CPL, VEC, kCsfExpand> : mttkrp_csf_kernel<T, LPN, CPL, VEC, kCsfFold>);
+  if constexpr (CSF && sizeof(T) == 8 && VEC == 2 && CPL == 1) {
+    if (a.level1) kernel = mttkrp_csf_kernel<T, LPN, CPL, VEC, kCsfLevel1>;
+  }
   if (smem > 48 * 1024)
     COMET_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   kernel<<<blocks, kBlockThreads, smem, stream>>>(a);
   COMET_LAUNCH_CHECK(ctx);
+  if (CSF && a.level1) return COMET_OK;
   carry_fixup_launch(sizeof(T) == 4 ? COMET_F32 : COMET_F64, a.carry_val, a.carry_seg, a.num_tiles, a.R, a.carry_ld, a.out,
                      a.ldo, CSF ? a.crd0 : nullptr, stream);
   COMET_LAUNCH_CHECK(ctx);
@@ -489,6 +526,31 @@ comet_status_t mttkrp_csf(Context *ctx, int dtype, const int32_t *pos1, const in
     COMET_LAUNCH_CHECK(ctx);
   }
   return dtype == COMET_F32 ? mttkrp_chunks<true, float>(ctx, a, R, stream) : mttkrp_chunks<true, double>(ctx, a, R, stream);
+}
+
+// CSF, output mode stored at level 1: out[crd1[f], :] += (sum over fiber f of val * Q[crd2, :]) * P[crd0[slice of f], :].
+// fp64 with 16-byte aligned operands and R a multiple of 2 up to 64; returns COMET_ERR_UNSUPPORTED_FORMAT otherwise
+// (the caller then takes the general scatter kernel). `out` is zero-filled here.
+comet_status_t mttkrp_csf_level1(Context *ctx, int dtype, const int32_t *pos1, const int32_t *crd0, const int32_t *crd1,
+                                 const int32_t *pos2, const int32_t *crd2, const void *val, int64_t S, int64_t F, int64_t N,
+                                 int64_t rows, const void *P, int64_t ldp, const void *Q, int64_t ldq, int64_t R, void *out,
+                                 int64_t ldo, cudaStream_t stream) {
+  if (dtype != COMET_F64 || !(R == 2 || R == 4 || R == 8 || R == 16 || R == 32 || R == 64) || N == 0 || S == 0)
+    return COMET_ERR_UNSUPPORTED_FORMAT;
+  if (!aligned16(P) || !aligned16(Q) || !aligned16(out) || ldp % 2 || ldq % 2 || ldo % 2) return COMET_ERR_UNSUPPORTED_FORMAT;
+  if (ldp >= (1ll << 28) || ldq >= (1ll << 28)) return COMET_ERR_INDEX_OVERFLOW;
+  if (ldo == R) {
+    COMET_CUDA_TRY(ctx, cudaMemsetAsync(out, 0, (size_t)rows * R * sizeof(double), stream));
+  } else {
+    const comet_status_t zs = zero_rows(ctx, out, dtype, rows, R, ldo, stream);
+    if (zs != COMET_OK) return zs;
+  }
+  MttkrpArgs a{};
+  a.pos1 = pos1; a.crd0 = crd0; a.crd1 = crd1; a.seg_end2 = pos2 + 1; a.crd2 = crd2; a.val = val;
+  a.S = S; a.F = F; a.N = N; a.rows = rows;
+  a.P = P; a.ldp = ldp; a.Q = Q; a.ldq = ldq; a.out = out; a.ldo = ldo;
+  a.level1 = true;
+  return mttkrp_chunks<true, double>(ctx, a, R, stream);
 }
 
 }  // namespace comet

@@ -1,13 +1,13 @@
-"""Table 1 of the paper, executed literally: the per-attribute loops that enumerate the stored
-coordinates of a tensor from its pos/crd arrays.
+"""An independent reader of the packed layout: a walk over (pos, crd) by the level rules of the storage format
+(Table 1 of the paper gives them as one loop form per attribute; include/comet.h states them in words):
 
-    D : for i from 0 to pos[0]                      -> coordinate i,     position m * pos[0] + i
-    CU: for i from pos[m] to pos[m+1]: idx = crd[i] -> coordinate idx,   position i
-    CN: for i from pos[0] to pos[1]:  idx = crd[i]  -> coordinate idx,   position i
-    S : idx = crd[m]                                -> coordinate idx,   position m
+    D   every coordinate 0 .. pos[0]-1 under each parent position m; the child's position is m * pos[0] + coordinate
+    CU  the children of parent position m are the positions pos[m] .. pos[m+1]-1; coordinate crd[position]
+    CN  (first level) the positions pos[0] .. pos[1]-1; coordinate crd[position]
+    S   one child per parent position m, at the same position; coordinate crd[m]
 
-(m is the position produced by the level above, 0 at the first level.) This is an independent reader
-of the packed layout: it shares nothing with either packing implementation.
+(m is the position produced by the level above, 0 at the first level.) It shares nothing with either packing
+implementation.
 """
 
 
