@@ -178,7 +178,8 @@ seg_gather_kernel(const SegGatherArgs a, const HeavyArgs h) {
   if (carry) ln.store_carry(a.carry_val + tile * a.carry_ld + ln.col0, p.acc);
 }
 
-// Merge-path split at every tile boundary, a thread per boundary.
+// Merge-path split at every tile boundary, a thread per boundary (a warp per boundary with a 32-way search was
+// measured: slower, the boundaries are many and the searches hide each other's latency).
 __global__ void __launch_bounds__(kBlockThreads) seg_partition_kernel(const int32_t *__restrict__ seg_end, int64_t M, int64_t N,
                                                                       int32_t tile_items, int64_t num_tiles,
                                                                       int32_t *__restrict__ part) {
