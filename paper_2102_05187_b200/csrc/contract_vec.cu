@@ -52,6 +52,9 @@ struct SegGatherPolicy {
   static constexpr int kPF = COMET_PF_GATHER;
   static constexpr bool kAux = false;
   static constexpr bool kFullUnroll = true;
+  // one copy of the unrolled body where the chunk is long (instruction cache; measured: SpMM config 2 -4 %); the
+  // narrow shapes have short tiles of short chunks, where the slower rolled tail costs more than it saves (TTM +5 %)
+  static constexpr bool kRolledTail = LPN >= 16;
   struct Slot { T r[CPL][VEC]; };
 
   const SegGatherArgs &a;

@@ -45,6 +45,7 @@ struct HeavyPolicy {
   static constexpr int kPF = CPL > 1 ? COMET_PF_HEAVY / 2 : COMET_PF_HEAVY;   // register budget: 64
   static constexpr bool kAux = false;
   static constexpr bool kFullUnroll = true;
+  static constexpr bool kRolledTail = true;
   struct Slot { T r[CPL][VEC]; };
   const L &ln;
   const T *val;
