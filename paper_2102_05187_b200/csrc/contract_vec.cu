@@ -59,66 +59,55 @@ struct SegGatherPolicy {
 
   const SegGatherArgs &a;
   const L &ln;
-  const T *val;
-  T *cmat;                  // this lane's piece 0 of row 0 of C
   const char *bcol;         // this lane's piece 0 of row 0 of B
-  int32_t ldb_bytes;
   double acc[CPL][VEC];
-  T *out;                   // this lane's piece 0 of the open segment's output row (identity mapping)
-  const int32_t *endp;      // seg_end + open segment
-  int32_t segs_left;        // segments from the open one to the last
-  int32_t next_end;         // leaf position where the open segment ends (-1: no segment left)
-  int32_t base, rel_end;    // chunk base and next_end relative to it
-  int32_t last_flush;       // leaf position of the latest flush (entries at or after it are still in acc)
+  // The segment state is three words (the rest is recomputed where a segment closes): registers are what the
+  // window of gathers in flight is made of.
+  int32_t seg;              // the open segment
+  int32_t base, rel_end;    // chunk base; where the open segment ends, relative to it (negative: no segment left)
   uint64_t pass;            // PASS_THROUGH: L2 evict-first policy of the gathers (the other role's block of B stays)
 
   __device__ __forceinline__ SegGatherPolicy(const SegGatherArgs &args, const L &lanes, int64_t i0, int32_t j0)
-      : a(args), ln(lanes), base(j0), last_flush(j0) {
+      : a(args), ln(lanes), seg((int32_t)i0), base(j0) {
     ln.zero(acc);
     if (PASS_THROUGH) pass = l2_policy_evict_first();
-    val = static_cast<const T *>(a.val);
     bcol = reinterpret_cast<const char *>(static_cast<const T *>(a.B) + ln.col0);
-    ldb_bytes = (int32_t)(a.ldb * sizeof(T));
-    cmat = static_cast<T *>(a.C) + ln.col0;
-    out = cmat + i0 * a.ldc;
-    endp = a.seg_end + i0;
-    segs_left = (int32_t)(a.M - i0);
-    next_end = segs_left > 0 ? __ldg(endp) : -1;
-    rel_end = next_end - base;
+    rel_end = end_of_open();
   }
-  __device__ __forceinline__ int64_t segment() const { return a.M - segs_left; }
+  __device__ __forceinline__ int32_t end_of_open() const {
+    return seg < a.M ? __ldg(a.seg_end + seg) - base : (int32_t)0x80000000 / 2;
+  }
+  __device__ __forceinline__ int64_t segment() const { return seg; }
   __device__ __forceinline__ void fetch(int32_t j, Entry16 &e, int32_t &) const {
-    e.v = (double)ld_stream(val + j);
+    e.v = (double)ld_stream(static_cast<const T *>(a.val) + j);
     e.a = ld_stream(a.crd + j);
   }
   __device__ __forceinline__ void prefetch(int32_t c, int32_t, Slot &s) const {
-    if (PASS_THROUGH) ln.gather_hint(reinterpret_cast<const T *>(bcol + (int64_t)c * ldb_bytes), s.r, pass);
-    else ln.gather(reinterpret_cast<const T *>(bcol + (int64_t)c * ldb_bytes), s.r);
+    const T *row = reinterpret_cast<const T *>(bcol + (int64_t)c * (int32_t)(a.ldb * sizeof(T)));
+    if (PASS_THROUGH) ln.gather_hint(row, s.r, pass);
+    else ln.gather(row, s.r);
   }
-  __device__ __forceinline__ void begin_chunk(int32_t b) { base = b; rel_end = next_end - b; }
+  __device__ __forceinline__ void begin_chunk(int32_t b) { rel_end -= b - base; base = b; }
 
   // Stores the open segment (and, for a compressed root level, zero-fills the rows in front of it).
-  __device__ __forceinline__ void flush(int32_t j) {
+  __device__ __forceinline__ void flush() {
+    T *cmat = static_cast<T *>(a.C) + ln.col0;
     if (MAPPED) {
-      const int64_t i = segment();
+      const int64_t i = seg;
       const int64_t r = __ldg(a.out_row + i);
       const int64_t lo = (i > 0) ? (int64_t)__ldg(a.out_row + i - 1) + 1 : 0;
       ln.zero_rows(cmat, a.ldc, lo, r);
       if (i == a.M - 1) ln.zero_rows(cmat, a.ldc, r + 1, a.out_rows);
       ln.store_row(cmat + r * a.ldc, acc);
     } else {
-      ln.store_row(out, acc);
-      out += a.ldc;
+      ln.store_row(cmat + (int64_t)seg * a.ldc, acc);
     }
     ln.zero(acc);
-    ++endp;
-    --segs_left;
-    next_end = segs_left > 0 ? __ldg(endp) : -1;
-    rel_end = next_end - base;
-    last_flush = j;
+    ++seg;
+    rel_end = end_of_open();
   }
   __device__ __forceinline__ void consume(int q, double v, int32_t, Slot &s) {
-    while (rel_end == q) flush(base + q);      // segments (possibly empty ones) that end in front of this leaf
+    while (rel_end == q) flush();              // segments (possibly empty ones) that end in front of this leaf
     ln.fma_rows(v, s.r, acc);
   }
 };
@@ -173,10 +162,12 @@ seg_gather_kernel(const SegGatherArgs a, const HeavyArgs h) {
 
   SegGatherPolicy<T, LPN, CPL, VEC, MAPPED, HEAVY> p(a, ln, i0, j0);
   walk_tile(ln, p, j0, j1, smem);
-  while (p.segment() < i1) p.flush(j1);                  // end markers that close the tile
+  while (p.segment() < i1) p.flush();                    // end markers that close the tile
 
+  // leaf entries of a segment that ends in a later tile: the open segment starts in front of the tile's end
   const int64_t seg = p.segment();
-  const bool carry = seg < a.M && j1 > p.last_flush;     // leaf entries of a segment that ends in a later tile
+  const int32_t open_from = seg > 0 ? __ldg(a.seg_end + seg - 1) : 0;
+  const bool carry = seg < a.M && (open_from > j0 ? open_from : j0) < j1;
   if (ln.g == 0) a.carry_seg[tile] = carry ? (int32_t)seg : -1;
   if (carry) ln.store_carry(a.carry_val + tile * a.carry_ld + ln.col0, p.acc);
 }
