@@ -4,14 +4,17 @@
 //
 //   1. keys      one 64-bit key per entry: the coordinates in storage-level order, level 0 in the most
 //                significant bits (so key order = lexicographic order); coordinates are range-checked.
-//   2. sort      stable LSD radix sort of (key, entry index), 8 bits per pass, only over the bits in use.
+//   2. sort      stable LSD radix sort of (key, 32-bit payload), 8 bits per pass, only over the bits in use; the
+//                first pass forms the keys from the caller's arrays, so steps 1 and 2 share their launches. The
+//                payload is the value itself when it has 32 bits, else the entry's index.
 //                Per pass: per-tile digit histogram -> exclusive scan of the (digit, tile) table ->
 //                stable scatter (warp-level match ranks, per-warp digit counters in shared memory).
 //   3. levels    head flags from key prefixes: entry p opens a new node at level l when the key prefix
 //                down to level l differs from its predecessor's. Counting pass -> scan -> ONE host
 //                synchronisation to learn the node counts -> exact allocation -> emit pass that writes
-//                crd (compaction), pos (rank of the first child at every parent head), and the values
-//                permuted into leaf order. Equal adjacent keys are duplicates and are reported.
+//                crd (compaction), pos (rank of the first child at every parent head), and the values in leaf
+//                order (64-bit ones gathered through the sorted indices). Equal adjacent keys are duplicates
+//                and are reported.
 //
 // No inter-CTA waiting anywhere: every scan is reduce / scan-of-sums / apply in separate launches.
 #include "common.cuh"
@@ -47,23 +50,53 @@ struct CoordPtrs { const int32_t *p[COMET_MAX_ORDER]; };   // level order
 // ORDER is a template parameter so that the per-level loops unroll and the by-value descriptor structs
 // are read with constant indices (a runtime index would push them into local memory).
 template <int ORDER>
-__global__ void make_keys_kernel(CoordPtrs c, KeyLayout k, int64_t n, uint64_t *__restrict__ keys,
-                                 uint32_t *__restrict__ idx, int32_t *__restrict__ status) {
-  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (p >= n) return;
+__device__ __forceinline__ uint64_t entry_key(const CoordPtrs &c, const KeyLayout &k, int64_t p, bool &bad) {
   int32_t v[ORDER];
 #pragma unroll
   for (int l = 0; l < ORDER; ++l) v[l] = __ldcs(c.p[l] + p);
   uint64_t key = 0;
-  bool bad = false;
 #pragma unroll
   for (int l = 0; l < ORDER; ++l) {
     bad |= (v[l] < 0) | ((int64_t)v[l] >= k.dim[l]);
     key |= ((uint64_t)(uint32_t)v[l] & ((1ull << k.bits[l]) - 1)) << k.shift[l];
   }
+  return key;
+}
+
+// Where a sort pass reads its (key, payload) pairs. The payload is one 32-bit word that travels with the key
+// through every pass: a 32-bit value itself (as raw bits; nothing is gathered afterwards), else the entry's index
+// (64-bit values are gathered through it once, at the end: carrying them would cost more per pass than the gather
+// saves from five passes on).
+struct SortedPairs {                 // the output of the pass before
+  const uint64_t *keys;
+  const uint32_t *pay;
+  __device__ __forceinline__ uint64_t key(int64_t i, bool &) const { return __ldcs(keys + i); }
+  __device__ __forceinline__ uint32_t payload(int64_t i) const { return __ldcs(pay + i); }
+};
+
+template <int ORDER>
+struct CooEntries {                  // the first pass: the caller's COO arrays; the keys are formed on the fly
+  CoordPtrs c;
+  KeyLayout k;
+  const uint32_t *val32;             // 32-bit values, or null: the payload is the entry's index
+  __device__ __forceinline__ uint64_t key(int64_t i, bool &bad) const { return entry_key<ORDER>(c, k, i, bad); }
+  __device__ __forceinline__ uint32_t payload(int64_t i) const {
+    uint32_t p = (uint32_t)i;
+    if (val32) p = __ldcs(val32 + i);
+    return p;
+  }
+};
+
+// Keys and payloads written out as they stand: only for keys of zero bits (every extent 1), where no pass runs.
+template <int ORDER>
+__global__ void make_keys_kernel(CooEntries<ORDER> src, int64_t n, uint64_t *__restrict__ keys,
+                                 uint32_t *__restrict__ pay, int32_t *__restrict__ status) {
+  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= n) return;
+  bool bad = false;
+  keys[p] = src.key(p, bad);
+  pay[p] = src.payload(p);
   if (bad) atomicOr(status + kStatusRange, 1);
-  keys[p] = key;
-  idx[p] = (uint32_t)p;
 }
 
 // ------------------------------------------------------------------------------------------------ scan
@@ -161,25 +194,37 @@ comet_status_t exclusive_scan(Context *ctx, const uint32_t *in, uint32_t *out, i
 }
 
 // ------------------------------------------------------------------------------------------------ radix sort
-__global__ void __launch_bounds__(kSortThreads) radix_histogram_kernel(const uint64_t *__restrict__ keys, int64_t n,
-                                                                       int shift, int64_t tiles,
-                                                                       uint32_t *__restrict__ table) {
+template <class Src>
+__global__ void __launch_bounds__(kSortThreads) radix_histogram_kernel(Src src, int64_t n, int shift, int64_t tiles,
+                                                                       uint32_t *__restrict__ table,
+                                                                       int32_t *__restrict__ status) {
   __shared__ uint32_t s_cnt[256];
   s_cnt[threadIdx.x] = 0;
   __syncthreads();
   const int64_t base = (int64_t)blockIdx.x * kSortTile;
+  bool bad = false;
+  uint64_t k[kSortItems];
+  const bool full = base + kSortTile <= n;
+#pragma unroll
+  for (int t = 0; t < kSortItems; ++t) {          // unconditional loads: the eight of a thread are in flight together
+    const int64_t i = base + (int64_t)t * kSortThreads + threadIdx.x;
+    k[t] = src.key(full || i < n ? i : n - 1, bad);
+  }
 #pragma unroll
   for (int t = 0; t < kSortItems; ++t) {
     const int64_t i = base + (int64_t)t * kSortThreads + threadIdx.x;
-    if (i < n) atomicAdd(&s_cnt[(keys[i] >> shift) & 255], 1u);
+    if (full || i < n) atomicAdd(&s_cnt[(k[t] >> shift) & 255], 1u);
   }
+  if (bad) atomicOr(status + kStatusRange, 1);    // only the pass that forms the keys can see a bad coordinate
   __syncthreads();
   table[(int64_t)threadIdx.x * tiles + blockIdx.x] = s_cnt[threadIdx.x];     // digit-major
 }
 
-__global__ void __launch_bounds__(kSortThreads, 4) radix_scatter_kernel(
-    const uint64_t *__restrict__ kin, const uint32_t *__restrict__ pin, uint64_t *__restrict__ kout,
-    uint32_t *__restrict__ pout, const uint32_t *__restrict__ table, int64_t n, int shift, int64_t tiles) {
+template <class Src>
+__global__ void __launch_bounds__(kSortThreads, 4) radix_scatter_kernel(Src src, uint64_t *__restrict__ kout,
+                                                                        uint32_t *__restrict__ pout,
+                                                                        const uint32_t *__restrict__ table, int64_t n,
+                                                                        int shift, int64_t tiles) {
   __shared__ uint32_t s_cnt[kSortWarps][256];     // per-warp digit counts, then where each warp's keys of a digit go
   __shared__ uint32_t s_delta[256];               // global position of digit d's run minus its start inside the tile
   __shared__ uint64_t s_key[kSortTile];           // the tile in sorted order
@@ -187,17 +232,30 @@ __global__ void __launch_bounds__(kSortThreads, 4) radix_scatter_kernel(
   __shared__ uint32_t s_warp[32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int w = 0; w < kSortWarps; ++w) s_cnt[w][tid] = 0;
+  // where digit `tid`'s run of this tile starts in the output: asked for now, needed after the ranking
+  const uint32_t digit_base = __ldg(table + (int64_t)tid * tiles + blockIdx.x);
 
   // Item r of lane l of warp w sits at tile_base + w*(32*ITEMS) + r*32 + l: memory order is (w, r, l).
   const int64_t tile_base = (int64_t)blockIdx.x * kSortTile;
   const int64_t warp_base = tile_base + (int64_t)warp * (32 * kSortItems);
   uint64_t key[kSortItems];
   uint32_t pay[kSortItems];
+  bool ignored = false;
+  if (tile_base + kSortTile <= n) {               // all loads first, none behind a branch
 #pragma unroll
-  for (int r = 0; r < kSortItems; ++r) {          // all loads first
-    const int64_t i = warp_base + r * 32 + lane;
-    key[r] = i < n ? __ldcs(kin + i) : ~0ull;     // slots past the end rank after every real key of the tile
-    pay[r] = i < n ? __ldcs(pin + i) : 0u;
+    for (int r = 0; r < kSortItems; ++r) {
+      const int64_t i = warp_base + r * 32 + lane;
+      key[r] = src.key(i, ignored);
+      pay[r] = src.payload(i);
+    }
+  } else {
+#pragma unroll
+    for (int r = 0; r < kSortItems; ++r) {
+      const int64_t i = warp_base + r * 32 + lane;
+      key[r] = src.key(i < n ? i : n - 1, ignored);
+      pay[r] = src.payload(i < n ? i : n - 1);
+      if (i >= n) key[r] = ~0ull;                  // slots past the end rank after every real key of the tile
+    }
   }
   __syncthreads();
   uint32_t rank[kSortItems];
@@ -228,7 +286,7 @@ __global__ void __launch_bounds__(kSortThreads, 4) radix_scatter_kernel(
       s_cnt[w][tid] = off;
       off += c;
     }
-    s_delta[tid] = table[(int64_t)tid * tiles + blockIdx.x] - start;
+    s_delta[tid] = digit_base - start;
   }
   __syncthreads();
 #pragma unroll
@@ -253,52 +311,88 @@ __global__ void __launch_bounds__(kSortThreads, 4) radix_scatter_kernel(
   }
 }
 
-// Stable LSD radix sort of (key, payload) pairs over the low `bits` key bits, 8 bits per pass. `ka`/`pa` hold
-// the input and, on return, the sorted pairs (the pointers are swapped with `kb`/`pb` after every pass); all four
-// buffers hold n + 1 elements. `table` holds radix_sort_table_words(n) words, `scan_tmp` scan_tmp_words of that.
 int64_t radix_sort_table_words(int64_t n) { return 256 * ceil_div(n > 0 ? n : 1, kSortTile); }
 
-comet_status_t radix_sort_pairs(Context *ctx, uint64_t *&ka, uint64_t *&kb, uint32_t *&pa, uint32_t *&pb, int64_t n,
-                                int bits, uint32_t *table, uint32_t *scan_tmp, cudaStream_t s) {
-  if (n <= 0) return COMET_OK;
+// One stable pass over the 8 key bits at `shift`: per-tile digit counts, their scan, the scatter.
+template <class Src>
+static comet_status_t radix_pass(Context *ctx, const Src &src, uint64_t *kout, uint32_t *pout, int64_t n, int shift,
+                                 uint32_t *table, uint32_t *scan_tmp, cudaStream_t s) {
   const int64_t tiles = ceil_div(n, kSortTile);
-  for (int shift = 0; shift < bits; shift += 8) {
-    radix_histogram_kernel<<<(unsigned)tiles, kSortThreads, 0, s>>>(ka, n, shift, tiles, table);
-    COMET_LAUNCH_CHECK(ctx);
-    comet_status_t st = exclusive_scan(ctx, table, table, 256 * tiles, scan_tmp, nullptr, s);
+  radix_histogram_kernel<Src><<<(unsigned)tiles, kSortThreads, 0, s>>>(src, n, shift, tiles, table, ctx->d_status);
+  COMET_LAUNCH_CHECK(ctx);
+  comet_status_t st = exclusive_scan(ctx, table, table, 256 * tiles, scan_tmp, nullptr, s);
+  if (st != COMET_OK) return st;
+  radix_scatter_kernel<Src><<<(unsigned)tiles, kSortThreads, 0, s>>>(src, kout, pout, table, n, shift, tiles);
+  COMET_LAUNCH_CHECK(ctx);
+  return COMET_OK;
+}
+
+// Stable LSD radix sort of (key, payload) pairs over the key bits [first_bit, bits), 8 bits per pass. `ka`/`pa`
+// hold the input and, on return, the sorted pairs (the pointers are swapped with `kb`/`pb` after every pass); all
+// four buffers hold n + 1 elements. `table` holds radix_sort_table_words(n) words, `scan_tmp` scan_tmp_words of
+// that.
+static comet_status_t radix_sort_from(Context *ctx, uint64_t *&ka, uint64_t *&kb, uint32_t *&pa, uint32_t *&pb,
+                                      int64_t n, int first_bit, int bits, uint32_t *table, uint32_t *scan_tmp,
+                                      cudaStream_t s) {
+  for (int shift = first_bit; shift < bits; shift += 8) {
+    const SortedPairs src{ka, pa};
+    comet_status_t st = radix_pass(ctx, src, kb, pb, n, shift, table, scan_tmp, s);
     if (st != COMET_OK) return st;
-    radix_scatter_kernel<<<(unsigned)tiles, kSortThreads, 0, s>>>(ka, pa, kb, pb, table, n, shift, tiles);
-    COMET_LAUNCH_CHECK(ctx);
     uint64_t *tk = ka; ka = kb; kb = tk;
     uint32_t *tp = pa; pa = pb; pb = tp;
   }
   return COMET_OK;
 }
 
+comet_status_t radix_sort_pairs(Context *ctx, uint64_t *&ka, uint64_t *&kb, uint32_t *&pa, uint32_t *&pb, int64_t n,
+                                int bits, uint32_t *table, uint32_t *scan_tmp, cudaStream_t s) {
+  if (n <= 0) return COMET_OK;
+  return radix_sort_from(ctx, ka, kb, pa, pb, n, 0, bits, table, scan_tmp, s);
+}
+
+// The packing's sort: the COO entries by their keys. The first pass reads the caller's arrays and forms the keys
+// on the fly (the coordinates are range-checked there); on return `ka`/`pa` hold the sorted keys and payloads.
+template <int ORDER>
+static comet_status_t sort_entries(Context *ctx, const CoordPtrs &coords, const KeyLayout &key, const uint32_t *val32,
+                                   uint64_t *&ka, uint64_t *&kb, uint32_t *&pa, uint32_t *&pb, int64_t n,
+                                   uint32_t *table, uint32_t *scan_tmp, cudaStream_t s) {
+  const CooEntries<ORDER> src{coords, key, val32};
+  if (key.total_bits == 0) {
+    make_keys_kernel<ORDER><<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(src, n, ka, pa, ctx->d_status);
+    COMET_LAUNCH_CHECK(ctx);
+    return COMET_OK;
+  }
+  comet_status_t st = radix_pass(ctx, src, kb, pb, n, 0, table, scan_tmp, s);
+  if (st != COMET_OK) return st;
+  uint64_t *tk = ka; ka = kb; kb = tk;
+  uint32_t *tp = pa; pa = pb; pb = tp;
+  return radix_sort_from(ctx, ka, kb, pa, pb, n, 8, key.total_bits, table, scan_tmp, s);
+}
+
 // ------------------------------------------------------------------------------------------------ duplicates
 // COMET_PACK_SUM_DUPLICATES: after the sort, entries with equal keys are adjacent and, the sort being stable,
 // in the order they were given. The first entry of each run keeps the key; its value becomes the sum of the
 // run, added one by one in double in that order (one thread per run: runs are short unless the input is
-// degenerate). The level pass then sees distinct keys, an identity permutation and the merged values.
+// degenerate). The level pass then sees distinct keys and the merged values.
 __global__ void dup_heads_kernel(const uint64_t *__restrict__ keys, int64_t n, uint32_t *__restrict__ head) {
   const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (p < n) head[p] = (p == 0 || keys[p] != keys[p - 1]) ? 1u : 0u;
 }
 
-template <class V>
+// GATHER: the values are the caller's, read through the sorted payload (entry indices); else they are in sorted
+// order already.
+template <class V, bool GATHER>
 __global__ void dup_merge_kernel(const uint64_t *__restrict__ keys, const uint32_t *__restrict__ perm,
                                  const V *__restrict__ val_in, int64_t n, const uint32_t *__restrict__ rank,
-                                 uint64_t *__restrict__ keys_out, uint32_t *__restrict__ perm_out,
-                                 V *__restrict__ val_out) {
+                                 uint64_t *__restrict__ keys_out, V *__restrict__ val_out) {
   const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (p >= n) return;
   const uint64_t k = keys[p];
   if (p > 0 && keys[p - 1] == k) return;
-  double sum = (double)val_in[perm[p]];
-  for (int64_t q = p + 1; q < n && keys[q] == k; ++q) sum = sum + (double)val_in[perm[q]];
+  double sum = (double)val_in[GATHER ? (int64_t)perm[p] : p];
+  for (int64_t q = p + 1; q < n && keys[q] == k; ++q) sum = sum + (double)val_in[GATHER ? (int64_t)perm[q] : q];
   const uint32_t r = rank[p];
   keys_out[r] = k;
-  perm_out[r] = r;
   val_out[r] = (V)sum;
 }
 
@@ -336,12 +430,19 @@ __global__ void __launch_bounds__(kLevelThreads) level_count_kernel(const uint64
 #pragma unroll
   for (int l = 0; l < ORDER; ++l) mine[l] = 0;
   bool dup = false;
+  uint64_t key[kLevelItems], prev[kLevelItems];
+#pragma unroll
+  for (int t = 0; t < kLevelItems; ++t) {         // unconditional loads: all of a thread's in flight together
+    const int64_t p = base + (int64_t)t * kLevelThreads + threadIdx.x;
+    const int64_t q = p < n ? p : n - 1;
+    key[t] = keys[q];
+    prev[t] = keys[q > 0 ? q - 1 : 0];
+  }
 #pragma unroll
   for (int t = 0; t < kLevelItems; ++t) {
     const int64_t p = base + (int64_t)t * kLevelThreads + threadIdx.x;
     if (p < n) {
-      const uint64_t k = keys[p];
-      const uint64_t kp = p > 0 ? keys[p - 1] : 0;
+      const uint64_t k = key[t], kp = prev[t];
       dup |= (p > 0) & (k == kp);
 #pragma unroll
       for (int l = 0; l < ORDER; ++l)
@@ -370,8 +471,9 @@ struct LevelOut {
   uint32_t nodes[COMET_MAX_ORDER];   // node count of every counted level (indexed by level)
 };
 
-// Per tile: ranks of the heads (tile-local scan + the tile's scanned offset), then crd / pos / val.
-template <int ORDER, class V>
+// Per tile: ranks of the heads (tile-local scan + the tile's scanned offset), then crd / pos / val. GATHER: the
+// values are the caller's, read through the sorted payload (entry indices); else they are in sorted order already.
+template <int ORDER, class V, bool GATHER>
 __global__ void __launch_bounds__(kLevelThreads) level_emit_kernel(const uint64_t *__restrict__ keys,
                                                                    const uint32_t *__restrict__ perm,
                                                                    const V *__restrict__ val_in, int64_t n,
@@ -381,16 +483,24 @@ __global__ void __launch_bounds__(kLevelThreads) level_emit_kernel(const uint64_
   __shared__ uint32_t s_warp[32];
   const int64_t base = (int64_t)blockIdx.x * kLevelTile + (int64_t)threadIdx.x * kLevelItems;   // blocked: 8 consecutive
   uint64_t k[kLevelItems + 1];
-  uint32_t src[kLevelItems];
-  k[0] = (base > 0 && base - 1 < n) ? keys[base - 1] : 0;
-#pragma unroll
-  for (int t = 0; t < kLevelItems; ++t) {
-    k[t + 1] = (base + t < n) ? keys[base + t] : 0;
-    src[t] = (base + t < n) ? perm[base + t] : 0;
-  }
   V vals[kLevelItems];
+  k[0] = (base > 0 && base - 1 < n) ? keys[base - 1] : 0;
+  if constexpr (GATHER) {
+    uint32_t src[kLevelItems];
 #pragma unroll
-  for (int t = 0; t < kLevelItems; ++t) vals[t] = (base + t < n) ? __ldg(val_in + src[t]) : (V)0;   // the random gather, all in flight
+    for (int t = 0; t < kLevelItems; ++t) {
+      k[t + 1] = (base + t < n) ? keys[base + t] : 0;
+      src[t] = (base + t < n) ? perm[base + t] : 0;
+    }
+#pragma unroll
+    for (int t = 0; t < kLevelItems; ++t) vals[t] = (base + t < n) ? __ldg(val_in + src[t]) : (V)0;   // the random gather, all in flight
+  } else {
+#pragma unroll
+    for (int t = 0; t < kLevelItems; ++t) {
+      k[t + 1] = (base + t < n) ? keys[base + t] : 0;
+      vals[t] = (base + t < n) ? __ldcs(val_in + base + t) : (V)0;
+    }
+  }
 
   // rank[l] = nodes of level l opened before this thread's first entry
   uint32_t rank[ORDER];
@@ -673,24 +783,26 @@ extern "C" comet_status_t comet_pack_ex(comet_handle_t handle, int32_t order, co
   TempBlocks tmp(ctx, s);
   uint64_t *keys_a = (uint64_t *)tmp.get((size_t)(n + 1) * 8);
   uint64_t *keys_b = (uint64_t *)tmp.get((size_t)(n + 1) * 8);
-  uint32_t *perm_a = (uint32_t *)tmp.get((size_t)(n + 1) * 4);
-  uint32_t *perm_b = (uint32_t *)tmp.get((size_t)(n + 1) * 4);
+  uint32_t *pay_a = (uint32_t *)tmp.get((size_t)(n + 1) * 4);   // fp32 values as raw bits, else entry indices
+  uint32_t *pay_b = (uint32_t *)tmp.get((size_t)(n + 1) * 4);
   const int64_t table_words = table_len > counts_len ? table_len : counts_len;
   uint32_t *table = (uint32_t *)tmp.get((size_t)table_words * 4);
   uint32_t *scan_tmp = (uint32_t *)tmp.get((size_t)(ceil_div(table_words, kScanTile) + 1) * 4);
-  if (!keys_a || !keys_b || !perm_a || !perm_b || !table || !scan_tmp) return COMET_ERR_ALLOC;
+  if (!keys_a || !keys_b || !pay_a || !pay_b || !table || !scan_tmp) return COMET_ERR_ALLOC;
 
   COMET_CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_status, 0, 16 * sizeof(int32_t), s));
   uint32_t *d_nodes = reinterpret_cast<uint32_t *>(ctx->d_status) + 8;   // node counts live beside the status words
 
+  const void *sorted_val = nullptr;    // the values in sorted order, once some array holds them so
   if (n > 0) {
-    if (order == 2) make_keys_kernel<2><<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(coords, key, n, keys_a, perm_a, ctx->d_status);
-    else if (order == 3) make_keys_kernel<3><<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(coords, key, n, keys_a, perm_a, ctx->d_status);
-    else make_keys_kernel<4><<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(coords, key, n, keys_a, perm_a, ctx->d_status);
-    COMET_LAUNCH_CHECK(ctx);
     {
-      comet_status_t st = radix_sort_pairs(ctx, keys_a, keys_b, perm_a, perm_b, n, total_bits, table, scan_tmp, s);
+      const uint32_t *val32 = dtype == COMET_F32 ? static_cast<const uint32_t *>(coo_val) : nullptr;
+      comet_status_t st;
+      if (order == 2) st = sort_entries<2>(ctx, coords, key, val32, keys_a, keys_b, pay_a, pay_b, n, table, scan_tmp, s);
+      else if (order == 3) st = sort_entries<3>(ctx, coords, key, val32, keys_a, keys_b, pay_a, pay_b, n, table, scan_tmp, s);
+      else st = sort_entries<4>(ctx, coords, key, val32, keys_a, keys_b, pay_a, pay_b, n, table, scan_tmp, s);
       if (st != COMET_OK) return st;
+      if (dtype == COMET_F32) sorted_val = pay_a;
     }
     if (flags & COMET_PACK_SUM_DUPLICATES) {
       // merge runs of equal keys; costs one more synchronisation (the number of distinct cells sizes the rest)
@@ -709,15 +821,14 @@ extern "C" comet_status_t comet_pack_ex(comet_handle_t handle, int32_t order, co
       const int64_t distinct = reinterpret_cast<uint32_t *>(ctx->h_pinned)[12];
       // keys_b is both the scan's scratch and the merge's output: the scan has finished (synchronised above)
       if (dtype == COMET_F32)
-        dup_merge_kernel<float><<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(keys_a, perm_a, (const float *)coo_val, n, rank,
-                                                                          keys_b, perm_b, (float *)merged);
+        dup_merge_kernel<float, false><<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(keys_a, nullptr, (const float *)sorted_val, n, rank,
+                                                                                 keys_b, (float *)merged);
       else
-        dup_merge_kernel<double><<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(keys_a, perm_a, (const double *)coo_val, n,
-                                                                           rank, keys_b, perm_b, (double *)merged);
+        dup_merge_kernel<double, true><<<(unsigned)ceil_div(n, 256), 256, 0, s>>>(keys_a, pay_a, (const double *)coo_val, n, rank,
+                                                                                 keys_b, (double *)merged);
       COMET_LAUNCH_CHECK(ctx);
       keys_a = keys_b;
-      perm_a = perm_b;
-      coo_val = merged;
+      sorted_val = merged;
       n = distinct;
       level_tiles = ceil_div(n > 0 ? n : 1, kLevelTile);
     }
@@ -775,15 +886,20 @@ extern "C" comet_status_t comet_pack_ex(comet_handle_t handle, int32_t order, co
   if (n > 0) {
     const unsigned g = (unsigned)level_tiles;
     if (dtype == COMET_F32) {
-      const float *vin = (const float *)coo_val;
-      if (order == 2) level_emit_kernel<2, float><<<g, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
-      else if (order == 3) level_emit_kernel<3, float><<<g, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
-      else level_emit_kernel<4, float><<<g, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
+      const float *vin = (const float *)sorted_val;
+      if (order == 2) level_emit_kernel<2, float, false><<<g, kLevelThreads, 0, s>>>(keys_a, nullptr, vin, n, plan, level_tiles, table, lo);
+      else if (order == 3) level_emit_kernel<3, float, false><<<g, kLevelThreads, 0, s>>>(keys_a, nullptr, vin, n, plan, level_tiles, table, lo);
+      else level_emit_kernel<4, float, false><<<g, kLevelThreads, 0, s>>>(keys_a, nullptr, vin, n, plan, level_tiles, table, lo);
+    } else if (sorted_val) {
+      const double *vin = (const double *)sorted_val;
+      if (order == 2) level_emit_kernel<2, double, false><<<g, kLevelThreads, 0, s>>>(keys_a, nullptr, vin, n, plan, level_tiles, table, lo);
+      else if (order == 3) level_emit_kernel<3, double, false><<<g, kLevelThreads, 0, s>>>(keys_a, nullptr, vin, n, plan, level_tiles, table, lo);
+      else level_emit_kernel<4, double, false><<<g, kLevelThreads, 0, s>>>(keys_a, nullptr, vin, n, plan, level_tiles, table, lo);
     } else {
       const double *vin = (const double *)coo_val;
-      if (order == 2) level_emit_kernel<2, double><<<g, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
-      else if (order == 3) level_emit_kernel<3, double><<<g, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
-      else level_emit_kernel<4, double><<<g, kLevelThreads, 0, s>>>(keys_a, perm_a, vin, n, plan, level_tiles, table, lo);
+      if (order == 2) level_emit_kernel<2, double, true><<<g, kLevelThreads, 0, s>>>(keys_a, pay_a, vin, n, plan, level_tiles, table, lo);
+      else if (order == 3) level_emit_kernel<3, double, true><<<g, kLevelThreads, 0, s>>>(keys_a, pay_a, vin, n, plan, level_tiles, table, lo);
+      else level_emit_kernel<4, double, true><<<g, kLevelThreads, 0, s>>>(keys_a, pay_a, vin, n, plan, level_tiles, table, lo);
     }
   }
   if (order == 2) level_finish_kernel<2><<<kSmCount, 256, 0, s>>>(keys_a, n, plan, lo);
