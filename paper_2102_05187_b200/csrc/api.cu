@@ -659,7 +659,7 @@ extern "C" comet_status_t comet_mttkrp(comet_handle_t handle, const comet_sptens
     if (h_ld[m1] >= (1ll << 28) || h_ld[m2] >= (1ll << 28)) return COMET_ERR_INDEX_OVERFLOW;
     if (coo)
       return mttkrp_scatter(ctx, X->dtype, 0, nullptr, X->crd[level], X->crd[la], nullptr, X->crd[lb], X->val, 0, 0,
-                            X->nnz, rows, P, h_ld[m1], Q, h_ld[m2], R, out, ldo, s);
+                            X->nnz, rows, X->dims[m1], X->dims[m2], P, h_ld[m1], Q, h_ld[m2], R, out, ldo, s);
     if (level == 1) {                    // the tiled walker with atomic adds per fiber, where its shapes apply
       const comet_status_t ws = mttkrp_csf_level1(ctx, X->dtype, X->pos[1], X->crd[0], X->crd[1], X->pos[2], X->crd[2], X->val,
                                                   X->crd_len[0], X->crd_len[1], X->nnz, rows, P, h_ld[m1], Q, h_ld[m2], R, out,
@@ -667,7 +667,8 @@ extern "C" comet_status_t comet_mttkrp(comet_handle_t handle, const comet_sptens
       if (ws != COMET_ERR_UNSUPPORTED_FORMAT) return ws;
     }
     return mttkrp_scatter(ctx, X->dtype, level, X->pos[1], X->crd[0], X->crd[1], X->pos[2], X->crd[2], X->val,
-                          X->crd_len[0], X->crd_len[1], X->nnz, rows, P, h_ld[m1], Q, h_ld[m2], R, out, ldo, s);
+                          X->crd_len[0], X->crd_len[1], X->nnz, rows, X->dims[m1], X->dims[m2], P, h_ld[m1], Q, h_ld[m2], R,
+                          out, ldo, s);
   }
   if (coo)
     return mttkrp_coo(ctx, X->dtype, X->crd[0], X->crd[1], X->crd[2], X->val, X->nnz, rows, P, h_ld[m1], Q, h_ld[m2], R, out,

@@ -39,11 +39,13 @@ comet_status_t mttkrp_csf_level1(Context *ctx, int dtype, const int32_t *pos1, c
 
 // MTTKRP with the output mode NOT stored first, by atomic accumulation (see mttkrp_scatter.cu). kind 0: COO,
 // crd0 = output-mode coordinates and crd1 / crd2 those of A's / B's modes; kind 1 / 2: CSF, output mode at
-// level 1 / 2, A = the root mode's factor, B = the factor of the remaining mode.
+// level 1 / 2, A = the root mode's factor, B = the factor of the remaining mode. rows / a_rows / b_rows: the
+// extents of the output mode and of A's and B's modes.
 comet_status_t mttkrp_scatter(Context *ctx, int dtype, int kind, const int32_t *pos1, const int32_t *crd0,
                               const int32_t *crd1, const int32_t *pos2, const int32_t *crd2, const void *val, int64_t S,
-                              int64_t F, int64_t N, int64_t rows, const void *A, int64_t lda, const void *B, int64_t ldb,
-                              int64_t R, void *out, int64_t ldo, cudaStream_t stream);
+                              int64_t F, int64_t N, int64_t rows, int64_t a_rows, int64_t b_rows, const void *A,
+                              int64_t lda, const void *B, int64_t ldb, int64_t R, void *out, int64_t ldo,
+                              cudaStream_t stream);
 
 // The same for 4-order tensors, every output mode. kind -1: COO (crd[0] = output-mode coordinates, crd[1..3] =
 // those of A's, B's, C's modes); kind 0..3: CSF, output mode at that level, A / B / C = the factors of the three

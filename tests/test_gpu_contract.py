@@ -417,6 +417,54 @@ def test_mttkrp_every_mode_of_a_fixed_tensor(dims, nnz, seed, mode_order, attr):
             assert_close(out, want, norm, what=f"mttkrp mode {mode} of {mode_order} R={R}")
 
 
+def _skewed_leaf_coo(dims, nnz, seed):
+    """Distinct cells whose last coordinate is drawn with very unequal frequencies (a few popular values)."""
+    g = np.random.default_rng(seed)
+    i = g.integers(0, dims[0], 3 * nnz)
+    j = g.integers(0, dims[1], 3 * nnz)
+    k = np.minimum((dims[2] * g.random(3 * nnz) ** 4).astype(np.int64), dims[2] - 1)
+    cells = np.unique((i * dims[1] + j) * dims[2] + k)
+    cells = g.permutation(cells)[:nnz]
+    c = [(cells // (dims[1] * dims[2])).astype(np.int32), (cells // dims[2] % dims[1]).astype(np.int32),
+         (cells % dims[2]).astype(np.int32)]
+    return c, g.uniform(-1.0, 1.0, cells.size)
+
+
+@pytest.mark.parametrize("dims,nnz", [((40, 30, 500), 20000), ((7, 9, 20), 700), ((300, 200, 3000), 60000)])
+@pytest.mark.parametrize("dtype", ["f64", "f32"])
+def test_mttkrp_leaf_mode_with_popular_rows_in_shared_memory(dims, nnz, dtype, monkeypatch):
+    """The leaf-mode kernel that keeps the most popular output rows in shared memory, forced on small tensors
+    (by default only large ones take it): fewer rows than slots, more rows than slots, R below, at and above a
+    warp's width, entries that straddle the 32-fiber window."""
+    monkeypatch.setenv("COMET_MTTKRP_HOT_ROWS", "1")
+    c, v = _skewed_leaf_coo(dims, nnz, 11)
+    if dtype == "f32":
+        v = v.astype(np.float32).astype(np.float64)
+    pk = oracle.pack(c, v, dims, (0, 1, 2), (CU, CU, CU))
+    if dtype == "f32":
+        pos = [dev(p, torch.int32) if p.size else None for p in pk.pos]
+        crd = [dev(q, torch.int32) if q.size else None for q in pk.crd]
+        X = comet.SpTensor.from_arrays(pk.dims, pk.mode_order, pk.attr, pos, crd, dev(pk.val.astype(np.float32)))
+    else:
+        X = upload_packed(pk)
+    for R in (1, 5, 32, 40, 64):
+        F = [synth.random_dense((d, R), 11, 60 + m).numpy() for m, d in enumerate(dims)]
+        if dtype == "f32":
+            F = [f.astype(np.float32).astype(np.float64) for f in F]
+        want, norm = oracle.mttkrp(c, v, dims, 2, F)
+        tdt = torch.float32 if dtype == "f32" else torch.float64
+        out = torch.full((dims[2], R), float("nan"), dtype=tdt, device="cuda")
+        comet.mttkrp(X, 2, [dev(F[0]).to(tdt), dev(F[1]).to(tdt), None], out)
+        assert_close(out.double(), want, norm, tol=FP64_TOL if dtype == "f64" else 4e-7, what=f"leaf mttkrp {dtype} R={R}")
+    monkeypatch.setenv("COMET_MTTKRP_HOT_ROWS", "0")
+    out0 = torch.full((dims[2], 5), float("nan"), dtype=torch.float64, device="cuda")
+    if dtype == "f64":
+        F = [synth.random_dense((d, 5), 11, 60 + m).numpy() for m, d in enumerate(dims)]
+        want, norm = oracle.mttkrp(c, v, dims, 2, F)
+        comet.mttkrp(X, 2, [dev(F[0]), dev(F[1]), None], out0)
+        assert_close(out0, want, norm, what="leaf mttkrp, general kernel")
+
+
 def test_mttkrp_non_root_strided_output_and_integers():
     dims = (25, 20, 15)
     coords, val = synth.random_coo(dims, 2000, 5, integer_values=True)
