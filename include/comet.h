@@ -79,6 +79,8 @@ typedef enum {
  *   COMET_PACK_CSR=1|0          forces / forbids the histogram CSR packing of comet_pack_ex (COMET_PACK_CSR_HISTOGRAM)
  *   COMET_SEG_PARTITION=0       matrix-operand kernels search their tile boundaries themselves (no pre-pass)
  *   COMET_CSF_FORM=fold|expand  root-mode CSF MTTKRP: per-fiber or per-entry form (default: by mean fiber length)
+ *   COMET_MTTKRP_HOT_ROWS=0|1   leaf-mode CSF MTTKRP: never / always keep the most popular output rows in shared memory
+ *                               (default: for R >= 16 and at least 2^20 entries)
  *   COMET_SPMM_LONG_ROWS=0      comet_spmm without the long-row path; COMET_SPMM_LONG_ROW, _LONG_TILE, _PIECE,
  *                               _BLOCK_MB, _BLOCKS, _LONG_CTAS, _LONG_MIN_NNZ, _LONG_MIN_B_MB: its threshold
  *                               (entries), tile and piece sizes, block size / count of B, CTAs of the long-row
@@ -237,7 +239,9 @@ comet_status_t comet_ttm(comet_handle_t handle, const comet_sptensor_t *X, int32
  *     the summation ORDER is not fixed and results agree from run to run only up to rounding (still
  *     within the stated tolerance). About 2-4x slower than the first-level case; callers that repeat the
  *     same mode many times may prefer a second comet_pack with that mode first. For fp32 tensors this
- *     path takes rows x R doubles of handle scratch.
+ *     path takes rows x R doubles of handle scratch. The leaf mode of a large CSF tensor keeps its most
+ *     popular output rows in shared memory (adds to one address retire one by one in L2) and allocates
+ *     4 bytes per fiber and 8 per output row for the duration of the call.
  * 4-order tensors ([CN,S,S,S] or [CU,CU,CU,CU]; out_{i_n r} = sum x * the three other factors' entries): every
  * mode, all by atomic accumulation (the note on the summation order applies to all four modes).
  *   h_factors[order]  HOST array of DEVICE pointers, factor of mode m is dims[m] x R with leading
