@@ -105,7 +105,7 @@ constexpr int kHotChunk = 1024;                    // entries per warp and step
 // memory is a compare-and-swap loop of about a dozen instructions, an add in L2 one instruction: past the rows
 // that L2 serialises, more slots cost more than they save).
 constexpr size_t kHotBytes = 32 * 1024;
-constexpr int64_t kHotMaxRows = 1ll << 22;         // the selection is one CTA's work: not for very long modes
+constexpr int64_t kHotMaxRows = 1ll << 24;         // two 32-bit words per output row are allocated for the call
 constexpr int64_t kHotSamples = 1ll << 22;
 
 __global__ void sample_rows_kernel(const int32_t *__restrict__ crd, int64_t n, int64_t stride, int32_t *__restrict__ counts) {
@@ -113,62 +113,57 @@ __global__ void sample_rows_kernel(const int32_t *__restrict__ crd, int64_t n, i
   if (p < n) atomicAdd(counts + __ldg(crd + p), 1);
 }
 
-__device__ __forceinline__ int block_sum_1024(int v, int *s_warp) {
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-  __syncthreads();                                  // s_warp may still be read from the call before
-  if ((threadIdx.x & 31) == 0) s_warp[threadIdx.x >> 5] = v;
-  __syncthreads();
-  int t = s_warp[threadIdx.x & 31];
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
-  return t;
+// Which rows get a slot: a histogram of the sampled counts over bins of 1/16 octave (counts within 6 % of each
+// other share a bin), the lowest bin that at most `slots` rows reach, and a slot for every row that reaches it
+// (slot numbers in the order the rows arrive; should the top bin alone hold more rows than slots, the first
+// `slots` of them are taken).
+constexpr int kCountBins = 512;
+
+__device__ __forceinline__ int count_bin(int32_t c) {         // c >= 1; monotone in c
+  const int e = 31 - __clz(c);
+  const int m = e >= 4 ? (c >> (e - 4)) & 15 : (c << (4 - e)) & 15;
+  return e * 16 + m;
 }
 
-// One CTA: the smallest count t >= 1 that at most `slots` rows reach (bisection), then slot numbers in row order.
-// hot_slot[row] = slot or -1; hot_rows[slot] = row; *n_hot = slots in use.
-__global__ void __launch_bounds__(1024) select_hot_rows_kernel(const int32_t *__restrict__ counts, int64_t rows,
-                                                                      int32_t slots, int32_t *__restrict__ hot_slot,
-                                                                      int32_t *__restrict__ hot_rows,
-                                                                      int32_t *__restrict__ n_hot) {
-  __shared__ int s_warp[32];
-  int top = 0;
-  for (int64_t r = threadIdx.x; r < rows; r += 1024) top = max(top, counts[r]);
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) top = max(top, __shfl_xor_sync(0xffffffffu, top, off));
-  if ((threadIdx.x & 31) == 0) s_warp[threadIdx.x >> 5] = top;
+__global__ void __launch_bounds__(256) count_histogram_kernel(const int32_t *__restrict__ counts, int64_t rows,
+                                                              int32_t *__restrict__ bins) {
+  __shared__ int32_t s_bins[kCountBins];
+  for (int b = threadIdx.x; b < kCountBins; b += 256) s_bins[b] = 0;
   __syncthreads();
-  top = 0;
-  for (int w = 0; w < 32; ++w) top = max(top, s_warp[w]);
-  int lo = 1, hi = top + 1;                         // no row reaches top + 1
-  while (lo < hi) {
-    const int mid = lo + (hi - lo) / 2;
-    int mine = 0;
-    for (int64_t r = threadIdx.x; r < rows; r += 1024) mine += counts[r] >= mid;
-    const int reach = block_sum_1024(mine, s_warp);
-    if (reach <= slots) hi = mid; else lo = mid + 1;
+  for (int64_t r = (int64_t)blockIdx.x * 256 + threadIdx.x; r < rows; r += (int64_t)gridDim.x * 256) {
+    const int32_t c = __ldg(counts + r);
+    if (c > 0) atomicAdd(&s_bins[count_bin(c)], 1);
   }
-  const int t = lo;
-  int running = 0;
-  for (int64_t base = 0; base < rows; base += 1024) {
-    const int64_t r = base + threadIdx.x;
-    const int flag = r < rows && counts[r] >= t;
-    // exclusive rank of this thread's flag inside the chunk
-    const unsigned ballot = __ballot_sync(0xffffffffu, flag);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    __syncthreads();
-    if (lane == 0) s_warp[warp] = __popc(ballot);
-    __syncthreads();
-    int before = 0, total = 0;
-    for (int w = 0; w < 32; ++w) { const int c = s_warp[w]; before += w < warp ? c : 0; total += c; }
-    if (r < rows) {
-      const int slot = running + before + __popc(ballot & ((1u << lane) - 1u));
-      hot_slot[r] = flag ? slot : -1;
-      if (flag) hot_rows[slot] = (int32_t)r;
-    }
-    running += total;
+  __syncthreads();
+  for (int b = threadIdx.x; b < kCountBins; b += 256)
+    if (s_bins[b]) atomicAdd(bins + b, s_bins[b]);
+}
+
+// *threshold = the lowest bin t such that at most `slots` rows have a count in bin t or above
+__global__ void pick_threshold_kernel(const int32_t *__restrict__ bins, int32_t slots, int32_t *__restrict__ threshold) {
+  __shared__ int32_t s_bins[kCountBins];
+  for (int b = threadIdx.x; b < kCountBins; b += blockDim.x) s_bins[b] = bins[b];
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int t = kCountBins - 1;
+    int64_t reach = s_bins[t];
+    while (t > 0 && reach + s_bins[t - 1] <= slots) { --t; reach += s_bins[t]; }
+    *threshold = t;
   }
-  if (threadIdx.x == 0) *n_hot = running;
+}
+
+__global__ void assign_slots_kernel(const int32_t *__restrict__ counts, int64_t rows, const int32_t *__restrict__ threshold,
+                                    int32_t slots, int32_t *__restrict__ hot_slot, int32_t *__restrict__ hot_rows,
+                                    int32_t *__restrict__ n_hot) {
+  const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= rows) return;
+  int32_t slot = -1;
+  const int32_t c = counts[r];
+  if (c > 0 && count_bin(c) >= *threshold) {
+    slot = atomicAdd(n_hot, 1);
+    if (slot < slots) hot_rows[slot] = (int32_t)r; else slot = -1;
+  }
+  hot_slot[r] = slot;
 }
 
 // fiber_root[f] = the root coordinate of the slice that holds fiber f (a warp per slice).
@@ -190,11 +185,11 @@ __global__ void __launch_bounds__(kHotThreads, kHotCtas) mttkrp_csf_leaf_hot_ker
                                                                                    const int32_t *__restrict__ fiber_root,
                                                                                    const int32_t *__restrict__ hot_slot,
                                                                                    const int32_t *__restrict__ hot_rows,
-                                                                                   const int32_t *__restrict__ n_hot) {
+                                                                                   const int32_t *__restrict__ n_hot, int32_t slots) {
   extern __shared__ double s_acc[];                // slots x R
   const T *const val = static_cast<const T *>(a.val);
   const T *const A = static_cast<const T *>(a.A), *const B = static_cast<const T *>(a.B);
-  const int used = *n_hot;
+  const int used = *n_hot < slots ? *n_hot : slots;
   for (int x = threadIdx.x; x < used * a.R; x += kHotThreads) s_acc[x] = 0.0;
   __syncthreads();
   const unsigned full = 0xffffffffu;
@@ -275,28 +270,33 @@ static comet_status_t leaf_hot(Context *ctx, const ScatterArgs &a, int64_t rows,
   int64_t slots = (int64_t)(kHotBytes / ((size_t)a.R * sizeof(double)));
   if (slots > rows) slots = rows;
   if (slots < 1) return COMET_OK;
-  int32_t *counts = (int32_t *)ctx_alloc(ctx, (size_t)rows * 4, stream);
+  // counts[rows] | bins[kCountBins] | slots in use | threshold: one block, zero-filled at once
+  int32_t *counts = (int32_t *)ctx_alloc(ctx, (size_t)(rows + kCountBins + 2) * 4, stream);
   int32_t *hot_slot = (int32_t *)ctx_alloc(ctx, (size_t)rows * 4, stream);
-  int32_t *hot_rows = (int32_t *)ctx_alloc(ctx, (size_t)(slots + 1) * 4, stream);   // the last word: slots in use
+  int32_t *hot_rows = (int32_t *)ctx_alloc(ctx, (size_t)slots * 4, stream);
   int32_t *fiber_root = (int32_t *)ctx_alloc(ctx, (size_t)a.F * 4, stream);
   comet_status_t st = (counts && hot_slot && hot_rows && fiber_root) ? COMET_OK : COMET_ERR_ALLOC;
   if (st == COMET_OK) {
-    cudaError_t e = cudaMemsetAsync(counts, 0, (size_t)rows * 4, stream);
+    cudaError_t e = cudaMemsetAsync(counts, 0, (size_t)(rows + kCountBins + 2) * 4, stream);
     if (e != cudaSuccess) st = cuda_fail(ctx, e);
   }
   if (st == COMET_OK) {
+    int32_t *bins = counts + rows, *n_hot = bins + kCountBins, *threshold = n_hot + 1;
     const int64_t stride = a.N > kHotSamples ? a.N / kHotSamples : 1;
     const int64_t samples = ceil_div(a.N, stride);
     sample_rows_kernel<<<(unsigned)ceil_div(samples, 256), 256, 0, stream>>>(a.crd2, a.N, stride, counts);
-    select_hot_rows_kernel<<<1, 1024, 0, stream>>>(counts, rows, (int32_t)slots, hot_slot, hot_rows, hot_rows + slots);
+    const int64_t hist_ctas = ceil_div(rows, 256) < 2 * kSmCount ? ceil_div(rows, 256) : 2 * kSmCount;
+    count_histogram_kernel<<<(unsigned)hist_ctas, 256, 0, stream>>>(counts, rows, bins);
+    pick_threshold_kernel<<<1, 256, 0, stream>>>(bins, (int32_t)slots, threshold);
+    assign_slots_kernel<<<(unsigned)ceil_div(rows, 256), 256, 0, stream>>>(counts, rows, threshold, (int32_t)slots, hot_slot, hot_rows, n_hot);
     fiber_root_kernel<<<(unsigned)ceil_div(a.S * 32, 256), 256, 0, stream>>>(a.pos1, a.crd0, a.S, fiber_root);
     auto kernel = mttkrp_csf_leaf_hot_kernel<T>;
     const size_t smem = (size_t)slots * a.R * sizeof(double);
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) st = cuda_fail(ctx, e);
     if (st == COMET_OK) {
-      kernel<<<kHotCtas * kSmCount, kHotThreads, smem, stream>>>(a, fiber_root, hot_slot, hot_rows, hot_rows + slots);
-      ctx->launches += 4;
+      kernel<<<kHotCtas * kSmCount, kHotThreads, smem, stream>>>(a, fiber_root, hot_slot, hot_rows, n_hot, (int32_t)slots);
+      ctx->launches += 6;
       e = cudaGetLastError();
       if (e != cudaSuccess) st = cuda_fail(ctx, e);
       else *done = 1;
