@@ -275,6 +275,20 @@ struct CsfPolicy {
   }
   // LEVEL1: out[row, :] += tac * arow (atomic), tac = 0
   __device__ __forceinline__ void scatter_fiber(int32_t row) {
+    if constexpr (CPL == 1 && VEC == 2) {
+      // A lane holds two ADJACENT columns. Added as they lie, each of the two requests would touch every other
+      // pair of the row: twice the 32-byte sectors for L2, which processes atomic adds sector by sector. The
+      // lanes exchange their products so that one request covers the first LPN columns and the other the rest.
+      const double p0 = tac[0][0] * (double)arow[0][0], p1 = tac[0][1] * (double)arow[0][1];
+      tac[0][0] = 0.0; tac[0][1] = 0.0;
+      const int lo_src = ln.g >> 1, hi_src = (LPN >> 1) + (ln.g >> 1);
+      const double l0 = __shfl_sync(ln.mask, p0, lo_src, LPN), l1 = __shfl_sync(ln.mask, p1, lo_src, LPN);
+      const double h0 = __shfl_sync(ln.mask, p0, hi_src, LPN), h1 = __shfl_sync(ln.mask, p1, hi_src, LPN);
+      double *base = reinterpret_cast<double *>(a.out) + (int64_t)row * a.ldo + (ln.col0 - ln.g * VEC);
+      atomicAdd(base + ln.g, (ln.g & 1) ? l1 : l0);
+      atomicAdd(base + LPN + ln.g, (ln.g & 1) ? h1 : h0);
+      return;
+    }
     double *dst = reinterpret_cast<double *>(a.out) + (int64_t)row * a.ldo + ln.col0;
 #pragma unroll
     for (int t = 0; t < CPL; ++t)

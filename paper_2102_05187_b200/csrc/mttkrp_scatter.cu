@@ -100,11 +100,12 @@ __global__ void __launch_bounds__(kScatterThreads) mttkrp_coo_scatter_kernel(con
 constexpr int kHotThreads = 512;
 constexpr int kHotCtas = 2;                        // CTAs per SM
 constexpr int kHotChunk = 1024;                    // entries per warp and step
-// Shared memory per CTA for the popular rows: 128 rows of 32 columns. Measured on config 5 (leaf frequencies
-// (k + 100)^-1.5 over 200,000 rows): 32 rows 16.6 ms, 100 rows 8.45, 200 rows 8.50, 400 rows 9.19 (an add in shared
-// memory is a compare-and-swap loop of about a dozen instructions, an add in L2 one instruction: past the rows
-// that L2 serialises, more slots cost more than they save).
-constexpr size_t kHotBytes = 32 * 1024;
+// Shared memory per CTA for the popular rows: 256 rows of 32 columns. Measured on config 5 (leaf frequencies
+// (k + 100)^-1.5 over 200,000 rows): 32 rows 16.6 ms, 128 rows 6.75 to 8.9 ms depending on where the output
+// matrix happened to be allocated (the next few hundred rows still collide in L2), 256 rows 6.87 ms wherever it
+// was, 384 rows 7.16 ms (an add in shared memory is a compare-and-swap loop of about a dozen instructions, an
+// add in L2 one instruction: past the rows that L2 serialises, more slots cost more than they save).
+constexpr size_t kHotBytes = 64 * 1024;
 constexpr int64_t kHotMaxRows = 1ll << 24;         // two 32-bit words per output row are allocated for the call
 constexpr int64_t kHotSamples = 1ll << 22;
 
