@@ -302,7 +302,7 @@ def per_kernel(comet, handle, steps, warm, peak, peak_kind="measured", scale=1.0
             "roofline": roofline_obj(nbytes, med, peak, peak_kind, f"comet_{op} ({fmt}) on {case.name}"),
             "pack_roofline": roofline_obj(pbytes, pmed, peak, peak_kind, f"comet_pack -> {fmt} on {case.name}"),
         })
-        if op == "mttkrp" and fmt == "csf":
+        if op == "mttkrp":
             # the two other modes of the SAME packed tensor (atomic accumulation, nothing re-packed)
             for mode in (1, 2):
                 Fm = [synth.random_dense((d, case.R), case.seed, 70 + m, device="cuda") for m, d in enumerate(case.dims)]
@@ -316,7 +316,7 @@ def per_kernel(comet, handle, steps, warm, peak, peak_kind="measured", scale=1.0
                     "frac_of_8000": round(nbytes / med / 1e6 / NOMINAL_GBS, 4),
                     "frac_of_peak": round(nbytes / med / 1e6 / peak, 4), "GFLOPs": round(flops / med / 1e6, 1),
                     "l2": "inputs larger than L2", "accumulation": "atomic adds (order not fixed)",
-                    "roofline": roofline_obj(nbytes, med, peak, peak_kind, f"comet_mttkrp mode {mode + 1} of the root-packed csf"),
+                    "roofline": roofline_obj(nbytes, med, peak, peak_kind, f"comet_mttkrp mode {mode + 1} of the root-packed {fmt}"),
                 })
                 del Fm, Am
         del T

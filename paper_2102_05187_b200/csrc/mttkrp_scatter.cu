@@ -176,12 +176,12 @@ __global__ void fiber_root_kernel(const int32_t *__restrict__ pos1, const int32_
   for (int64_t f = (int64_t)__ldg(pos1 + s) + (threadIdx.x & 31); f < (int64_t)__ldg(pos1 + s + 1); f += 32) fiber_root[f] = i;
 }
 
-// CSF, output mode at the leaf level: out[k, :] += val * (A[i, :] * B[j, :]), one row add per entry; rows with a
-// slot are added in shared memory. A warp takes kHotChunk consecutive ENTRIES per step. Its lanes first work
+// CSF with the output mode at the leaf level, out[k, :] += val * (A[i, :] * B[j, :]), or (COO) a sorted coordinate
+// list with the output mode anywhere but first: one row add per entry; rows with a slot are added in shared memory. A warp takes kHotChunk consecutive ENTRIES per step. Its lanes first work
 // entry-parallel: each reads one entry's coordinate, value and slot and finds the entry's fiber in a window of 32
 // fiber ends held one per lane (so the loads of 32 entries are in flight together, whatever the fiber lengths);
 // then the lanes are the columns (R > 32: several sweeps) and the 32 entries are handed round with shuffles.
-template <class T>
+template <class T, bool COO>
 __global__ void __launch_bounds__(kHotThreads, kHotCtas) mttkrp_csf_leaf_hot_kernel(const ScatterArgs a,
                                                                                    const int32_t *__restrict__ fiber_root,
                                                                                    const int32_t *__restrict__ hot_slot,
@@ -200,33 +200,46 @@ __global__ void __launch_bounds__(kHotThreads, kHotCtas) mttkrp_csf_leaf_hot_ker
   for (int64_t chunk = (int64_t)blockIdx.x * (kHotThreads / 32) + (threadIdx.x >> 5); chunk < chunks; chunk += warps) {
     const int64_t p0 = chunk * kHotChunk;
     const int64_t p1 = p0 + kHotChunk < a.N ? p0 + kHotChunk : a.N;
-    int64_t lo = 0, hi = a.F;                      // the fiber of entry p0: the largest f with pos2[f] <= p0
-    while (hi - lo > 1) {
-      const int64_t mid = (lo + hi) >> 1;
-      if ((int64_t)__ldg(a.pos2 + mid) <= p0) lo = mid; else hi = mid;
+    int64_t fw = 0;                                // CSF: the window of fibers fw .. fw + 31, one per lane
+    int32_t w_end = 0x7fffffff, w_i = 0, w_j = 0;
+    if constexpr (!COO) {
+      int64_t lo = 0, hi = a.F;                    // the fiber of entry p0: the largest f with pos2[f] <= p0
+      while (hi - lo > 1) {
+        const int64_t mid = (lo + hi) >> 1;
+        if ((int64_t)__ldg(a.pos2 + mid) <= p0) lo = mid; else hi = mid;
+      }
+      fw = lo;
+      w_end = fw + lane < a.F ? __ldg(a.pos2 + fw + lane + 1) : 0x7fffffff;
+      w_i = fw + lane < a.F ? __ldg(fiber_root + fw + lane) : 0;
+      w_j = fw + lane < a.F ? __ldg(a.crd1 + fw + lane) : 0;
     }
-    int64_t fw = lo;                               // the window: fibers fw .. fw + 31, one per lane
-    int32_t w_end = fw + lane < a.F ? __ldg(a.pos2 + fw + lane + 1) : 0x7fffffff;
-    int32_t w_i = fw + lane < a.F ? __ldg(fiber_root + fw + lane) : 0, w_j = fw + lane < a.F ? __ldg(a.crd1 + fw + lane) : 0;
     for (int64_t pb = p0; pb < p1; pb += 32) {
       const int cnt = p1 - pb < 32 ? (int)(p1 - pb) : 32;
       const int32_t p = (int32_t)pb + lane;
-      const int32_t kk = lane < cnt ? __ldg(a.crd2 + p) : 0;
+      // the output coordinate: the leaf's (CSF) or the one listed first (COO: crd0 / crd1 / crd2 = output, A's, B's)
+      const int32_t kk = lane < cnt ? __ldg((COO ? a.crd0 : a.crd2) + p) : 0;
       const double vv = lane < cnt ? (double)ld_stream(val + p) : 0.0;
       const int32_t qq = lane < cnt ? __ldg(hot_slot + kk) : -1;
       uint32_t row_a = 0, row_b = 0;               // element offsets of this entry's rows of A and B (32 bits: the host checks the sizes)
-      bool found = lane >= cnt;
-      while (true) {                               // this entry's fiber: the ends at or below p, counted over the window
-        int u = 0;
+      if constexpr (COO) {
+        if (lane < cnt) {
+          row_a = (uint32_t)__ldg(a.crd1 + p) * (uint32_t)a.lda;
+          row_b = (uint32_t)__ldg(a.crd2 + p) * (uint32_t)a.ldb;
+        }
+      } else {
+        bool found = lane >= cnt;
+        while (true) {                             // this entry's fiber: the ends at or below p, counted over the window
+          int u = 0;
 #pragma unroll
-        for (int t = 0; t < 32; ++t) u += __shfl_sync(full, w_end, t) <= p;
-        const int32_t ci = __shfl_sync(full, w_i, u & 31), cj = __shfl_sync(full, w_j, u & 31);
-        if (!found && u < 32) { row_a = (uint32_t)ci * (uint32_t)a.lda; row_b = (uint32_t)cj * (uint32_t)a.ldb; found = true; }
-        if (__all_sync(full, found)) break;
-        fw += 32;                                  // entries beyond the window's last fiber: next window
-        w_end = fw + lane < a.F ? __ldg(a.pos2 + fw + lane + 1) : 0x7fffffff;
-        w_i = fw + lane < a.F ? __ldg(fiber_root + fw + lane) : 0;
-        w_j = fw + lane < a.F ? __ldg(a.crd1 + fw + lane) : 0;
+          for (int t = 0; t < 32; ++t) u += __shfl_sync(full, w_end, t) <= p;
+          const int32_t ci = __shfl_sync(full, w_i, u & 31), cj = __shfl_sync(full, w_j, u & 31);
+          if (!found && u < 32) { row_a = (uint32_t)ci * (uint32_t)a.lda; row_b = (uint32_t)cj * (uint32_t)a.ldb; found = true; }
+          if (__all_sync(full, found)) break;
+          fw += 32;                                // entries beyond the window's last fiber: next window
+          w_end = fw + lane < a.F ? __ldg(a.pos2 + fw + lane + 1) : 0x7fffffff;
+          w_i = fw + lane < a.F ? __ldg(fiber_root + fw + lane) : 0;
+          w_j = fw + lane < a.F ? __ldg(a.crd1 + fw + lane) : 0;
+        }
       }
       // where the entry's term goes: a slot's row in shared memory (bit 31 set) or the output row's element offset
       const uint32_t dest = qq >= 0 ? 0x80000000u | (uint32_t)(qq * a.R) : (uint32_t)kk * (uint32_t)a.ldacc;
@@ -255,11 +268,11 @@ __global__ void __launch_bounds__(kHotThreads, kHotCtas) mttkrp_csf_leaf_hot_ker
   }
 }
 
-// The leaf-mode product with the popular rows in shared memory; *done = 0 when the shape is not this path's
-// (the caller then runs the general kernel).
+// The per-entry product (CSF leaf mode, or any non-root mode of a COO tensor) with the popular rows in shared
+// memory; *done = 0 when the shape is not this path's (the caller then runs the general kernel).
 template <class T>
-static comet_status_t leaf_hot(Context *ctx, const ScatterArgs &a, int64_t rows, int64_t a_rows, int64_t b_rows, int *done,
-                               cudaStream_t stream) {
+static comet_status_t entries_hot(Context *ctx, const ScatterArgs &a, bool coo, int64_t rows, int64_t a_rows, int64_t b_rows,
+                                  int *done, cudaStream_t stream) {
   *done = 0;
   const char *force = getenv("COMET_MTTKRP_HOT_ROWS");      // tests: "1" takes this path on any size, "0" never
   if (force && force[0] == '0') return COMET_OK;
@@ -271,12 +284,13 @@ static comet_status_t leaf_hot(Context *ctx, const ScatterArgs &a, int64_t rows,
   int64_t slots = (int64_t)(kHotBytes / ((size_t)a.R * sizeof(double)));
   if (slots > rows) slots = rows;
   if (slots < 1) return COMET_OK;
+  const int32_t *out_crd = coo ? a.crd0 : a.crd2;
   // counts[rows] | bins[kCountBins] | slots in use | threshold: one block, zero-filled at once
   int32_t *counts = (int32_t *)ctx_alloc(ctx, (size_t)(rows + kCountBins + 2) * 4, stream);
   int32_t *hot_slot = (int32_t *)ctx_alloc(ctx, (size_t)rows * 4, stream);
   int32_t *hot_rows = (int32_t *)ctx_alloc(ctx, (size_t)slots * 4, stream);
-  int32_t *fiber_root = (int32_t *)ctx_alloc(ctx, (size_t)a.F * 4, stream);
-  comet_status_t st = (counts && hot_slot && hot_rows && fiber_root) ? COMET_OK : COMET_ERR_ALLOC;
+  int32_t *fiber_root = coo ? nullptr : (int32_t *)ctx_alloc(ctx, (size_t)a.F * 4, stream);
+  comet_status_t st = (counts && hot_slot && hot_rows && (coo || fiber_root)) ? COMET_OK : COMET_ERR_ALLOC;
   if (st == COMET_OK) {
     cudaError_t e = cudaMemsetAsync(counts, 0, (size_t)(rows + kCountBins + 2) * 4, stream);
     if (e != cudaSuccess) st = cuda_fail(ctx, e);
@@ -285,19 +299,23 @@ static comet_status_t leaf_hot(Context *ctx, const ScatterArgs &a, int64_t rows,
     int32_t *bins = counts + rows, *n_hot = bins + kCountBins, *threshold = n_hot + 1;
     const int64_t stride = a.N > kHotSamples ? a.N / kHotSamples : 1;
     const int64_t samples = ceil_div(a.N, stride);
-    sample_rows_kernel<<<(unsigned)ceil_div(samples, 256), 256, 0, stream>>>(a.crd2, a.N, stride, counts);
+    sample_rows_kernel<<<(unsigned)ceil_div(samples, 256), 256, 0, stream>>>(out_crd, a.N, stride, counts);
     const int64_t hist_ctas = ceil_div(rows, 256) < 2 * kSmCount ? ceil_div(rows, 256) : 2 * kSmCount;
     count_histogram_kernel<<<(unsigned)hist_ctas, 256, 0, stream>>>(counts, rows, bins);
     pick_threshold_kernel<<<1, 256, 0, stream>>>(bins, (int32_t)slots, threshold);
     assign_slots_kernel<<<(unsigned)ceil_div(rows, 256), 256, 0, stream>>>(counts, rows, threshold, (int32_t)slots, hot_slot, hot_rows, n_hot);
-    fiber_root_kernel<<<(unsigned)ceil_div(a.S * 32, 256), 256, 0, stream>>>(a.pos1, a.crd0, a.S, fiber_root);
-    auto kernel = mttkrp_csf_leaf_hot_kernel<T>;
+    ctx->launches += 4;
+    if (!coo) {
+      fiber_root_kernel<<<(unsigned)ceil_div(a.S * 32, 256), 256, 0, stream>>>(a.pos1, a.crd0, a.S, fiber_root);
+      ctx->launches += 1;
+    }
+    auto kernel = coo ? mttkrp_csf_leaf_hot_kernel<T, true> : mttkrp_csf_leaf_hot_kernel<T, false>;
     const size_t smem = (size_t)slots * a.R * sizeof(double);
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) st = cuda_fail(ctx, e);
     if (st == COMET_OK) {
       kernel<<<kHotCtas * kSmCount, kHotThreads, smem, stream>>>(a, fiber_root, hot_slot, hot_rows, n_hot, (int32_t)slots);
-      ctx->launches += 6;
+      ctx->launches += 1;
       e = cudaGetLastError();
       if (e != cudaSuccess) st = cuda_fail(ctx, e);
       else *done = 1;
@@ -369,9 +387,9 @@ comet_status_t mttkrp_scatter(Context *ctx, int dtype, int kind, const int32_t *
   }
   if (N > 0) {
     int done = 0;
-    if (kind == 2) {
-      comet_status_t st = dtype == COMET_F32 ? leaf_hot<float>(ctx, a, rows, a_rows, b_rows, &done, stream)
-                                              : leaf_hot<double>(ctx, a, rows, a_rows, b_rows, &done, stream);
+    if (kind == 2 || kind == 0) {                   // one add per entry: the popular output rows go to shared memory
+      comet_status_t st = dtype == COMET_F32 ? entries_hot<float>(ctx, a, kind == 0, rows, a_rows, b_rows, &done, stream)
+                                              : entries_hot<double>(ctx, a, kind == 0, rows, a_rows, b_rows, &done, stream);
       if (st != COMET_OK) return st;
     }
     if (!done) {

@@ -432,37 +432,41 @@ def _skewed_leaf_coo(dims, nnz, seed):
 
 @pytest.mark.parametrize("dims,nnz", [((40, 30, 500), 20000), ((7, 9, 20), 700), ((300, 200, 3000), 60000)])
 @pytest.mark.parametrize("dtype", ["f64", "f32"])
-def test_mttkrp_leaf_mode_with_popular_rows_in_shared_memory(dims, nnz, dtype, monkeypatch):
-    """The leaf-mode kernel that keeps the most popular output rows in shared memory, forced on small tensors
-    (by default only large ones take it): fewer rows than slots, more rows than slots, R below, at and above a
-    warp's width, entries that straddle the 32-fiber window."""
+@pytest.mark.parametrize("attr,modes", [((CU, CU, CU), (2,)), ((CN, S, S), (1, 2))])
+def test_mttkrp_with_popular_rows_in_shared_memory(dims, nnz, dtype, attr, modes, monkeypatch):
+    """The per-entry kernel that keeps the most popular output rows in shared memory (CSF: leaf mode; COO: both
+    non-root modes), forced on small tensors (by default only large ones take it): fewer rows than slots, more
+    rows than slots, R below, at and above a warp's width, entries that straddle the 32-fiber window."""
     monkeypatch.setenv("COMET_MTTKRP_HOT_ROWS", "1")
     c, v = _skewed_leaf_coo(dims, nnz, 11)
     if dtype == "f32":
         v = v.astype(np.float32).astype(np.float64)
-    pk = oracle.pack(c, v, dims, (0, 1, 2), (CU, CU, CU))
+    pk = oracle.pack(c, v, dims, (0, 1, 2), attr)
     if dtype == "f32":
         pos = [dev(p, torch.int32) if p.size else None for p in pk.pos]
         crd = [dev(q, torch.int32) if q.size else None for q in pk.crd]
         X = comet.SpTensor.from_arrays(pk.dims, pk.mode_order, pk.attr, pos, crd, dev(pk.val.astype(np.float32)))
     else:
         X = upload_packed(pk)
+    tdt = torch.float32 if dtype == "f32" else torch.float64
     for R in (1, 5, 32, 40, 64):
         F = [synth.random_dense((d, R), 11, 60 + m).numpy() for m, d in enumerate(dims)]
         if dtype == "f32":
             F = [f.astype(np.float32).astype(np.float64) for f in F]
-        want, norm = oracle.mttkrp(c, v, dims, 2, F)
-        tdt = torch.float32 if dtype == "f32" else torch.float64
-        out = torch.full((dims[2], R), float("nan"), dtype=tdt, device="cuda")
-        comet.mttkrp(X, 2, [dev(F[0]).to(tdt), dev(F[1]).to(tdt), None], out)
-        assert_close(out.double(), want, norm, tol=FP64_TOL if dtype == "f64" else 4e-7, what=f"leaf mttkrp {dtype} R={R}")
-    monkeypatch.setenv("COMET_MTTKRP_HOT_ROWS", "0")
-    out0 = torch.full((dims[2], 5), float("nan"), dtype=torch.float64, device="cuda")
-    if dtype == "f64":
+        for mode in modes:
+            want, norm = oracle.mttkrp(c, v, dims, mode, F)
+            out = torch.full((dims[mode], R), float("nan"), dtype=tdt, device="cuda")
+            comet.mttkrp(X, mode, [None if m == mode else dev(f).to(tdt) for m, f in enumerate(F)], out)
+            assert_close(out.double(), want, norm, tol=FP64_TOL if dtype == "f64" else 4e-7,
+                         what=f"mttkrp {attr} mode {mode} {dtype} R={R}")
+    if dtype == "f64":                                   # the general kernel on the same input
+        monkeypatch.setenv("COMET_MTTKRP_HOT_ROWS", "0")
         F = [synth.random_dense((d, 5), 11, 60 + m).numpy() for m, d in enumerate(dims)]
-        want, norm = oracle.mttkrp(c, v, dims, 2, F)
-        comet.mttkrp(X, 2, [dev(F[0]), dev(F[1]), None], out0)
-        assert_close(out0, want, norm, what="leaf mttkrp, general kernel")
+        for mode in modes:
+            want, norm = oracle.mttkrp(c, v, dims, mode, F)
+            out0 = torch.full((dims[mode], 5), float("nan"), dtype=torch.float64, device="cuda")
+            comet.mttkrp(X, mode, [None if m == mode else dev(f) for m, f in enumerate(F)], out0)
+            assert_close(out0, want, norm, what=f"mttkrp {attr} mode {mode}, general kernel")
 
 
 def test_mttkrp_non_root_strided_output_and_integers():
