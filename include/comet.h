@@ -193,6 +193,20 @@ comet_status_t comet_spmv(comet_handle_t handle, const comet_sptensor_t *A, cons
 comet_status_t comet_spmm(comet_handle_t handle, const comet_sptensor_t *A, const void *B, int64_t R, int64_t ldb,
                           void *C, int64_t ldc, void *stream);
 
+/* The SpMM path from HOST buffers in one call: copies the COO entries and B to the device, packs the matrix
+ * to CSR ([D,CU], comet_pack), multiplies (comet_spmm) and copies C back; returns when C has landed in h_C.
+ * The transfers overlap: B and C travel in column chunks of 256 bytes per row on two copy streams of the handle,
+ * so C's first chunk leaves while the rest of B still arrives (COMET_HOST_CHUNK_BYTES=n changes the chunk width,
+ * 0 = one chunk). Every h_ pointer is HOST memory and should be pinned (page-locked): with pageable memory the
+ * copies are staged by the driver and nothing overlaps. Device buffers come from the handle's allocator and are
+ * released before the call returns.
+ *   h_dims[2]      rows, columns;   h_row / h_col / h_val: nnz coordinates (int32) and values, any order, distinct cells
+ *   h_B            columns x R, row-major, leading dimension ldb;   h_C: rows x R, leading dimension ldc, every row written
+ * Errors as for comet_pack and comet_spmm. */
+comet_status_t comet_spmm_from_host(comet_handle_t handle, const int64_t *h_dims, int64_t nnz, const int32_t *h_row,
+                                    const int32_t *h_col, const void *h_val, comet_dtype_t dtype, const void *h_B,
+                                    int64_t ldb, int64_t R, void *h_C, int64_t ldc, void *stream);
+
 /* TTV  Y = X x_n v  (SpTTV definition; `mode` = n, 0-based, must be the mode of X's LAST level).
  * X: 3 levels, [CU,CU,CU] (CSF) or [CN,S,S] (sorted COO), or 4 levels, [CU,CU,CU,CU] (CSF) or [CN,S,S,S] (sorted
  * COO; its symbolic call derives the compressed levels by packing the entries once more). The result

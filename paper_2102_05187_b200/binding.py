@@ -51,7 +51,7 @@ EXPORTS = [
     "comet_pack",
     "comet_sptensor_free", "comet_validate", "comet_spmv", "comet_spmm", "comet_ttv_symbolic", "comet_ttv",
     "comet_ttm_symbolic", "comet_ttm", "comet_mttkrp", "comet_spmv_static", "comet_pack_ex", "comet_ttm_symbolic_ex", "comet_reorder",
-    "comet_elementwise_mul",
+    "comet_elementwise_mul", "comet_spmm_from_host",
 ]
 
 
@@ -452,29 +452,23 @@ def reorder(coords, dims, iterations: int = 5, handle: Handle | None = None):
     return labels
 
 
-_copy_stream = None
-
-
 def spmm_from_host(h_coords, h_val, dims, h_B, h_out, handle: Handle | None = None):
-    """The whole SpMM path from HOST buffers: copies the COO entries and B to the device (pinned host
-    tensors make the copies asynchronous), packs to CSR, multiplies, and copies C back into `h_out`.
-    B travels on a second stream, so the packing kernels run while B is still crossing the bus; the
-    multiplication waits for it. Returns after the result has landed in `h_out`."""
-    global _copy_stream
+    """comet_spmm_from_host: the whole SpMM path from HOST buffers (pinned host tensors make the copies
+    asynchronous): COO entries and B in, CSR packing, multiplication, C back into `h_out`, with B and C
+    travelling in column chunks so that the two directions of the bus overlap. Returns after the result has
+    landed in `h_out`."""
     handle = handle or default_handle()
-    cur = torch.cuda.current_stream()
-    if _copy_stream is None or _copy_stream.device != cur.device:
-        _copy_stream = torch.cuda.Stream(device=cur.device)
-    coords = [c.to("cuda", non_blocking=True) for c in h_coords]
-    val = h_val.to("cuda", non_blocking=True)
-    _copy_stream.wait_stream(cur)                     # the bus serves the COO entries first
-    with torch.cuda.stream(_copy_stream):
-        B = h_B.to("cuda", non_blocking=True)
-    A = pack(coords, val, dims, (0, 1), (D, CU), handle)
-    cur.wait_stream(_copy_stream)
-    B.record_stream(cur)
-    C_dev = spmm(A, B)
-    h_out.copy_(C_dev, non_blocking=True)
-    cur.synchronize()
-    A.free()
+    tensors = list(h_coords) + [h_val, h_B, h_out]
+    if any(t.is_cuda for t in tensors):
+        raise ValueError("spmm_from_host takes host tensors")
+    assert len(h_coords) == 2 and all(c.dtype == torch.int32 and c.is_contiguous() for c in h_coords)
+    assert h_val.is_contiguous() and h_B.dim() == 2 and h_out.dim() == 2 and h_B.stride(1) == 1 and h_out.stride(1) == 1
+    assert h_B.dtype == h_val.dtype == h_out.dtype
+    R = int(h_B.shape[1])
+    assert tuple(h_out.shape) == (int(dims[0]), R) and int(h_B.shape[0]) == int(dims[1])
+    h_dims = (C.c_int64 * 2)(int(dims[0]), int(dims[1]))
+    st = handle.lib.comet_spmm_from_host(handle._h, h_dims, C.c_int64(h_val.numel()), _ptr(h_coords[0]), _ptr(h_coords[1]),
+                                         _ptr(h_val), C.c_int32(_dtype_code(h_val)), _ptr(h_B), C.c_int64(h_B.stride(0)),
+                                         C.c_int64(R), _ptr(h_out), C.c_int64(h_out.stride(0)), _stream_ptr())
+    handle.check(st, "comet_spmm_from_host")
     return h_out

@@ -24,7 +24,13 @@ struct Context {
   cudaStream_t last_stream;               // stream of the latest call that used the scratch or the counters
   bool has_last_stream;
   bool counters_dirty;                    // a CUDA call failed: the device counters may not be back at zero
+  bool has_copy_streams;                  // comet_spmm_from_host: its two copy streams and events, made on first use
+  cudaStream_t copy_in, copy_out;
+  cudaEvent_t copy_event[2 * 8 + 2];
 };
+constexpr int kCopyChunks = 8;            // most column chunks of comet_spmm_from_host
+constexpr int kCopyEvents = 2 * kCopyChunks + 2;
+void host_streams_destroy(Context *ctx);
 
 // Grows the cached scratch buffer to at least `bytes` and returns it (NULL on allocation failure).
 void *scratch_get(Context *ctx, size_t bytes, cudaStream_t stream);

@@ -77,6 +77,7 @@ extern "C" comet_status_t comet_create(comet_handle_t *handle, const comet_alloc
   ctx->has_last_stream = false;
   ctx->last_stream = nullptr;
   ctx->counters_dirty = false;
+  ctx->has_copy_streams = false;
   ctx->launches = 0;
   ctx->scratch = nullptr;
   ctx->scratch_bytes = 0;
@@ -105,6 +106,7 @@ extern "C" comet_status_t comet_destroy(comet_handle_t handle) {
   if (!handle) return COMET_OK;
   Context *ctx = reinterpret_cast<Context *>(handle);
   cudaDeviceSynchronize();
+  comet::host_streams_destroy(ctx);
   if (ctx->scratch) comet::ctx_free(ctx, ctx->scratch, nullptr);
   if (ctx->h_pinned) cudaFreeHost(ctx->h_pinned);
   if (ctx->d_status) cudaFree(ctx->d_status);

@@ -504,10 +504,55 @@ def test_spmm_from_host_buffers():
     h_coords = [t.pin_memory() for t in case.coords]
     h_val, h_B = case.val.pin_memory(), case.dense["B"].pin_memory()
     h_C = torch.full((case.dims[0], case.R), float("nan"), dtype=torch.float64).pin_memory()
-    for _ in range(2):                                  # the second call reuses the side stream
+    for _ in range(2):                                  # the second call reuses the copy streams
         h_C.fill_(float("nan"))
         comet.spmm_from_host(h_coords, h_val, case.dims, h_B, h_C)
         assert_close(h_C, want, norm, what="spmm_from_host")
+
+
+@pytest.mark.parametrize("R,chunk_bytes", [(64, None), (40, None), (5, None), (64, "128"), (64, "0"), (33, "64")])
+@pytest.mark.parametrize("dtype", ["f64", "f32"])
+def test_spmm_from_host_column_chunks(R, chunk_bytes, dtype, monkeypatch):
+    """comet_spmm_from_host with B and C cut into column chunks: even and ragged chunk counts, one chunk, strided
+    host matrices (leading dimension above R, padding untouched), pageable as well as pinned memory, an empty
+    matrix, and a bad coordinate reported as a status."""
+    if chunk_bytes is None:
+        monkeypatch.delenv("COMET_HOST_CHUNK_BYTES", raising=False)
+    else:
+        monkeypatch.setenv("COMET_HOST_CHUNK_BYTES", chunk_bytes)
+    tdt = torch.float32 if dtype == "f32" else torch.float64
+    dims = (300, 200)
+    coords, val = synth.random_coo(dims, 4000, 21)
+    Bm = synth.random_dense((dims[1], R), 21, 3)
+    if dtype == "f32":
+        val, Bm = val.float().double(), Bm.float().double()
+    want, norm = oracle.spmm(_np(coords), val.numpy(), dims, Bm.numpy())
+    tol = FP64_TOL if dtype == "f64" else 4e-7
+    h_coords = [t.pin_memory() for t in coords]
+    h_val = val.to(tdt).pin_memory()
+    h_Bbuf = torch.full((dims[1], R + 3), 5.0, dtype=tdt).pin_memory()
+    h_Bbuf[:, :R] = Bm.to(tdt)
+    h_Cbuf = torch.full((dims[0], R + 2), 7.0, dtype=tdt).pin_memory()
+    comet.spmm_from_host(h_coords, h_val, dims, h_Bbuf[:, :R], h_Cbuf[:, :R])
+    assert_close(h_Cbuf[:, :R].double(), want, norm, tol=tol, what=f"spmm_from_host R={R} chunks of {chunk_bytes}")
+    assert bool((h_Cbuf[:, R:] == 7.0).all())
+    # pageable host memory: correct, only slower
+    p_C = torch.full((dims[0], R), float("nan"), dtype=tdt)
+    comet.spmm_from_host([t.clone() for t in coords], val.to(tdt), dims, Bm.to(tdt).contiguous(), p_C)
+    assert_close(p_C.double(), want, norm, tol=tol, what="spmm_from_host, pageable memory")
+    # no entries: C = 0
+    e_C = torch.full((dims[0], R), float("nan"), dtype=tdt).pin_memory()
+    empty = [torch.zeros(0, dtype=torch.int32).pin_memory() for _ in range(2)]
+    comet.spmm_from_host(empty, torch.zeros(0, dtype=tdt).pin_memory(), dims, h_Bbuf[:, :R], e_C)
+    assert bool((e_C == 0).all())
+    # a coordinate outside the matrix is a status, and the handle keeps working
+    bad = [h_coords[0].clone(), h_coords[1].clone()]
+    bad[1][7] = dims[1]
+    with pytest.raises(comet.CometError) as err:
+        comet.spmm_from_host(bad, h_val, dims, h_Bbuf[:, :R], h_Cbuf[:, :R])
+    assert err.value.status == -3
+    comet.spmm_from_host(h_coords, h_val, dims, h_Bbuf[:, :R], h_Cbuf[:, :R])
+    assert_close(h_Cbuf[:, :R].double(), want, norm, tol=tol, what="spmm_from_host after an error")
 
 
 def test_results_are_reproducible_run_to_run():
