@@ -245,29 +245,44 @@ __global__ void __launch_bounds__(kBlockThreads) heavy_tiles_kernel(const HeavyA
   }
 }
 
-// C[row, :] = the sum of the row's slots in slot order (a thread per column, a long row per step). The loads of
-// sixteen slots are issued together; the additions keep the slot order.
+// C[row, :] = the sum of the row's slots, a long row per CTA and step. The 256 threads are G groups of R columns
+// (G = 256 / R, at least 1); group g adds the slots g, g + G, g + 2G, ... in that order (up to sixteen loads in
+// flight), and the groups' sums are then added in group order: a fixed order, so results stay bit-identical from
+// run to run.
 template <class T>
 __global__ void __launch_bounds__(kBlockThreads) heavy_fixup_kernel(const HeavyArgs a) {
+  __shared__ double s_part[kBlockThreads];
   const int32_t H = __ldcg(a.counters + 0);
-  const int64_t total = (int64_t)H * a.R;
   T *C = static_cast<T *>(a.C);
-  for (int64_t idx = (int64_t)blockIdx.x * kBlockThreads + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * kBlockThreads) {
-    const int32_t h = (int32_t)(idx / a.R);
-    const int32_t c = (int32_t)(idx - (int64_t)h * a.R);
+  const int R = a.R;
+  const int G = R < kBlockThreads ? kBlockThreads / R : 1;      // R is a power of two here (the shapes of the long-row path)
+  const int g = threadIdx.x / R;
+  for (int32_t h = blockIdx.x; h < H; h += gridDim.x) {
     const int32_t n = a.row_nt[h];
-    const double *src = a.carry_val + (int64_t)a.row_slot0[h] * a.carry_ld + c;
-    double sum = 0.0;
-    int32_t t = 0;
-    for (; t + 16 <= n; t += 16) {
-      double v[16];
+    for (int c = threadIdx.x % R; c < R; c += kBlockThreads) {  // one sweep unless R > 256
+      const double *src = a.carry_val + (int64_t)a.row_slot0[h] * a.carry_ld + c;
+      double sum = 0.0;
+      int32_t t = g;
+      for (; t + 15 * G < n; t += 16 * G) {
+        double v[16];
 #pragma unroll
-      for (int u = 0; u < 16; ++u) v[u] = __ldcs(src + (int64_t)(t + u) * a.carry_ld);
+        for (int u = 0; u < 16; ++u) v[u] = __ldcs(src + (int64_t)(t + u * G) * a.carry_ld);
 #pragma unroll
-      for (int u = 0; u < 16; ++u) sum += v[u];
+        for (int u = 0; u < 16; ++u) sum += v[u];
+      }
+      for (; t < n; t += G) sum += __ldcs(src + (int64_t)t * a.carry_ld);
+      if (G > 1) {
+        __syncthreads();                                        // the sums of the row before have been read
+        s_part[threadIdx.x] = sum;
+        __syncthreads();
+        if (g == 0) {
+          for (int x = 1; x < G; ++x) sum += s_part[x * R + c];
+          C[(int64_t)a.hrow[h] * a.ldc + c] = (T)sum;
+        }
+      } else {
+        C[(int64_t)a.hrow[h] * a.ldc + c] = (T)sum;
+      }
     }
-    for (; t < n; ++t) sum += __ldcs(src + (int64_t)t * a.carry_ld);
-    C[(int64_t)a.hrow[h] * a.ldc + c] = (T)sum;
   }
 }
 
