@@ -256,6 +256,26 @@ def test_pack_sum_duplicates_is_a_no_op_on_distinct_cells_and_handles_empty_and_
     assert np.array_equal(got.val.cpu().numpy(), want.val.astype(np.float32))   # summed in double, rounded once
 
 
+@pytest.mark.parametrize("dtype", [torch.float64, torch.float32])
+def test_pack_of_extent_one_tensors_and_of_keys_that_fill_a_whole_number_of_passes(dtype):
+    """Keys of zero bits (every extent 1: no sort pass runs), of exactly 8 and 16 bits (the last pass is a full
+    digit), and of 9 bits (a last pass over a single bit), fp64 values (gathered through the sorted indices) and
+    fp32 ones (carried through the sort)."""
+    one = [torch.zeros(1, dtype=torch.int32, device="cuda")] * 3
+    t = comet.pack(one, torch.tensor([2.5], dtype=dtype, device="cuda"), (1, 1, 1), (0, 1, 2), (CU, CU, CU))
+    assert t.nnz == 1 and t.val.tolist() == [2.5] and t.crd(2).tolist() == [0]
+    dup = [torch.zeros(3, dtype=torch.int32, device="cuda")] * 2
+    s = comet.pack(dup, torch.tensor([1.0, 2.0, 4.0], dtype=dtype, device="cuda"), (1, 1), (0, 1), (D, CU), sum_duplicates=True)
+    assert s.nnz == 1 and s.val.tolist() == [7.0]
+    for dims in [(16, 16), (256, 256), (32, 16)]:
+        coords, val = synth.random_coo(dims, min(200, dims[0] * dims[1] // 2), 9)
+        val = val.to(dtype)
+        want = oracle.pack(_np(coords), val.double().numpy(), dims, (1, 0), (D, CU))
+        got = comet.pack([c.cuda() for c in coords], val.cuda(), dims, (1, 0), (D, CU))
+        assert got.pos(1).tolist() == want.pos[1].tolist() and got.crd(1).tolist() == want.crd[1].tolist()
+        assert np.array_equal(got.val.double().cpu().numpy(), want.val)
+
+
 def test_pack_csr_histogram_flag_gives_the_same_tensor():
     dims = (300, 200)
     coords, val = synth.random_coo(dims, 5000, 7)
