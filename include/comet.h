@@ -79,8 +79,9 @@ typedef enum {
  *   COMET_PACK_CSR=1|0          forces / forbids the histogram CSR packing of comet_pack_ex (COMET_PACK_CSR_HISTOGRAM)
  *   COMET_SEG_PARTITION=0       matrix-operand kernels search their tile boundaries themselves (no pre-pass)
  *   COMET_CSF_FORM=fold|expand  root-mode CSF MTTKRP: per-fiber or per-entry form (default: by mean fiber length)
- *   COMET_MTTKRP_HOT_ROWS=0|1   leaf-mode CSF MTTKRP: never / always keep the most popular output rows in shared memory
+ *   COMET_MTTKRP_HOT_ROWS=0|1   per-entry MTTKRP (CSF leaf mode, COO non-root modes): never / always keep the most popular output rows in shared memory
  *                               (default: for R >= 16 and at least 2^20 entries)
+ *   COMET_HOST_CHUNK_BYTES=n    comet_spmm_from_host: bytes per row of a column chunk of B and C (default 256; 0 = one chunk)
  *   COMET_SPMM_LONG_ROWS=0      comet_spmm without the long-row path; COMET_SPMM_LONG_ROW, _LONG_TILE, _PIECE,
  *                               _BLOCK_MB, _BLOCKS, _LONG_CTAS, _LONG_MIN_NNZ, _LONG_MIN_B_MB: its threshold
  *                               (entries), tile and piece sizes, block size / count of B, CTAs of the long-row
