@@ -99,9 +99,10 @@ __global__ void __launch_bounds__(kScatterThreads) mttkrp_coo_scatter_kernel(con
 // adds that copy into the output once, at the end. Which rows are chosen changes the speed only, not the sums.
 constexpr int kHotThreads = 512;
 constexpr int kHotCtas = 2;                        // CTAs per SM
-// Entries per warp and step. The chunks are dealt out round-robin, so the last round is only partly filled: 100 M
-// entries over 9,472 warps take 42 rounds of 256 (2 % idle at the end) but 3 rounds of 4,096 where 2.6 would do
-// (measured: 6.70 / 6.76 / 7.88 ms with 256 / 1,024 / 4,096 entries; 128 entries 6.98 ms: a search per chunk).
+// Entries per warp and step; the warps draw chunk numbers from a counter. Dealt out round-robin instead, the last
+// round is only partly filled: 100 M entries over 9,472 warps take 42 rounds of 256 (2 % idle) but 3 rounds of
+// 4,096 where 2.6 would do (measured, round-robin: 6.70 / 6.76 / 7.88 ms with 256 / 1,024 / 4,096 entries; with the
+// counter 6.43 / 6.44 / 6.45 ms with 256 / 512 / 1,024).
 constexpr int kHotChunk = 256;
 // Shared memory per CTA for the popular rows: 256 rows of 32 columns. Measured on config 5 (leaf frequencies
 // (k + 100)^-1.5 over 200,000 rows): 32 rows 16.6 ms, 128 rows 6.75 to 8.9 ms depending on where the output
@@ -189,7 +190,8 @@ __global__ void __launch_bounds__(kHotThreads, kHotCtas) mttkrp_csf_leaf_hot_ker
                                                                                    const int32_t *__restrict__ fiber_root,
                                                                                    const int32_t *__restrict__ hot_slot,
                                                                                    const int32_t *__restrict__ hot_rows,
-                                                                                   const int32_t *__restrict__ n_hot, int32_t slots) {
+                                                                                   const int32_t *__restrict__ n_hot, int32_t slots,
+                                                                                   unsigned long long *__restrict__ next_chunk) {
   extern __shared__ double s_acc[];                // slots x R
   const T *const val = static_cast<const T *>(a.val);
   const T *const A = static_cast<const T *>(a.A), *const B = static_cast<const T *>(a.B);
@@ -198,9 +200,12 @@ __global__ void __launch_bounds__(kHotThreads, kHotCtas) mttkrp_csf_leaf_hot_ker
   __syncthreads();
   const unsigned full = 0xffffffffu;
   const int lane = threadIdx.x & 31;
-  const int64_t warps = (int64_t)gridDim.x * (kHotThreads / 32);
   const int64_t chunks = (a.N + kHotChunk - 1) / kHotChunk;
-  for (int64_t chunk = (int64_t)blockIdx.x * (kHotThreads / 32) + (threadIdx.x >> 5); chunk < chunks; chunk += warps) {
+  while (true) {                                   // chunks are handed out as the warps ask: no partly filled last round
+    unsigned long long ticket = 0;
+    if (lane == 0) ticket = atomicAdd(next_chunk, 1ull);
+    const int64_t chunk = (int64_t)__shfl_sync(full, ticket, 0);
+    if (chunk >= chunks) break;
     const int64_t p0 = chunk * kHotChunk;
     const int64_t p1 = p0 + kHotChunk < a.N ? p0 + kHotChunk : a.N;
     int64_t fw = 0;                                // CSF: the window of fibers fw .. fw + 31, one per lane
@@ -290,14 +295,16 @@ static comet_status_t entries_hot(Context *ctx, const ScatterArgs &a, bool coo, 
   if (slots > rows) slots = rows;
   if (slots < 1) return COMET_OK;
   const int32_t *out_crd = coo ? a.crd0 : a.crd2;
-  // counts[rows] | bins[kCountBins] | slots in use | threshold: one block, zero-filled at once
-  int32_t *counts = (int32_t *)ctx_alloc(ctx, (size_t)(rows + kCountBins + 2) * 4, stream);
+  // counts[rows] | bins[kCountBins] | slots in use | threshold | chunk counter (64 bits, 8-byte aligned): one block,
+  // zero-filled at once
+  const int64_t words = align_up((size_t)(rows + kCountBins + 2), 2) + 2;
+  int32_t *counts = (int32_t *)ctx_alloc(ctx, (size_t)words * 4, stream);
   int32_t *hot_slot = (int32_t *)ctx_alloc(ctx, (size_t)rows * 4, stream);
   int32_t *hot_rows = (int32_t *)ctx_alloc(ctx, (size_t)slots * 4, stream);
   int32_t *fiber_root = coo ? nullptr : (int32_t *)ctx_alloc(ctx, (size_t)a.F * 4, stream);
   comet_status_t st = (counts && hot_slot && hot_rows && (coo || fiber_root)) ? COMET_OK : COMET_ERR_ALLOC;
   if (st == COMET_OK) {
-    cudaError_t e = cudaMemsetAsync(counts, 0, (size_t)(rows + kCountBins + 2) * 4, stream);
+    cudaError_t e = cudaMemsetAsync(counts, 0, (size_t)words * 4, stream);
     if (e != cudaSuccess) st = cuda_fail(ctx, e);
   }
   if (st == COMET_OK) {
@@ -319,7 +326,8 @@ static comet_status_t entries_hot(Context *ctx, const ScatterArgs &a, bool coo, 
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) st = cuda_fail(ctx, e);
     if (st == COMET_OK) {
-      kernel<<<kHotCtas * kSmCount, kHotThreads, smem, stream>>>(a, fiber_root, hot_slot, hot_rows, n_hot, (int32_t)slots);
+      kernel<<<kHotCtas * kSmCount, kHotThreads, smem, stream>>>(a, fiber_root, hot_slot, hot_rows, n_hot, (int32_t)slots,
+                                                                 reinterpret_cast<unsigned long long *>(counts + words - 2));
       ctx->launches += 1;
       e = cudaGetLastError();
       if (e != cudaSuccess) st = cuda_fail(ctx, e);
