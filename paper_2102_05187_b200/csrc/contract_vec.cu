@@ -189,10 +189,11 @@ __global__ void __launch_bounds__(kBlockThreads) seg_partition_kernel(const int3
 // A heavy segment spans hundreds of tiles, so the run is read eight tiles at a time with all loads in
 // flight together (the additions keep the tile order).
 template <class T>
-__global__ void carry_fixup_kernel(const double *__restrict__ carry_val, const int32_t *__restrict__ carry_seg,
-                                   int64_t num_tiles, int32_t R, int32_t carry_ld, T *__restrict__ C,
-                                   int64_t ldc, const int32_t *__restrict__ out_row) {
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+__device__ __forceinline__ void carry_fixup_role(int64_t block, const double *__restrict__ carry_val,
+                                                 const int32_t *__restrict__ carry_seg, int64_t num_tiles, int32_t R,
+                                                 int32_t carry_ld, T *__restrict__ C, int64_t ldc,
+                                                 const int32_t *__restrict__ out_row) {
+  const int64_t idx = block * blockDim.x + threadIdx.x;
   const int64_t tile = idx / R;
   const int32_t c = (int32_t)(idx - tile * R);
   if (tile >= num_tiles) return;
@@ -218,6 +219,26 @@ __global__ void carry_fixup_kernel(const double *__restrict__ carry_val, const i
   }
   const int64_t row = out_row ? (int64_t)out_row[seg] : (int64_t)seg;
   C[row * ldc + c] = (T)((double)C[row * ldc + c] + sum);
+}
+
+template <class T>
+__global__ void __launch_bounds__(kBlockThreads) carry_fixup_kernel(const double *__restrict__ carry_val,
+                                                                    const int32_t *__restrict__ carry_seg, int64_t num_tiles,
+                                                                    int32_t R, int32_t carry_ld, T *__restrict__ C, int64_t ldc,
+                                                                    const int32_t *__restrict__ out_row) {
+  carry_fixup_role<T>(blockIdx.x, carry_val, carry_seg, num_tiles, R, carry_ld, C, ldc, out_row);
+}
+
+// SpMM with the long-row path: both fix-ups in one launch. They read different scratch and write different rows
+// of C (the general tiles leave the long rows out, so no carry names one), so the first `heavy_blocks` CTAs add
+// the long rows' slots while the others add the carries.
+template <class T>
+__global__ void __launch_bounds__(kBlockThreads) spmm_fixups_kernel(const HeavyArgs h, int heavy_blocks,
+                                                                    const double *__restrict__ carry_val,
+                                                                    const int32_t *__restrict__ carry_seg, int64_t num_tiles,
+                                                                    int32_t R, int32_t carry_ld, T *__restrict__ C, int64_t ldc) {
+  if ((int)blockIdx.x < heavy_blocks) heavy_fixup_role<T>(h, (int)blockIdx.x, heavy_blocks);
+  else carry_fixup_role<T>((int64_t)blockIdx.x - heavy_blocks, carry_val, carry_seg, num_tiles, R, carry_ld, C, ldc, nullptr);
 }
 
 void carry_fixup_launch(int dtype, const double *carry_val, const int32_t *carry_seg, int64_t num_tiles, int32_t R,
@@ -303,9 +324,14 @@ static comet_status_t launch_one(Context *ctx, SegGatherArgs a, HeavyArgs *heavy
   a.carry_seg = (int32_t *)(scratch + heavy_bytes + val_bytes);
   if (part_bytes) {
     int32_t *part = (int32_t *)(scratch + heavy_bytes + carry_bytes(a.num_tiles, a.carry_ld));
-    seg_partition_kernel<<<(unsigned)ceil_div(a.num_tiles + 1, kBlockThreads), kBlockThreads, 0, stream>>>(a.seg_end, a.M, a.N,
-                                                                                                         a.tile_items, a.num_tiles, part);
-    COMET_LAUNCH_CHECK(ctx);
+    if (heavy_bytes) {                                     // a role of the long-row path's pieces launch
+      h.part_seg_end = a.seg_end; h.part_M = a.M; h.part_N = a.N; h.part_tiles = a.num_tiles;
+      h.part_tile_items = a.tile_items; h.part = part;
+    } else {
+      seg_partition_kernel<<<(unsigned)ceil_div(a.num_tiles + 1, kBlockThreads), kBlockThreads, 0, stream>>>(a.seg_end, a.M, a.N,
+                                                                                                           a.tile_items, a.num_tiles, part);
+      COMET_LAUNCH_CHECK(ctx);
+    }
     a.part = part;
   }
   const int64_t blocks = ceil_div(a.num_tiles, WORKERS);
@@ -317,10 +343,10 @@ static comet_status_t launch_one(Context *ctx, SegGatherArgs a, HeavyArgs *heavy
       a.skip_len = h.threshold;
       st = launch_mapped<T, LPN, CPL, VEC, false, true>(ctx, a, h, blocks, stream);
       if (st != COMET_OK) return st;
-      st = spmm_heavy_finish(ctx, h, sizeof(T) == 4 ? COMET_F32 : COMET_F64, stream);
-      if (st != COMET_OK) return st;
-      carry_fixup_launch(sizeof(T) == 4 ? COMET_F32 : COMET_F64, a.carry_val, a.carry_seg, a.num_tiles, a.R, a.carry_ld, a.C,
-                         a.ldc, a.out_row, stream);
+      const int heavy_blocks = kSmCount * 8;
+      const unsigned fix_blocks = (unsigned)(heavy_blocks + ceil_div(a.num_tiles * a.R, kBlockThreads));
+      spmm_fixups_kernel<T><<<fix_blocks, kBlockThreads, 0, stream>>>(h, heavy_blocks, a.carry_val, a.carry_seg, a.num_tiles,
+                                                                     (int32_t)a.R, a.carry_ld, static_cast<T *>(a.C), a.ldc);
       COMET_LAUNCH_CHECK(ctx);
       return COMET_OK;
     }

@@ -115,6 +115,14 @@ __global__ void __launch_bounds__(kBlockThreads) heavy_count_kernel(const HeavyA
 // Pass 2: numbers the long rows in ascending order, cuts each into its pieces (one binary search per block
 // boundary, a warp per row) and counts the tiles of every phase.
 __global__ void __launch_bounds__(kBlockThreads) heavy_pieces_kernel(const HeavyArgs a) {
+  if ((int)blockIdx.x >= a.num_scan_ctas) {                    // second role: a thread per boundary of the general tiles
+    const int64_t t = (int64_t)(blockIdx.x - a.num_scan_ctas) * kBlockThreads + threadIdx.x;
+    if (t > a.part_tiles) return;
+    const int64_t total = a.part_M + a.part_N;
+    const int64_t d = t * a.part_tile_items < total ? t * a.part_tile_items : total;
+    a.part[t] = (int32_t)merge_path_segments(a.part_seg_end, a.part_M, a.part_N, d);
+    return;
+  }
   __shared__ int32_t warp_sums[kBlockThreads / 32];
   __shared__ int32_t local_h[kScanCta];
   __shared__ int32_t local_n, is_last;
@@ -245,47 +253,6 @@ __global__ void __launch_bounds__(kBlockThreads) heavy_tiles_kernel(const HeavyA
   }
 }
 
-// C[row, :] = the sum of the row's slots, a long row per CTA and step. The 256 threads are G groups of R columns
-// (G = 256 / R, at least 1); group g adds the slots g, g + G, g + 2G, ... in that order (up to sixteen loads in
-// flight), and the groups' sums are then added in group order: a fixed order, so results stay bit-identical from
-// run to run.
-template <class T>
-__global__ void __launch_bounds__(kBlockThreads) heavy_fixup_kernel(const HeavyArgs a) {
-  __shared__ double s_part[kBlockThreads];
-  const int32_t H = __ldcg(a.counters + 0);
-  T *C = static_cast<T *>(a.C);
-  const int R = a.R;
-  const int G = R < kBlockThreads ? kBlockThreads / R : 1;      // R is a power of two here (the shapes of the long-row path)
-  const int g = threadIdx.x / R;
-  for (int32_t h = blockIdx.x; h < H; h += gridDim.x) {
-    const int32_t n = a.row_nt[h];
-    for (int c = threadIdx.x % R; c < R; c += kBlockThreads) {  // one sweep unless R > 256
-      const double *src = a.carry_val + (int64_t)a.row_slot0[h] * a.carry_ld + c;
-      double sum = 0.0;
-      int32_t t = g;
-      for (; t + 15 * G < n; t += 16 * G) {
-        double v[16];
-#pragma unroll
-        for (int u = 0; u < 16; ++u) v[u] = __ldcs(src + (int64_t)(t + u * G) * a.carry_ld);
-#pragma unroll
-        for (int u = 0; u < 16; ++u) sum += v[u];
-      }
-      for (; t < n; t += G) sum += __ldcs(src + (int64_t)t * a.carry_ld);
-      if (G > 1) {
-        __syncthreads();                                        // the sums of the row before have been read
-        s_part[threadIdx.x] = sum;
-        __syncthreads();
-        if (g == 0) {
-          for (int x = 1; x < G; ++x) sum += s_part[x * R + c];
-          C[(int64_t)a.hrow[h] * a.ldc + c] = (T)sum;
-        }
-      } else {
-        C[(int64_t)a.hrow[h] * a.ldc + c] = (T)sum;
-      }
-    }
-  }
-}
-
 static int env_int(const char *name, int dflt) {
   const char *e = getenv(name);
   return e ? atoi(e) : dflt;
@@ -357,16 +324,10 @@ comet_status_t spmm_heavy_prepare(Context *ctx, HeavyArgs *args, const int32_t *
   // the tickets and the tile cursor must start at zero; the scratch is shared with other calls, so clear them here
   COMET_CUDA_TRY(ctx, cudaMemsetAsync(a.counters, 0, 16 * 4, stream));
   heavy_count_kernel<<<a.num_scan_ctas, kBlockThreads, 0, stream>>>(a);
-  heavy_pieces_kernel<<<a.num_scan_ctas, kBlockThreads, 0, stream>>>(a);
+  const int64_t part_ctas = a.part ? ceil_div(a.part_tiles + 1, (int64_t)kBlockThreads) : 0;
+  heavy_pieces_kernel<<<(unsigned)(a.num_scan_ctas + part_ctas), kBlockThreads, 0, stream>>>(a);
   heavy_tiles_kernel<<<kSmCount * 2, kBlockThreads, 0, stream>>>(a);
   COMET_LAUNCHED(ctx, 3);
-  return COMET_OK;
-}
-
-comet_status_t spmm_heavy_finish(Context *ctx, const HeavyArgs &a, int dtype, cudaStream_t stream) {
-  if (dtype == COMET_F32) heavy_fixup_kernel<float><<<kSmCount * 8, kBlockThreads, 0, stream>>>(a);
-  else heavy_fixup_kernel<double><<<kSmCount * 8, kBlockThreads, 0, stream>>>(a);
-  COMET_LAUNCH_CHECK(ctx);
   return COMET_OK;
 }
 

@@ -36,6 +36,11 @@ struct HeavyArgs {
   void *C;
   int64_t ldc;
   int32_t R;
+  // the tile boundaries of the GENERAL tiles (merge-path splits), computed by extra CTAs of the pieces launch
+  const int32_t *part_seg_end;
+  int64_t part_M, part_N, part_tiles;
+  int32_t part_tile_items;
+  int32_t *part;
 };
 
 // A tile of one row: no segment ends, only the window of gathers and the sum.
@@ -95,12 +100,55 @@ __device__ __forceinline__ void heavy_role(const HeavyArgs &a, unsigned char *sm
 }
 
 // Host side (spmm_heavy.cu). plan: decides whether the path applies (returns 0 if not) and how much scratch it
-// needs; prepare: lays the arrays out in `scratch` and runs the three analysis kernels; finish: the fix-up that
-// writes the long rows of C, after the gather kernel.
+// needs; prepare: lays the arrays out in `scratch` and runs the three analysis kernels. The fix-up that writes the
+// long rows of C after the gather kernel is heavy_fixup_role below.
 size_t spmm_heavy_plan(int dtype, int64_t M, int64_t N, int64_t cols, const void *B, int64_t ldb, int64_t R, const void *C,
                        int64_t ldc, int32_t min_threshold, HeavyArgs *out);
 comet_status_t spmm_heavy_prepare(Context *ctx, HeavyArgs *args, const int32_t *pos, const int32_t *crd, const void *val,
                                   char *scratch, cudaStream_t stream);
-comet_status_t spmm_heavy_finish(Context *ctx, const HeavyArgs &a, int dtype, cudaStream_t stream);
+
+
+// The long rows' fix-up, a role of the fix-up launch (contract_vec.cu; `block` of `blocks` CTAs play it):
+// C[row, :] = the sum of the row's slots, a long row per CTA and step. The 256 threads are G groups of R columns
+// (G = 256 / R, at least 1); group g adds the slots g, g + G, g + 2G, ... in that order (up to sixteen loads in
+// flight), and the groups' sums are then added in group order: a fixed order, so results stay bit-identical from
+// run to run.
+template <class T>
+__device__ __forceinline__ void heavy_fixup_role(const HeavyArgs &a, int block, int blocks) {
+  __shared__ double s_part[kBlockThreads];
+  const int32_t H = __ldcg(a.counters + 0);
+  T *C = static_cast<T *>(a.C);
+  const int R = a.R;
+  const int G = R < kBlockThreads ? kBlockThreads / R : 1;      // R is a power of two here (the shapes of the long-row path)
+  const int g = threadIdx.x / R;
+  for (int32_t h = block; h < H; h += blocks) {
+    const int32_t n = a.row_nt[h];
+    for (int c = threadIdx.x % R; c < R; c += kBlockThreads) {  // one sweep unless R > 256
+      const double *src = a.carry_val + (int64_t)a.row_slot0[h] * a.carry_ld + c;
+      double sum = 0.0;
+      int32_t t = g;
+      for (; t + 15 * G < n; t += 16 * G) {
+        double v[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) v[u] = __ldcs(src + (int64_t)(t + u * G) * a.carry_ld);
+#pragma unroll
+        for (int u = 0; u < 16; ++u) sum += v[u];
+      }
+      for (; t < n; t += G) sum += __ldcs(src + (int64_t)t * a.carry_ld);
+      if (G > 1) {
+        __syncthreads();                                        // the sums of the row before have been read
+        s_part[threadIdx.x] = sum;
+        __syncthreads();
+        if (g == 0) {
+          for (int x = 1; x < G; ++x) sum += s_part[x * R + c];
+          C[(int64_t)a.hrow[h] * a.ldc + c] = (T)sum;
+        }
+      } else {
+        C[(int64_t)a.hrow[h] * a.ldc + c] = (T)sum;
+      }
+    }
+  }
+}
+
 
 }  // namespace comet
