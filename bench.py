@@ -478,7 +478,7 @@ def run_ours(args):
     roofline = roofline_obj(
         spmm_bytes, spmm_med, peak, peak_kind,
         "comet_spmm: seg_gather_kernel<32,1,2> with two CTA roles (long rows by column blocks of B | general tiles), "
-        "3 analysis kernels, 2 fix-ups", traffic=traffic, traffic_source=traffic_info,
+        "3 analysis kernels, 1 two-role fix-up launch", traffic=traffic, traffic_source=traffic_info,
         note="gather-bound: the 64-column rows of B (537 MB, 4x the L2) are gathered nnz times; the long rows are "
              "processed by column blocks so that their gathers hit L2, the short rows still pull their rows from DRAM")
 
