@@ -171,3 +171,34 @@ def test_scaled_workload_with_long_rows(force_long_rows):
     C = torch.full((case.dims[0], case.R), float("nan"), dtype=torch.float64, device="cuda")
     comet.spmm(A, dev(B), C)
     assert_close(C, want, norm, what="spmm long rows, scaled workload")
+
+
+@pytest.mark.parametrize("tile_items", [16, 64, 100])
+@pytest.mark.parametrize("R", [2, 16, 40])
+def test_rows_around_the_length_that_one_tile_takes_whole(tile_items, R, monkeypatch):
+    """Without the long-row role, a row of at most a quarter tile is processed whole by the tile that holds its
+    end marker and longer rows are split with carries: rows of exactly that length, one less, one more, a whole
+    tile and more, with runs of empty rows between them and at both ends of the matrix."""
+    monkeypatch.setenv("COMET_SPMM_LONG_ROWS", "0")
+    monkeypatch.setenv("COMET_TILE_ITEMS", str(tile_items))
+    q = tile_items // 4
+    rng = np.random.default_rng(tile_items + R)
+    ln = []
+    for _ in range(40):
+        ln += [q - 1, 0, q, q + 1, 0, 0, int(rng.integers(0, q + 3)), tile_items, 1, 2 * tile_items + 3, 0, int(rng.integers(1, 4))]
+    ln = [0, 0] + [max(0, x) for x in ln] + [0, q, 0]
+    cols = 3 * tile_items + 50
+    c, v = matrix_from_row_lengths(np.array(ln), cols, 5)
+    dims = (len(ln), cols)
+    B = synth.random_dense((cols, R), 8).numpy()
+    want, norm = oracle.spmm(c, v, dims, B)
+    A = upload_packed(oracle.pack(c, v, dims, (0, 1), (D, CU)))
+    C = torch.full((dims[0], R), float("nan"), dtype=torch.float64, device="cuda")
+    comet.spmm(A, dev(B), C)
+    assert_close(C, want, norm, what=f"spmm tile {tile_items} R={R}")
+    x = B[:, 0].copy()
+    y = torch.full((dims[0],), float("nan"), dtype=torch.float64, device="cuda")
+    comet.spmv(A, dev(x), y)
+    wy, ny = oracle.spmv(c, v, dims, x)
+    assert_close(y, wy, ny, what=f"spmv tile {tile_items}")
+
